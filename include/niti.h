@@ -1,0 +1,184 @@
+/*
+ * niti.h -- C ABI of the B200 (sm_100a) library for NITI integer training
+ * ("NITI: Training Integer Neural Networks Using Integer-only Arithmetic",
+ * arXiv 2009.13108).
+ *
+ * Every tensor pointer below is a DEVICE pointer owned by the caller unless a
+ * function says otherwise.  The library allocates no device memory after
+ * niti_create(); scratch comes from the caller's workspace `ws` (size from
+ * niti_workspace_bytes(), 256-byte aligned).  All work is enqueued on the
+ * caller's stream (`stream` is a cudaStream_t passed as void*) and the calls
+ * return without synchronising; one workspace must not be used by two calls
+ * that can overlap on the GPU.
+ *
+ * Number format (Section 3.1): a tensor is an int8 payload plus ONE shared
+ * exponent s, value = payload * 2^s.  Exponents and effective bit-widths live
+ * in device int32 scalars so that a whole training step needs no host sync.
+ * The payload value -128 never appears in any output.
+ *
+ * Layouts: activations / errors are row-major [M][K] (fully connected) or
+ * NHWC [B][H][W][C] (convolution); weights are [N_out][K_in] or
+ * [Cout][R][S][Cin]; gradients have the layout of the weights.
+ *
+ * Rounding (Section 3.4): after each matrix multiply the int32 accumulator
+ * tensor V is reduced to its effective bit-width b = bit_length(max|V|)
+ * (Section 3.2), the binary point is bp = max(0, b - mbits) (Algorithm 1),
+ * and every element is rounded by Algorithm 3 (round_mode 0, pseudo-
+ * stochastic: the top half of the discarded bits is compared with the bottom
+ * half) or to nearest (round_mode 1, magnitude half-up), on the magnitude
+ * with the sign re-applied, saturating at 2^mbits - 1.  mbits is 7 for
+ * activations and errors and m_u (1..7) for weight gradients.
+ *
+ * Contract on accumulators: the caller guarantees |sum| < 2^31 for every
+ * output (always true when the contraction length is <= 133144).
+ *
+ * Return value: NITI_OK or an error code; nothing is enqueued on error.
+ */
+#ifndef NITI_H_
+#define NITI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NITI_OK 0
+#define NITI_ERR_ARG 1       /* null pointer, non-positive size, bad flag          */
+#define NITI_ERR_SHAPE 2     /* shape not supported by this build                  */
+#define NITI_ERR_WORKSPACE 3 /* ws is NULL, misaligned or smaller than required    */
+#define NITI_ERR_RANGE 4     /* exponent outside the supported domain              */
+#define NITI_ERR_CUDA 5      /* a CUDA call failed; see niti_last_error()          */
+#define NITI_ERR_DEVICE 6    /* a kernel raised the device status word             */
+
+#define NITI_ROUND_PSR 0
+#define NITI_ROUND_NEAREST 1
+
+/* op ids for niti_workspace_bytes(); dims as listed */
+#define NITI_OP_LINEAR_FWD 0  /* dims = {M, N, K}                 */
+#define NITI_OP_LINEAR_BWD 1  /* dims = {M, N, K}                 */
+#define NITI_OP_CONV_FWD 2    /* dims = {B, H, W, Cin, Cout, R, S, pad} */
+#define NITI_OP_CONV_DGRAD 3  /* same                              */
+#define NITI_OP_CONV_WGRAD 4  /* same                              */
+#define NITI_OP_INT_XENT 5    /* dims = {B, N}                    */
+
+/* device status bits returned by niti_check() */
+#define NITI_DEV_TIMEOUT 1u      /* a bounded wait inside a kernel gave up     */
+#define NITI_DEV_EXP_RANGE 2u    /* an exponent left the int8 range            */
+#define NITI_DEV_XENT_RANGE 4u   /* s_a outside [-22, 24] in niti_int_xent     */
+#define NITI_DEV_BAD_LABEL 8u    /* a label outside [0, N)                     */
+
+typedef struct niti_ctx niti_ctx;
+
+/* Creates a context on CUDA device `device` (the device must be sm_100).
+ * Allocates a few bytes of device memory for the status word.  The caller
+ * destroys it with niti_destroy().  Not thread-safe per context. */
+int niti_create(niti_ctx **out, int device);
+int niti_destroy(niti_ctx *ctx);
+
+/* Text of the last host-side error of this context (owned by the context). */
+const char *niti_last_error(niti_ctx *ctx);
+
+/* Synchronises `stream`, reads and clears the device status word; returns
+ * NITI_OK, NITI_ERR_CUDA or NITI_ERR_DEVICE (bits in *status if non-NULL). */
+int niti_check(niti_ctx *ctx, void *stream, uint32_t *status);
+
+/* Bytes of workspace the op needs for these dims (0 on bad arguments). */
+size_t niti_workspace_bytes(int op, const int64_t *dims, int ndims);
+
+/* Selects the matrix-multiply engine: 0 = automatic (tensor cores whenever
+ * the shape allows, default), 1 = force the plain CUDA-core kernels (used by
+ * tests to cross-check the two engines).  Returns the previous value. */
+int niti_set_engine(niti_ctx *ctx, int engine);
+
+/* Number of kernels / memsets this context has enqueued so far. */
+uint64_t niti_launch_count(niti_ctx *ctx);
+/* Of those, launches of the tensor-core (tcgen05) matrix-multiply kernel. */
+uint64_t niti_tc_launch_count(niti_ctx *ctx);
+
+/* Fully connected forward (Algorithm 1, forward loop; Section 3.2):
+ *   acc[m][n] = sum_k a[m][k] * w[n][k];  b = B(acc);  bp = max(0, b - 7);
+ *   out = Round(acc, bp) (then max(.,0) if relu);  *s_out = *s_a + *s_w + bp.
+ * a [M][K], w [N][K], out [M][N]; s_a, s_w, s_out, b_out device scalars
+ * (s_out, b_out may be NULL). b is taken before the ReLU. */
+int niti_linear_fwd(niti_ctx *ctx, void *stream, const int8_t *a, const int32_t *s_a,
+                    const int8_t *w, const int32_t *s_w, int8_t *out, int32_t *s_out,
+                    int32_t *b_out, int M, int N, int K, int relu, int round_mode, void *ws,
+                    size_t ws_bytes);
+
+/* Fully connected backward (Algorithm 1, reverse loop; Section 3.3):
+ *   g32[n][k] = sum_m e[m][n] * a[m][k]  -> g = Round(g32, max(0, B(g32) - m_u))
+ *   e32[m][k] = sum_n e[m][n] * w[n][k]  -> e_prev = Round(e32, max(0, B(e32) - 7))
+ * Both use w as it is on entry (the update is a separate call).  e_prev may be
+ * NULL (first layer).  relu_mask_src, if not NULL, is an int8 [M][K] tensor
+ * (the ReLU output that fed this layer); e_prev is zeroed where it is <= 0.
+ * b_e, b_g: device scalars, may be NULL. */
+int niti_linear_bwd(niti_ctx *ctx, void *stream, const int8_t *a, const int8_t *e, const int8_t *w,
+                    int8_t *e_prev, const int8_t *relu_mask_src, int8_t *g, int32_t *b_e,
+                    int32_t *b_g, int M, int N, int K, int m_u, int round_mode, void *ws,
+                    size_t ws_bytes);
+
+/* Convolution forward as an implicit matrix multiply (Section 3.2), stride 1,
+ * zero padding `pad`, R x S taps:
+ *   acc[b][i][j][co] = sum_{r,s,ci} x[b][i+r-pad][j+s-pad][ci] * w[co][r][s][ci]
+ * followed by the same bit-width / shift / round / exponent rule as
+ * niti_linear_fwd.  x [B][H][W][Cin], y [B][H+2pad-R+1][W+2pad-S+1][Cout]. */
+int niti_conv_fwd(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x,
+                  const int8_t *w, const int32_t *s_w, int8_t *y, int32_t *s_y, int32_t *b_y, int B,
+                  int H, int W, int Cin, int Cout, int R, int S, int pad, int relu, int round_mode,
+                  void *ws, size_t ws_bytes);
+
+/* Error back-propagation through the convolution (Algorithm 1, reverse loop):
+ *   e32[b][i][j][ci] = sum_{r,s,co} e[b][i-r+pad][j-s+pad][co] * w[co][r][s][ci]
+ * rounded to 7 bits.  H, W are the INPUT sizes of the forward convolution;
+ * e has the forward output's shape.  relu_mask_src as in niti_linear_bwd
+ * (shape of e_prev). */
+int niti_conv_dgrad(niti_ctx *ctx, void *stream, const int8_t *e, const int8_t *w, int8_t *e_prev,
+                    const int8_t *relu_mask_src, int32_t *b_e, int B, int H, int W, int Cin,
+                    int Cout, int R, int S, int pad, int round_mode, void *ws, size_t ws_bytes);
+
+/* Weight gradient of the convolution (Algorithm 1, reverse loop; Section 3.3):
+ *   g32[co][r][s][ci] = sum_{b,i,j} e[b][i][j][co] * x[b][i+r-pad][j+s-pad][ci]
+ * rounded to m_u bits (values in [-(2^m_u - 1), 2^m_u - 1] in an int8). */
+int niti_conv_wgrad(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
+                    int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
+                    int m_u, int round_mode, void *ws, size_t ws_bytes);
+
+/* Integer cross-entropy gradient (Section 3.5, Eq. 1-4).  Per sample r:
+ *   e32[r][i] = T_i - [i == labels[r]] * sum_j T_j
+ * with T_i = 2^(1-2s) + a_i 2^(1-s) + a_i^2 when s = *s_a <= -7 (Eq. 2), else
+ * T_i = 1 << max(0, xh_i - p), xh_i = (47274 a_i) >> (15 - s) (arithmetic
+ * shift; a left shift if 15 - s < 0), p = the smallest xh_i greater than
+ * max(xh) - 10 (Eq. 3-4).  The whole [B][N] tensor is then rounded to 7 bits
+ * with one shared binary point.  a [B][N] int8, labels [B] int32, e [B][N].
+ * n_correct (may be NULL): number of rows whose first arg-max equals the
+ * label.  *s_a outside [-22, 24] or a bad label sets the device status word
+ * and writes zeros.  N <= 65536. */
+int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const int32_t *s_a,
+                  const int32_t *labels, int8_t *e, int32_t *b_e, int32_t *n_correct, int B, int N,
+                  int round_mode, void *ws, size_t ws_bytes);
+
+/* Weight update (Algorithm 1 last line; Section 3.3): w <- clamp(w - g, -127, 127), in place. */
+int niti_int_sgd_update(niti_ctx *ctx, void *stream, int8_t *w, const int8_t *g, int64_t n);
+
+/* Support ops on int8 tensors between the layers (implied by the paper's
+ * networks, Section 4); exponents are unchanged.
+ *   relu_fwd: y = max(x, 0) (y may alias x).
+ *   relu_bwd: e_in = e_out where y > 0 else 0 (e_in may alias e_out).
+ *   maxpool2_fwd: 2x2 window, stride 2, NHWC, H and W even.
+ *   maxpool2_bwd: routes e_out to the first maximum of each window in
+ *     (row, col) order, zero elsewhere; if relu != 0 the result is also zeroed
+ *     where x <= 0 (x is the pooled ReLU output). */
+int niti_relu_fwd(niti_ctx *ctx, void *stream, const int8_t *x, int8_t *y, int64_t n);
+int niti_relu_bwd(niti_ctx *ctx, void *stream, const int8_t *y, const int8_t *e_out, int8_t *e_in,
+                  int64_t n);
+int niti_maxpool2_fwd(niti_ctx *ctx, void *stream, const int8_t *x, int8_t *y, int B, int H, int W,
+                      int C);
+int niti_maxpool2_bwd(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e_out,
+                      int8_t *e_in, int B, int H, int W, int C, int relu);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NITI_H_ */

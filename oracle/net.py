@@ -63,7 +63,8 @@ def oracle_train_step(net, x, labels, state: OracleNetState, round_mode=ref.ROUN
             # a_in is the ReLU output that was pooled: route to the arg-max, then ReLU mask
             e = ref.maxpool2_bwd(a_in, e.reshape(a_in.shape[0], a_in.shape[1] // 2,
                                                  a_in.shape[2] // 2, a_in.shape[3]))
-            e = ref.relu_bwd(a_in, e)
+            if li > 0 and net.layers[li - 1].get("relu"):
+                e = ref.relu_bwd(a_in, e)
             continue
         wi -= 1
         w = state.weights[wi]

@@ -1,0 +1,261 @@
+// C-ABI entry points of the NITI library: argument checks, engine selection, and the
+// accumulate -> bit-width -> shift-and-round sequence of Algorithm 1 for each layer op.
+#include "niti_common.cuh"
+
+int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr);
+
+extern "C" int niti_create(niti_ctx **out, int device) {
+  if (!out) return NITI_ERR_ARG;
+  *out = nullptr;
+  niti_ctx *ctx = new niti_ctx();
+  memset(ctx, 0, sizeof(*ctx));
+  ctx->device = device;
+  cudaDeviceProp prop;
+  cudaError_t e = cudaSetDevice(device);
+  if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, device);
+  if (e != cudaSuccess) {
+    delete ctx;
+    return NITI_ERR_CUDA;
+  }
+  if (prop.major != 10) {   // the kernels are built for sm_100a only
+    delete ctx;
+    return NITI_ERR_SHAPE;
+  }
+  ctx->sm_count = prop.multiProcessorCount;
+  e = cudaMalloc(&ctx->d_status, 256);
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
+  if (e != cudaSuccess) {
+    delete ctx;
+    return NITI_ERR_CUDA;
+  }
+  cudaDriverEntryPointQueryResult qres;
+  void *fn = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+      qres == cudaDriverEntryPointSuccess)
+    ctx->encode_tiled = fn;
+  *out = ctx;
+  return NITI_OK;
+}
+
+extern "C" int niti_destroy(niti_ctx *ctx) {
+  if (!ctx) return NITI_ERR_ARG;
+  cudaFree(ctx->d_status);
+  delete ctx;
+  return NITI_OK;
+}
+
+extern "C" const char *niti_last_error(niti_ctx *ctx) { return ctx ? ctx->err : "null context"; }
+
+extern "C" int niti_set_engine(niti_ctx *ctx, int engine) {
+  if (!ctx) return -1;
+  int old = ctx->engine;
+  ctx->engine = engine;
+  return old;
+}
+
+extern "C" uint64_t niti_launch_count(niti_ctx *ctx) { return ctx ? ctx->launches : 0; }
+extern "C" uint64_t niti_tc_launch_count(niti_ctx *ctx) { return ctx ? ctx->tc_launches : 0; }
+
+extern "C" int niti_check(niti_ctx *ctx, void *stream, uint32_t *status) {
+  if (!ctx) return NITI_ERR_ARG;
+  uint32_t h = 0;
+  NITI_CUDA_TRY(ctx, cudaStreamSynchronize((cudaStream_t)stream));
+  NITI_CUDA_TRY(ctx, cudaMemcpy(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost));
+  if (h) NITI_CUDA_TRY(ctx, cudaMemset(ctx->d_status, 0, sizeof(h)));
+  if (status) *status = h;
+  if (h) {
+    snprintf(ctx->err, sizeof(ctx->err), "device status word 0x%x", h);
+    return NITI_ERR_DEVICE;
+  }
+  return NITI_OK;
+}
+
+static inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static bool fill_conv(GemmProblem &p, int kind, int B, int H, int W, int Ci, int Co, int R, int S,
+                      int pad) {
+  p.kind = kind;
+  p.B = B; p.H = H; p.W = W; p.Ci = Ci; p.Co = Co; p.R = R; p.S = S; p.pad = pad;
+  p.Ho = H + 2 * pad - R + 1;
+  p.Wo = W + 2 * pad - S + 1;
+  if (p.Ho <= 0 || p.Wo <= 0) return false;
+  if (kind == GK_CONV_FWD) { p.gm = (long long)B * p.Ho * p.Wo; p.gn = Co; p.gk = (long long)R * S * Ci; }
+  else if (kind == GK_CONV_DGRAD) { p.gm = (long long)B * H * W; p.gn = Ci; p.gk = (long long)R * S * Co; }
+  else { p.gm = Co; p.gn = (long long)R * S * Ci; p.gk = (long long)B * p.Ho * p.Wo; }
+  return true;
+}
+
+static void fill_fc(GemmProblem &p, int kind, int M, int N, int K) {
+  memset(&p, 0, sizeof(p));
+  p.kind = kind; p.M = M; p.N = N; p.K = K;
+  if (kind == GK_FC_FWD) { p.gm = M; p.gn = N; p.gk = K; }
+  else if (kind == GK_FC_DGRAD) { p.gm = M; p.gn = K; p.gk = N; }
+  else { p.gm = N; p.gn = K; p.gk = M; }
+}
+
+extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
+  if (!d) return 0;
+  GemmProblem p, p2;
+  memset(&p, 0, sizeof(p));
+  memset(&p2, 0, sizeof(p2));
+  size_t outs = 0, extra = 0;
+  switch (op) {
+    case NITI_OP_LINEAR_FWD:
+      if (nd != 3 || d[0] <= 0 || d[1] <= 0 || d[2] <= 0) return 0;
+      fill_fc(p, GK_FC_FWD, (int)d[0], (int)d[1], (int)d[2]);
+      outs = (size_t)(d[0] * d[1]);
+      extra = niti_tc_scratch_bytes(p);
+      break;
+    case NITI_OP_LINEAR_BWD: {
+      if (nd != 3 || d[0] <= 0 || d[1] <= 0 || d[2] <= 0) return 0;
+      size_t a = (size_t)(d[0] * d[2]), b = (size_t)(d[1] * d[2]);
+      outs = a > b ? a : b;
+      fill_fc(p, GK_FC_DGRAD, (int)d[0], (int)d[1], (int)d[2]);
+      fill_fc(p2, GK_FC_WGRAD, (int)d[0], (int)d[1], (int)d[2]);
+      size_t e1 = niti_tc_scratch_bytes(p), e2 = niti_tc_scratch_bytes(p2);
+      extra = e1 > e2 ? e1 : e2;
+      break;
+    }
+    case NITI_OP_CONV_FWD:
+    case NITI_OP_CONV_DGRAD:
+    case NITI_OP_CONV_WGRAD: {
+      if (nd != 8) return 0;
+      for (int i = 0; i < 7; ++i)
+        if (d[i] <= 0) return 0;
+      int kind = op == NITI_OP_CONV_FWD ? GK_CONV_FWD : (op == NITI_OP_CONV_DGRAD ? GK_CONV_DGRAD : GK_CONV_WGRAD);
+      if (!fill_conv(p, kind, (int)d[0], (int)d[1], (int)d[2], (int)d[3], (int)d[4], (int)d[5], (int)d[6], (int)d[7]))
+        return 0;
+      outs = (size_t)(p.gm * p.gn);
+      extra = niti_tc_scratch_bytes(p);
+      break;
+    }
+    case NITI_OP_INT_XENT:
+      if (nd != 2 || d[0] <= 0 || d[1] <= 0) return 0;
+      return NITI_WS_HEADER + round_up((size_t)(d[0] * d[1]) * 8, 256);
+    default:
+      return 0;
+  }
+  return NITI_WS_HEADER + round_up(outs * 4, 256) + round_up(extra, 256);
+}
+
+static inline bool misaligned16(const void *p) { return ((uintptr_t)p & 15) != 0; }
+
+// One matrix multiply of Algorithm 1 followed by EffectiveBitwidth + ShiftAndRound.
+static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, void *ws, size_t ws_bytes,
+                          size_t need, int8_t *out, int mbits, int round_mode, int relu,
+                          const int8_t *mask, const int32_t *s_a, const int32_t *s_w, int32_t *s_out,
+                          int32_t *b_out) {
+  if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
+    return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+  WsHeader *hdr = (WsHeader *)ws;
+  int32_t *acc = (int32_t *)((char *)ws + NITI_WS_HEADER);
+  size_t acc_bytes = round_up((size_t)(p.gm * p.gn) * 4, 256);
+  void *scratch = (char *)ws + NITI_WS_HEADER + acc_bytes;
+  size_t scratch_bytes = ws_bytes - NITI_WS_HEADER - acc_bytes;
+  NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, sizeof(WsHeader), st));
+  ctx->launches++;
+  int rc = NITI_ERR_SHAPE;
+  if (ctx->engine == 0) rc = niti_tc_gemm(ctx, st, p, acc, hdr, scratch, scratch_bytes);
+  if (rc == NITI_ERR_SHAPE) rc = niti_simt_gemm(ctx, st, p, acc, hdr);
+  if (rc != NITI_OK) return rc;
+  return niti_launch_round(ctx, st, acc, hdr, out, p.gm * p.gn, mbits, round_mode, relu, mask, s_a, s_w,
+                           s_out, b_out);
+}
+
+extern "C" int niti_linear_fwd(niti_ctx *ctx, void *stream, const int8_t *a, const int32_t *s_a,
+                               const int8_t *w, const int32_t *s_w, int8_t *out, int32_t *s_out,
+                               int32_t *b_out, int M, int N, int K, int relu, int round_mode, void *ws,
+                               size_t ws_bytes) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!a || !w || !out || !s_a || !s_w || M <= 0 || N <= 0 || K <= 0 || (round_mode != 0 && round_mode != 1) ||
+      misaligned16(a) || misaligned16(w) || misaligned16(out))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_linear_fwd: bad argument (pointers must be 16-byte aligned)");
+  GemmProblem p;
+  fill_fc(p, GK_FC_FWD, M, N, K);
+  p.p0 = a; p.p1 = w;
+  int64_t dims[3] = {M, N, K};
+  return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes,
+                        niti_workspace_bytes(NITI_OP_LINEAR_FWD, dims, 3), out, 7, round_mode, relu,
+                        nullptr, s_a, s_w, s_out, b_out);
+}
+
+extern "C" int niti_linear_bwd(niti_ctx *ctx, void *stream, const int8_t *a, const int8_t *e,
+                               const int8_t *w, int8_t *e_prev, const int8_t *relu_mask_src, int8_t *g,
+                               int32_t *b_e, int32_t *b_g, int M, int N, int K, int m_u, int round_mode,
+                               void *ws, size_t ws_bytes) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!a || !e || !w || !g || M <= 0 || N <= 0 || K <= 0 || m_u < 1 || m_u > 7 ||
+      (round_mode != 0 && round_mode != 1) || misaligned16(a) || misaligned16(e) || misaligned16(w) ||
+      misaligned16(g) || misaligned16(e_prev) || misaligned16(relu_mask_src))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_linear_bwd: bad argument (pointers must be 16-byte aligned)");
+  int64_t dims[3] = {M, N, K};
+  size_t need = niti_workspace_bytes(NITI_OP_LINEAR_BWD, dims, 3);
+  GemmProblem p;
+  fill_fc(p, GK_FC_WGRAD, M, N, K);
+  p.p0 = e; p.p1 = a;
+  int rc = run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, g, m_u, round_mode, 0, nullptr,
+                          nullptr, nullptr, nullptr, b_g);
+  if (rc != NITI_OK || !e_prev) return rc;
+  fill_fc(p, GK_FC_DGRAD, M, N, K);
+  p.p0 = e; p.p1 = w;
+  return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, e_prev, 7, round_mode, 0,
+                        relu_mask_src, nullptr, nullptr, nullptr, b_e);
+}
+
+static int conv_args_ok(int B, int H, int W, int Ci, int Co, int R, int S, int pad, int round_mode) {
+  return B > 0 && H > 0 && W > 0 && Ci > 0 && Co > 0 && R > 0 && S > 0 && pad >= 0 &&
+         (round_mode == 0 || round_mode == 1);
+}
+
+extern "C" int niti_conv_fwd(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x,
+                             const int8_t *w, const int32_t *s_w, int8_t *y, int32_t *s_y, int32_t *b_y,
+                             int B, int H, int W, int Cin, int Cout, int R, int S, int pad, int relu,
+                             int round_mode, void *ws, size_t ws_bytes) {
+  if (!ctx) return NITI_ERR_ARG;
+  GemmProblem p;
+  memset(&p, 0, sizeof(p));
+  if (!x || !w || !y || !s_x || !s_w || !conv_args_ok(B, H, W, Cin, Cout, R, S, pad, round_mode) ||
+      misaligned16(x) || misaligned16(w) || misaligned16(y) ||
+      !fill_conv(p, GK_CONV_FWD, B, H, W, Cin, Cout, R, S, pad))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_fwd: bad argument (pointers must be 16-byte aligned)");
+  p.p0 = x; p.p1 = w;
+  int64_t dims[8] = {B, H, W, Cin, Cout, R, S, pad};
+  return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes,
+                        niti_workspace_bytes(NITI_OP_CONV_FWD, dims, 8), y, 7, round_mode, relu, nullptr,
+                        s_x, s_w, s_y, b_y);
+}
+
+extern "C" int niti_conv_dgrad(niti_ctx *ctx, void *stream, const int8_t *e, const int8_t *w,
+                               int8_t *e_prev, const int8_t *relu_mask_src, int32_t *b_e, int B, int H,
+                               int W, int Cin, int Cout, int R, int S, int pad, int round_mode, void *ws,
+                               size_t ws_bytes) {
+  if (!ctx) return NITI_ERR_ARG;
+  GemmProblem p;
+  memset(&p, 0, sizeof(p));
+  if (!e || !w || !e_prev || !conv_args_ok(B, H, W, Cin, Cout, R, S, pad, round_mode) || misaligned16(e) ||
+      misaligned16(w) || misaligned16(e_prev) || misaligned16(relu_mask_src) ||
+      !fill_conv(p, GK_CONV_DGRAD, B, H, W, Cin, Cout, R, S, pad))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_dgrad: bad argument (pointers must be 16-byte aligned)");
+  p.p0 = e; p.p1 = w;
+  int64_t dims[8] = {B, H, W, Cin, Cout, R, S, pad};
+  return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes,
+                        niti_workspace_bytes(NITI_OP_CONV_DGRAD, dims, 8), e_prev, 7, round_mode, 0,
+                        relu_mask_src, nullptr, nullptr, nullptr, b_e);
+}
+
+extern "C" int niti_conv_wgrad(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
+                               int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
+                               int m_u, int round_mode, void *ws, size_t ws_bytes) {
+  if (!ctx) return NITI_ERR_ARG;
+  GemmProblem p;
+  memset(&p, 0, sizeof(p));
+  if (!x || !e || !g || m_u < 1 || m_u > 7 || !conv_args_ok(B, H, W, Cin, Cout, R, S, pad, round_mode) ||
+      misaligned16(x) || misaligned16(e) || misaligned16(g) ||
+      !fill_conv(p, GK_CONV_WGRAD, B, H, W, Cin, Cout, R, S, pad))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_wgrad: bad argument (pointers must be 16-byte aligned)");
+  p.p0 = e; p.p1 = x;
+  int64_t dims[8] = {B, H, W, Cin, Cout, R, S, pad};
+  return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes,
+                        niti_workspace_bytes(NITI_OP_CONV_WGRAD, dims, 8), g, m_u, round_mode, 0, nullptr,
+                        nullptr, nullptr, nullptr, b_g);
+}

@@ -1,0 +1,108 @@
+// Shared declarations of the NITI sm_100a library (internal; the public boundary is include/niti.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/niti.h"
+
+struct niti_ctx {
+  int device;
+  int sm_count;
+  int engine;               // 0 auto, 1 force CUDA-core kernels
+  uint32_t *d_status;       // device status word
+  uint64_t launches;
+  uint64_t tc_launches;     // launches of the tensor-core matrix-multiply kernel
+  char err[256];
+  // cuTensorMapEncodeTiled, fetched through the runtime so that libcuda is not a link dependency
+  void *encode_tiled;
+};
+
+#define NITI_WS_HEADER 256  // bytes reserved at the start of every workspace for reduction scalars
+
+// Scalars at the start of a workspace.
+struct WsHeader {
+  unsigned int maxabs32;            // max |acc| of an int32 accumulator tensor
+  unsigned int pad0;
+  unsigned long long maxabs64;      // same for the 64-bit loss accumulators
+  unsigned int tile_counter;        // dynamic tile scheduler / arrival counter
+  unsigned int pad1[3];
+};
+
+#define NITI_CUDA_TRY(ctx, expr)                                                        \
+  do {                                                                                  \
+    cudaError_t e__ = (expr);                                                           \
+    if (e__ != cudaSuccess) {                                                           \
+      snprintf((ctx)->err, sizeof((ctx)->err), "%s failed: %s (%s:%d)", #expr,          \
+               cudaGetErrorString(e__), __FILE__, __LINE__);                            \
+      return NITI_ERR_CUDA;                                                             \
+    }                                                                                   \
+  } while (0)
+
+static inline int niti_fail(niti_ctx *ctx, int code, const char *msg) {
+  if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s", msg);
+  return code;
+}
+
+// ---- rounding arithmetic (Algorithm 3 and round-to-nearest), on the magnitude ----------------
+template <typename U>
+__device__ __forceinline__ U niti_round_mag(U m, int bp, U qmax, int round_mode) {
+  U q = m >> bp;
+  U f = m & ((U(1) << bp) - 1);
+  if (round_mode == NITI_ROUND_PSR) {
+    f >>= (bp & 1);               // odd binary point: the lowest discarded bit is dropped
+    int h = bp >> 1;              // width of each half
+    U top = f >> h;
+    U bot = f & ((U(1) << h) - 1);
+    q += (top > bot) ? 1 : 0;
+  } else {
+    q += (bp > 0 && (f >> (bp - 1))) ? 1 : 0;
+  }
+  return q > qmax ? qmax : q;
+}
+
+__device__ __forceinline__ int niti_round_i32(int x, int bp, unsigned qmax, int round_mode) {
+  unsigned m = x < 0 ? 0u - (unsigned)x : (unsigned)x;
+  int q = (int)niti_round_mag<unsigned>(m, bp, qmax, round_mode);
+  return x < 0 ? -q : q;
+}
+
+__device__ __forceinline__ int niti_bitlen32(unsigned v) { return 32 - __clz(v); }
+
+// ---- internal launchers (defined across the .cu files) ----------------------------------------
+// Shape of one matrix multiply D[m][n] = sum_k A(m,k) * B(n,k) with implicit operand addressing.
+enum NitiGemmKind {
+  GK_FC_FWD = 0,   // A = a[M][K],        B = w[N][K]
+  GK_FC_DGRAD,     // A = e[M][N],        B(k', n) = w[n][k']
+  GK_FC_WGRAD,     // A(n, m) = e[m][n],  B(k', m) = a[m][k']
+  GK_CONV_FWD,     // A(pix, (r,s,ci)) = x shifted, B = w[co][(r,s,ci)]
+  GK_CONV_DGRAD,   // A(pix, (r,s,co)) = e shifted, B(ci, (r,s,co)) = w[co][r][s][ci]
+  GK_CONV_WGRAD    // A(co, pix) = e[pix][co],      B((r,s,ci), pix) = x shifted
+};
+
+struct GemmProblem {
+  int kind;
+  const int8_t *p0;  // first operand  (a / e / x)
+  const int8_t *p1;  // second operand (w / a / e)
+  // fully connected: M, N, K of the layer.  convolution: B,H,W (input), Ho,Wo (output), Ci, Co, R, S, pad
+  int M, N, K;
+  int B, H, W, Ho, Wo, Ci, Co, R, S, pad;
+  // the matrix multiply actually run
+  long long gm, gn, gk;
+};
+
+// Plain CUDA-core engine: writes int32 accumulators to acc[gm][gn] and max|acc| to hdr->maxabs32.
+int niti_simt_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t *acc, WsHeader *hdr);
+// Tensor-core engine (tcgen05); returns NITI_ERR_SHAPE if the shape is not eligible.
+int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t *acc, WsHeader *hdr,
+                 void *scratch, size_t scratch_bytes);
+size_t niti_tc_scratch_bytes(const GemmProblem &p);
+
+// Epilogue pass: b from hdr->maxabs32, bp = max(0, b - mbits), out = Round(acc) with optional ReLU
+// and optional mask; s_out = s_a + s_w + bp if s_out != NULL; b_out = b if != NULL.
+int niti_launch_round(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, const WsHeader *hdr,
+                      int8_t *out, long long n, int mbits, int round_mode, int relu,
+                      const int8_t *mask, const int32_t *s_a, const int32_t *s_w, int32_t *s_out,
+                      int32_t *b_out);

@@ -1,0 +1,447 @@
+// HBM-bound kernels of the NITI library: the shift-and-round pass (Algorithm 2/3), the integer
+// cross-entropy gradient (Section 3.5), the weight update (Algorithm 1) and the int8 support ops.
+#include "niti_common.cuh"
+
+// ---------------------------------------------------------------------------------------------
+// Shift-and-round pass over an int32 accumulator tensor (Algorithm 2, with Algorithm 3 rounding).
+// Every thread handles 16 consecutive elements: four 16-byte loads, one 16-byte store.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+round_i32_kernel(const int32_t *__restrict__ acc, const WsHeader *__restrict__ hdr,
+                 int8_t *__restrict__ out, long long n, int mbits, int round_mode, int relu,
+                 const int8_t *__restrict__ mask, const int32_t *__restrict__ s_a,
+                 const int32_t *__restrict__ s_w, int32_t *__restrict__ s_out,
+                 int32_t *__restrict__ b_out, uint32_t *__restrict__ status) {
+  const int b = niti_bitlen32(hdr->maxabs32);
+  const int bp = b > mbits ? b - mbits : 0;
+  const unsigned qmax = (1u << mbits) - 1u;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (b_out) *b_out = b;
+    if (s_out) {
+      int s = bp + (s_a ? *s_a : 0) + (s_w ? *s_w : 0);
+      *s_out = s;
+      if (s < -128 || s > 127) atomicOr(status, NITI_DEV_EXP_RANGE);
+    }
+  }
+  const long long nvec = n >> 4;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += stride) {
+    const int4 *src = reinterpret_cast<const int4 *>(acc) + v * 4;
+    int4 x0 = __ldcs(src), x1 = __ldcs(src + 1), x2 = __ldcs(src + 2), x3 = __ldcs(src + 3);
+    int xs[16] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w,
+                  x2.x, x2.y, x2.z, x2.w, x3.x, x3.y, x3.z, x3.w};
+    int4 mk = make_int4(-1, -1, -1, -1);
+    if (mask) {
+      int4 mv = *(reinterpret_cast<const int4 *>(mask) + v);
+      mk.x = __vcmpgts4(mv.x, 0); mk.y = __vcmpgts4(mv.y, 0);
+      mk.z = __vcmpgts4(mv.z, 0); mk.w = __vcmpgts4(mv.w, 0);
+    }
+    unsigned o[4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      unsigned word = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int q = niti_round_i32(xs[w * 4 + j], bp, qmax, round_mode);
+        if (relu && q < 0) q = 0;
+        word |= (unsigned)(q & 0xff) << (8 * j);
+      }
+      o[w] = word;
+    }
+    int4 ov = make_int4(o[0] & mk.x, o[1] & mk.y, o[2] & mk.z, o[3] & mk.w);
+    *(reinterpret_cast<int4 *>(out) + v) = ov;
+  }
+  // ragged tail (fewer than 16 elements)
+  long long t = (nvec << 4) + (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n) {
+    int q = niti_round_i32(acc[t], bp, qmax, round_mode);
+    if (relu && q < 0) q = 0;
+    if (mask && mask[t] <= 0) q = 0;
+    out[t] = (int8_t)q;
+  }
+}
+
+int niti_launch_round(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, const WsHeader *hdr,
+                      int8_t *out, long long n, int mbits, int round_mode, int relu,
+                      const int8_t *mask, const int32_t *s_a, const int32_t *s_w, int32_t *s_out,
+                      int32_t *b_out) {
+  long long nvec = n >> 4;
+  long long blocks = (nvec + 255) / 256;
+  long long cap = (long long)ctx->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  round_i32_kernel<<<(unsigned)blocks, 256, 0, st>>>(acc, hdr, out, n, mbits, round_mode, relu, mask,
+                                                     s_a, s_w, s_out, b_out, ctx->d_status);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Integer cross-entropy gradient, Section 3.5.  Pass 1: one block per sample computes the integer
+// T_i (Eq. 2 or Eq. 3-4), their sum, e32 = T_i - [i == label] * sum (64-bit), the tensor-wide
+// max magnitude, and the arg-max hit count.  Pass 2: shared binary point, rounding to int8.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ long long block_reduce_ll(long long v, int op /*0 sum,1 max,2 min*/,
+                                                     long long *sh) {
+  for (int o = 16; o > 0; o >>= 1) {
+    long long u = __shfl_xor_sync(0xffffffffu, v, o);
+    v = op == 0 ? v + u : (op == 1 ? (u > v ? u : v) : (u < v ? u : v));
+  }
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
+  __syncthreads();
+  if (lane == 0) sh[warp] = v;
+  __syncthreads();
+  long long r = sh[0];
+  for (int i = 1; i < nw; ++i) {
+    long long u = sh[i];
+    r = op == 0 ? r + u : (op == 1 ? (u > r ? u : r) : (u < r ? u : r));
+  }
+  return r;
+}
+
+__global__ void __launch_bounds__(256)
+xent_acc_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
+                const int32_t *__restrict__ labels, long long *__restrict__ e64, WsHeader *hdr,
+                int32_t *__restrict__ n_correct, int N, uint32_t *__restrict__ status) {
+  __shared__ long long sh[8];
+  const int r = blockIdx.x;
+  const int s = *s_a_ptr;
+  const int label = labels[r];
+  const int8_t *row = a + (long long)r * N;
+  long long *erow = e64 + (long long)r * N;
+  if (s < -22 || s > 24 || label < 0 || label >= N) {
+    if (threadIdx.x == 0) atomicOr(status, (s < -22 || s > 24) ? NITI_DEV_XENT_RANGE : NITI_DEV_BAD_LABEL);
+    for (int i = threadIdx.x; i < N; i += blockDim.x) erow[i] = 0;
+    return;
+  }
+  const long long LLMIN = -0x7fffffffffffffffLL - 1, LLMAX = 0x7fffffffffffffffLL;
+  long long mx = LLMIN;
+  long long sh_amt = 15 - (long long)s;
+  if (s > -7) {
+    for (int i = threadIdx.x; i < N; i += blockDim.x) {
+      long long P = 47274LL * (long long)row[i];
+      long long xh = sh_amt >= 0 ? (P >> sh_amt) : P * (1LL << (-sh_amt));
+      mx = xh > mx ? xh : mx;
+    }
+    mx = block_reduce_ll(mx, 1, sh);
+  }
+  long long p = LLMAX;
+  if (s > -7) {
+    for (int i = threadIdx.x; i < N; i += blockDim.x) {
+      long long P = 47274LL * (long long)row[i];
+      long long xh = sh_amt >= 0 ? (P >> sh_amt) : P * (1LL << (-sh_amt));
+      if (xh > mx - 10 && xh < p) p = xh;
+    }
+    p = block_reduce_ll(p, 2, sh);
+  }
+  // T_i and their sum; also the first arg-max of the row for the hit count
+  long long csum = 0;
+  int best_v = -1000, best_i = 0x7fffffff;
+  for (int i = threadIdx.x; i < N; i += blockDim.x) {
+    long long ai = row[i];
+    long long T;
+    if (s <= -7) {
+      T = (1LL << (1 - 2 * s)) + ai * (1LL << (1 - s)) + ai * ai;
+    } else {
+      long long P = 47274LL * ai;
+      long long xh = sh_amt >= 0 ? (P >> sh_amt) : P * (1LL << (-sh_amt));
+      long long xt = xh - p;
+      T = 1LL << (xt > 0 ? xt : 0);
+    }
+    erow[i] = T;
+    csum += T;
+    if ((int)ai > best_v) { best_v = (int)ai; best_i = i; }
+  }
+  csum = block_reduce_ll(csum, 0, sh);
+  // first arg-max: maximise (value, -index)
+  long long key = ((long long)(best_v + 1000) << 32) | (unsigned)(0x7fffffff - best_i);
+  key = block_reduce_ll(key, 1, sh);
+  __syncthreads();
+  unsigned long long lmax = 0;
+  for (int i = threadIdx.x; i < N; i += blockDim.x) {
+    long long v = erow[i] - (i == label ? csum : 0);
+    erow[i] = v;
+    unsigned long long m = v < 0 ? 0ull - (unsigned long long)v : (unsigned long long)v;
+    lmax = m > lmax ? m : lmax;
+  }
+  long long bm = block_reduce_ll((long long)lmax, 1, sh);
+  if (threadIdx.x == 0) {
+    atomicMax(&hdr->maxabs64, (unsigned long long)bm);
+    if (n_correct) {
+      int arg = 0x7fffffff - (int)(key & 0xffffffffLL);
+      if (arg == label) atomicAdd(n_correct, 1);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256)
+round_i64_kernel(const long long *__restrict__ e64, const WsHeader *__restrict__ hdr,
+                 int8_t *__restrict__ out, long long n, int round_mode, int32_t *__restrict__ b_out) {
+  unsigned long long mxv = hdr->maxabs64;
+  const int b = 64 - __clzll((long long)mxv);
+  const int bp = b > 7 ? b - 7 : 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0 && b_out) *b_out = b;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x) {
+    long long v = e64[i];
+    unsigned long long m = v < 0 ? 0ull - (unsigned long long)v : (unsigned long long)v;
+    long long q = (long long)niti_round_mag<unsigned long long>(m, bp, 127ull, round_mode);
+    out[i] = (int8_t)(v < 0 ? -q : q);
+  }
+}
+
+extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const int32_t *s_a,
+                             const int32_t *labels, int8_t *e, int32_t *b_e, int32_t *n_correct,
+                             int B, int N, int round_mode, void *ws, size_t ws_bytes) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!a || !s_a || !labels || !e || B <= 0 || N <= 0 || N > 65536 || (round_mode != 0 && round_mode != 1))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_int_xent: bad argument");
+  int64_t dims[2] = {B, N};
+  if (!ws || ((uintptr_t)ws & 255) || ws_bytes < niti_workspace_bytes(NITI_OP_INT_XENT, dims, 2))
+    return niti_fail(ctx, NITI_ERR_WORKSPACE, "niti_int_xent: workspace missing, misaligned or too small");
+  cudaStream_t st = (cudaStream_t)stream;
+  WsHeader *hdr = (WsHeader *)ws;
+  long long *e64 = (long long *)((char *)ws + NITI_WS_HEADER);
+  NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, sizeof(WsHeader), st));
+  ctx->launches++;
+  if (n_correct) {
+    NITI_CUDA_TRY(ctx, cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st));
+    ctx->launches++;
+  }
+  xent_acc_kernel<<<B, 256, 0, st>>>(a, s_a, labels, e64, hdr, n_correct, N, ctx->d_status);
+  ctx->launches++;
+  long long n = (long long)B * N;
+  long long blocks = (n + 255) / 256;
+  if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+  round_i64_kernel<<<(unsigned)blocks, 256, 0, st>>>(e64, hdr, e, n, round_mode, b_e);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Byte-wise SIMD elementwise ops: 16 int8 per thread per iteration (one 16-byte load per operand).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned sat_sub_clamp127(unsigned w, unsigned g) {
+  // per byte: clamp(w - g, -127, 127): saturating subtract gives [-128, 127]; lift -128 to -127
+  return __vmaxs4(__vsubss4(w, g), 0x81818181u);
+}
+
+__global__ void __launch_bounds__(256)
+sgd_update_kernel(int8_t *__restrict__ w, const int8_t *__restrict__ g, long long n) {
+  const long long nvec = n >> 4;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  for (long long v = tid; v < nvec; v += stride) {
+    int4 wv = *(reinterpret_cast<int4 *>(w) + v);
+    int4 gv = __ldcs(reinterpret_cast<const int4 *>(g) + v);
+    wv.x = sat_sub_clamp127(wv.x, gv.x); wv.y = sat_sub_clamp127(wv.y, gv.y);
+    wv.z = sat_sub_clamp127(wv.z, gv.z); wv.w = sat_sub_clamp127(wv.w, gv.w);
+    *(reinterpret_cast<int4 *>(w) + v) = wv;
+  }
+  long long t = (nvec << 4) + tid;
+  if (t < n) {
+    int d = (int)w[t] - (int)g[t];
+    d = d > 127 ? 127 : (d < -127 ? -127 : d);
+    w[t] = (int8_t)d;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+relu_fwd_kernel(const int8_t *__restrict__ x, int8_t *__restrict__ y, long long n) {
+  const long long nvec = n >> 4;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  for (long long v = tid; v < nvec; v += stride) {
+    int4 xv = *(reinterpret_cast<const int4 *>(x) + v);
+    xv.x = __vmaxs4(xv.x, 0); xv.y = __vmaxs4(xv.y, 0); xv.z = __vmaxs4(xv.z, 0); xv.w = __vmaxs4(xv.w, 0);
+    *(reinterpret_cast<int4 *>(y) + v) = xv;
+  }
+  long long t = (nvec << 4) + tid;
+  if (t < n) y[t] = x[t] > 0 ? x[t] : 0;
+}
+
+__global__ void __launch_bounds__(256)
+relu_bwd_kernel(const int8_t *__restrict__ y, const int8_t *__restrict__ eo, int8_t *__restrict__ ei,
+                long long n) {
+  const long long nvec = n >> 4;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  for (long long v = tid; v < nvec; v += stride) {
+    int4 yv = *(reinterpret_cast<const int4 *>(y) + v);
+    int4 ev = *(reinterpret_cast<const int4 *>(eo) + v);
+    ev.x &= __vcmpgts4(yv.x, 0); ev.y &= __vcmpgts4(yv.y, 0);
+    ev.z &= __vcmpgts4(yv.z, 0); ev.w &= __vcmpgts4(yv.w, 0);
+    *(reinterpret_cast<int4 *>(ei) + v) = ev;
+  }
+  long long t = (nvec << 4) + tid;
+  if (t < n) ei[t] = y[t] > 0 ? eo[t] : 0;
+}
+
+// 2x2 max-pool, NHWC.  VEC = 16: one thread per 16 channels of one output pixel; VEC = 1: scalar.
+template <int VEC>
+__global__ void __launch_bounds__(256)
+maxpool2_fwd_kernel(const int8_t *__restrict__ x, int8_t *__restrict__ y, int B, int H, int W, int C) {
+  const int Ho = H >> 1, Wo = W >> 1, Cv = C / VEC;
+  const long long total = (long long)B * Ho * Wo * Cv;
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (long long)gridDim.x * blockDim.x) {
+    int cv = (int)(t % Cv);
+    long long pix = t / Cv;
+    int j = (int)(pix % Wo);
+    long long bi = pix / Wo;
+    int i = (int)(bi % Ho);
+    long long b = bi / Ho;
+    long long base = (((b * H + 2 * i) * W + 2 * j) * (long long)C) + (long long)cv * VEC;
+    long long rs = (long long)W * C;
+    if (VEC == 16) {
+      int4 v0 = *reinterpret_cast<const int4 *>(x + base);
+      int4 v1 = *reinterpret_cast<const int4 *>(x + base + C);
+      int4 v2 = *reinterpret_cast<const int4 *>(x + base + rs);
+      int4 v3 = *reinterpret_cast<const int4 *>(x + base + rs + C);
+      int4 m;
+      m.x = __vmaxs4(__vmaxs4(v0.x, v1.x), __vmaxs4(v2.x, v3.x));
+      m.y = __vmaxs4(__vmaxs4(v0.y, v1.y), __vmaxs4(v2.y, v3.y));
+      m.z = __vmaxs4(__vmaxs4(v0.z, v1.z), __vmaxs4(v2.z, v3.z));
+      m.w = __vmaxs4(__vmaxs4(v0.w, v1.w), __vmaxs4(v2.w, v3.w));
+      *reinterpret_cast<int4 *>(y + pix * C + (long long)cv * VEC) = m;
+    } else {
+      int8_t m = x[base];
+      int8_t v = x[base + C]; m = v > m ? v : m;
+      v = x[base + rs]; m = v > m ? v : m;
+      v = x[base + rs + C]; m = v > m ? v : m;
+      y[pix * C + cv] = m;
+    }
+  }
+}
+
+__device__ __forceinline__ void pool_bwd_word(unsigned x0, unsigned x1, unsigned x2, unsigned x3,
+                                              unsigned e, int relu, unsigned &o0, unsigned &o1,
+                                              unsigned &o2, unsigned &o3) {
+  unsigned m = __vmaxs4(__vmaxs4(x0, x1), __vmaxs4(x2, x3));
+  unsigned s0 = __vcmpeq4(x0, m);
+  unsigned s1 = __vcmpeq4(x1, m) & ~s0;
+  unsigned s2 = __vcmpeq4(x2, m) & ~(s0 | s1);
+  unsigned s3 = ~(s0 | s1 | s2);
+  if (relu) {
+    unsigned pos = __vcmpgts4(m, 0);   // the routed position holds the maximum
+    e &= pos;
+  }
+  o0 = e & s0; o1 = e & s1; o2 = e & s2; o3 = e & s3;
+}
+
+template <int VEC>
+__global__ void __launch_bounds__(256)
+maxpool2_bwd_kernel(const int8_t *__restrict__ x, const int8_t *__restrict__ eo,
+                    int8_t *__restrict__ ei, int B, int H, int W, int C, int relu) {
+  const int Ho = H >> 1, Wo = W >> 1, Cv = C / VEC;
+  const long long total = (long long)B * Ho * Wo * Cv;
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (long long)gridDim.x * blockDim.x) {
+    int cv = (int)(t % Cv);
+    long long pix = t / Cv;
+    int j = (int)(pix % Wo);
+    long long bi = pix / Wo;
+    int i = (int)(bi % Ho);
+    long long b = bi / Ho;
+    long long base = (((b * H + 2 * i) * W + 2 * j) * (long long)C) + (long long)cv * VEC;
+    long long rs = (long long)W * C;
+    if (VEC == 16) {
+      int4 v0 = *reinterpret_cast<const int4 *>(x + base);
+      int4 v1 = *reinterpret_cast<const int4 *>(x + base + C);
+      int4 v2 = *reinterpret_cast<const int4 *>(x + base + rs);
+      int4 v3 = *reinterpret_cast<const int4 *>(x + base + rs + C);
+      int4 e = *reinterpret_cast<const int4 *>(eo + pix * C + (long long)cv * VEC);
+      int4 o0, o1, o2, o3;
+      pool_bwd_word(v0.x, v1.x, v2.x, v3.x, e.x, relu, (unsigned &)o0.x, (unsigned &)o1.x, (unsigned &)o2.x, (unsigned &)o3.x);
+      pool_bwd_word(v0.y, v1.y, v2.y, v3.y, e.y, relu, (unsigned &)o0.y, (unsigned &)o1.y, (unsigned &)o2.y, (unsigned &)o3.y);
+      pool_bwd_word(v0.z, v1.z, v2.z, v3.z, e.z, relu, (unsigned &)o0.z, (unsigned &)o1.z, (unsigned &)o2.z, (unsigned &)o3.z);
+      pool_bwd_word(v0.w, v1.w, v2.w, v3.w, e.w, relu, (unsigned &)o0.w, (unsigned &)o1.w, (unsigned &)o2.w, (unsigned &)o3.w);
+      *reinterpret_cast<int4 *>(ei + base) = o0;
+      *reinterpret_cast<int4 *>(ei + base + C) = o1;
+      *reinterpret_cast<int4 *>(ei + base + rs) = o2;
+      *reinterpret_cast<int4 *>(ei + base + rs + C) = o3;
+    } else {
+      long long idx[4] = {base, base + C, base + rs, base + rs + C};
+      int best = 0;
+      for (int k = 1; k < 4; ++k)
+        if (x[idx[k]] > x[idx[best]]) best = k;
+      int8_t e = eo[pix * C + cv];
+      if (relu && x[idx[best]] <= 0) e = 0;
+      for (int k = 0; k < 4; ++k) ei[idx[k]] = k == best ? e : (int8_t)0;
+    }
+  }
+}
+
+static inline unsigned ew_blocks(niti_ctx *ctx, long long work_items) {
+  long long blocks = (work_items + 255) / 256;
+  long long cap = (long long)ctx->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return (unsigned)blocks;
+}
+
+extern "C" int niti_int_sgd_update(niti_ctx *ctx, void *stream, int8_t *w, const int8_t *g, int64_t n) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!w || !g || n <= 0) return niti_fail(ctx, NITI_ERR_ARG, "niti_int_sgd_update: bad argument");
+  if (((uintptr_t)w | (uintptr_t)g) & 15)
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_int_sgd_update: pointers must be 16-byte aligned");
+  sgd_update_kernel<<<ew_blocks(ctx, (n >> 4) + 16), 256, 0, (cudaStream_t)stream>>>(w, g, n);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+extern "C" int niti_relu_fwd(niti_ctx *ctx, void *stream, const int8_t *x, int8_t *y, int64_t n) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!x || !y || n <= 0 || (((uintptr_t)x | (uintptr_t)y) & 15))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_relu_fwd: bad argument");
+  relu_fwd_kernel<<<ew_blocks(ctx, (n >> 4) + 16), 256, 0, (cudaStream_t)stream>>>(x, y, n);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+extern "C" int niti_relu_bwd(niti_ctx *ctx, void *stream, const int8_t *y, const int8_t *e_out,
+                             int8_t *e_in, int64_t n) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!y || !e_out || !e_in || n <= 0 || (((uintptr_t)y | (uintptr_t)e_out | (uintptr_t)e_in) & 15))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_relu_bwd: bad argument");
+  relu_bwd_kernel<<<ew_blocks(ctx, (n >> 4) + 16), 256, 0, (cudaStream_t)stream>>>(y, e_out, e_in, n);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+extern "C" int niti_maxpool2_fwd(niti_ctx *ctx, void *stream, const int8_t *x, int8_t *y, int B, int H,
+                                 int W, int C) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!x || !y || B <= 0 || H <= 0 || W <= 0 || C <= 0 || (H & 1) || (W & 1))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_maxpool2_fwd: bad argument (H and W must be even)");
+  bool vec = (C % 16 == 0) && !(((uintptr_t)x | (uintptr_t)y) & 15);
+  long long items = (long long)B * (H / 2) * (W / 2) * (vec ? C / 16 : C);
+  if (vec)
+    maxpool2_fwd_kernel<16><<<ew_blocks(ctx, items), 256, 0, (cudaStream_t)stream>>>(x, y, B, H, W, C);
+  else
+    maxpool2_fwd_kernel<1><<<ew_blocks(ctx, items), 256, 0, (cudaStream_t)stream>>>(x, y, B, H, W, C);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+extern "C" int niti_maxpool2_bwd(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e_out,
+                                 int8_t *e_in, int B, int H, int W, int C, int relu) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!x || !e_out || !e_in || B <= 0 || H <= 0 || W <= 0 || C <= 0 || (H & 1) || (W & 1))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_maxpool2_bwd: bad argument (H and W must be even)");
+  bool vec = (C % 16 == 0) && !(((uintptr_t)x | (uintptr_t)e_out | (uintptr_t)e_in) & 15);
+  long long items = (long long)B * (H / 2) * (W / 2) * (vec ? C / 16 : C);
+  if (vec)
+    maxpool2_bwd_kernel<16><<<ew_blocks(ctx, items), 256, 0, (cudaStream_t)stream>>>(x, e_out, e_in, B, H, W, C, relu);
+  else
+    maxpool2_bwd_kernel<1><<<ew_blocks(ctx, items), 256, 0, (cudaStream_t)stream>>>(x, e_out, e_in, B, H, W, C, relu);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}

@@ -1,0 +1,691 @@
+// Tensor-core engine: int8 x int8 -> int32 matrix multiply on the 5th-generation tensor cores
+// (tcgen05.mma kind::i8, accumulators in tensor memory, operands staged by TMA), sm_100a only.
+//
+// One persistent CTA per SM; warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner),
+// warps 2..5 = epilogue (each reads its 32-lane quarter of TMEM with tcgen05.ld).  The accumulator
+// is double-buffered in TMEM so the epilogue of one tile overlaps the main loop of the next.
+//
+// The six operand mappings of the layer ops (Int8MatrixMultiply of Algorithm 1; implicit GEMM for
+// convolutions, Section 3.2) differ only in the TMA tensor maps, the per-k-block coordinates the
+// producer issues, and the shared-memory matrix descriptors (K-major or MN-major operands).
+//
+// Every wait in the kernel is bounded: after ~1 s without progress a thread raises
+// NITI_DEV_TIMEOUT in the status word, and all roles drain and leave through the common exit
+// that frees the tensor memory.
+#include "niti_common.cuh"
+
+namespace {
+
+constexpr int BM = 128;               // rows of an output tile = TMEM lanes
+constexpr int NUM_THREADS = 192;
+constexpr int MAX_STAGES = 8;
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;
+
+struct TcParams {
+  int kind;
+  int n_tiles_n;                // tiles along the output columns
+  int kb_total;                 // k-blocks of the whole contraction
+  int kb_per_split;
+  int splits;
+  long long items;              // tiles * splits
+  long long gm, gn;             // output extent (rows, columns); row pitch of acc is gn
+  int bn;                       // tile width (multiple of 32, <= 256)
+  int kdepth;                   // contraction elements per k-block (32, 64 or 128)
+  int ksteps;                   // kdepth / 32 MMAs per k-block
+  int stages;
+  int atomic_out;               // 1: add into acc (split contraction), 0: store + max
+  // shared-memory layout of one stage
+  int a_bytes, b_bytes;         // bytes of the A and B parts of a stage
+  int a_boxes, b_boxes;         // TMA copies per operand per stage
+  int a_box_bytes, b_box_bytes;
+  int a_box_step, b_box_step;   // coordinate step between consecutive boxes (MN-major operands)
+  // MMA descriptors
+  unsigned idesc;
+  unsigned long long a_desc, b_desc;   // descriptor without the start address
+  unsigned a_kstep16, b_kstep16;       // start-address advance per MMA, in 16-byte units
+  // convolution geometry (pixels of the tensor that the 4-D map covers)
+  int Wt, Ht, Bt;               // pixel box of a tile / k-block: Wt * Ht * Bt == 128
+  int w_tiles, h_tiles, b_tiles;
+  int PW, PH, PB;               // extent of the pixel grid the output rows (or k-blocks) run over
+  int R, S, pad;
+  int c_chunks;                 // channel chunks per tap along the contraction (fwd / dgrad)
+  int Cn;                       // wgrad: input channels Ci (columns per tap)
+  int n_chunks;                 // wgrad: column chunks per tap
+};
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void *p) {
+  return (unsigned)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(unsigned bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the abort flag) if the barrier did not flip in time or
+// another thread already gave up.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int *abort_flag,
+                                          uint32_t *status) {
+  if (mbar_try(bar, parity)) return true;
+  long long t0 = clock64();
+  while (true) {
+    if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      *abort_flag = 1;
+      atomicOr(status, NITI_DEV_TIMEOUT);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1,
+                                            int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(unsigned bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_i8(unsigned tmem_d, unsigned long long da, unsigned long long db,
+                                          unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(unsigned taddr, int (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Coordinates of an output tile / k-block in the pixel grid of a convolution.
+__device__ __forceinline__ void pixel_box(const TcParams &p, int idx, int &w0, int &h0, int &b0) {
+  int wt = idx % p.w_tiles;
+  int t = idx / p.w_tiles;
+  int ht = t % p.h_tiles;
+  int bt = t / p.h_tiles;
+  w0 = wt * p.Wt; h0 = ht * p.Ht; b0 = bt * p.Bt;
+}
+
+// ------------------------------------------------------------------------------------------
+// The kernel
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const TcParams p, int32_t *__restrict__ acc, WsHeader *hdr, uint32_t *status) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 4];
+  __shared__ unsigned tmem_base_slot;
+  __shared__ volatile int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int stage_bytes = p.a_bytes + p.b_bytes;
+  const unsigned full0 = smem_u32(&bars[0]);
+  const unsigned empty0 = smem_u32(&bars[MAX_STAGES]);
+  const unsigned tfull0 = smem_u32(&bars[2 * MAX_STAGES]);
+  const unsigned tempty0 = smem_u32(&bars[2 * MAX_STAGES + 2]);
+
+  // TMEM columns: two accumulator buffers of bn columns, rounded up to a power of two >= 32
+  unsigned tmem_cols = 32;
+  while (tmem_cols < 2u * (unsigned)p.bn) tmem_cols <<= 1;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull0 + 8 * b, 1);
+      mbar_init(tempty0 + 8 * b, 4);     // one arrival per epilogue warp
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    // ================= TMA producer =================
+    if (lane == 0) {
+      int stage = 0;
+      unsigned phase = 0;
+      bool ok = true;
+      for (long long item = blockIdx.x; ok && item < p.items; item += gridDim.x) {
+        const long long tile = item / p.splits;
+        const int split = (int)(item % p.splits);
+        const int mt = (int)(tile / p.n_tiles_n), nt = (int)(tile % p.n_tiles_n);
+        const int kb0 = split * p.kb_per_split;
+        int kb1 = kb0 + p.kb_per_split;
+        if (kb1 > p.kb_total) kb1 = p.kb_total;
+        int w0 = 0, h0 = 0, b0 = 0, tap_n = 0, ci0 = 0;
+        if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) pixel_box(p, mt, w0, h0, b0);
+        if (p.kind == GK_CONV_WGRAD) { tap_n = nt / p.n_chunks; ci0 = (nt % p.n_chunks) * p.bn; }
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
+          const unsigned full = full0 + 8 * stage;
+          const unsigned sa = smem_base + stage * stage_bytes;
+          const unsigned sb = sa + p.a_bytes;
+          mbar_expect_tx(full, (unsigned)(p.a_boxes * p.a_box_bytes + p.b_boxes * p.b_box_bytes));
+          switch (p.kind) {
+            case GK_FC_FWD:       // A [M][K] K-major, B [N][K] K-major
+              tma_load_2d(sa, &map_a, full, kb * p.kdepth, mt * BM);
+              tma_load_2d(sb, &map_b, full, kb * p.kdepth, nt * p.bn);
+              break;
+            case GK_FC_DGRAD:     // A = e [M][N] K-major; B(k', n) = w[n][k'] MN-major
+              tma_load_2d(sa, &map_a, full, kb * p.kdepth, mt * BM);
+              for (int j = 0; j < p.b_boxes; ++j)
+                tma_load_2d(sb + j * p.b_box_bytes, &map_b, full, nt * p.bn + j * p.b_box_step, kb * p.kdepth);
+              break;
+            case GK_FC_WGRAD:     // A(n, m) = e[m][n] MN-major; B(k', m) = a[m][k'] MN-major
+              for (int j = 0; j < p.a_boxes; ++j)
+                tma_load_2d(sa + j * p.a_box_bytes, &map_a, full, mt * BM + j * p.a_box_step, kb * p.kdepth);
+              for (int j = 0; j < p.b_boxes; ++j)
+                tma_load_2d(sb + j * p.b_box_bytes, &map_b, full, nt * p.bn + j * p.b_box_step, kb * p.kdepth);
+              break;
+            case GK_CONV_FWD: {   // k-block = (tap, channel chunk)
+              int tap = kb / p.c_chunks, cc = kb % p.c_chunks;
+              int r = tap / p.S, s = tap % p.S;
+              tma_load_4d(sa, &map_a, full, cc * p.kdepth, w0 + s - p.pad, h0 + r - p.pad, b0);
+              tma_load_2d(sb, &map_b, full, kb * p.kdepth, nt * p.bn);
+              break;
+            }
+            case GK_CONV_DGRAD: { // A = e shifted the other way; B(ci, (tap, co)) = w[co][tap][ci]
+              int tap = kb / p.c_chunks, cc = kb % p.c_chunks;
+              int r = tap / p.S, s = tap % p.S;
+              tma_load_4d(sa, &map_a, full, cc * p.kdepth, w0 - s + p.pad, h0 - r + p.pad, b0);
+              for (int j = 0; j < p.b_boxes; ++j)
+                tma_load_2d(sb + j * p.b_box_bytes, &map_b, full, tap * p.Cn + nt * p.bn + j * p.b_box_step,
+                            cc * p.kdepth);
+              break;
+            }
+            default: {            // GK_CONV_WGRAD: k-block = pixel box; A = e, B = x shifted by the tap
+              int kw0, kh0, kbb0;
+              pixel_box(p, kb, kw0, kh0, kbb0);
+              int r = tap_n / p.S, s = tap_n % p.S;
+              for (int j = 0; j < p.a_boxes; ++j)
+                tma_load_4d(sa + j * p.a_box_bytes, &map_a, full, mt * BM + j * p.a_box_step, kw0, kh0, kbb0);
+              for (int j = 0; j < p.b_boxes; ++j)
+                tma_load_4d(sb + j * p.b_box_bytes, &map_b, full, ci0 + j * p.b_box_step, kw0 + s - p.pad,
+                            kh0 + r - p.pad, kbb0);
+              break;
+            }
+          }
+          if (++stage == p.stages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ================= MMA issuer =================
+    if (lane == 0) {
+      int stage = 0;
+      unsigned phase = 0;
+      unsigned use = 0;                 // tiles processed by this CTA
+      bool ok = true;
+      for (long long item = blockIdx.x; ok && item < p.items; item += gridDim.x, ++use) {
+        const int split = (int)(item % p.splits);
+        const int kb0 = split * p.kb_per_split;
+        int kb1 = kb0 + p.kb_per_split;
+        if (kb1 > p.kb_total) kb1 = p.kb_total;
+        const unsigned buf = use & 1u;
+        // wait until the epilogue has drained this accumulator buffer (first two uses pass at once)
+        if (!mbar_wait(tempty0 + 8 * buf, ((use >> 1) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
+        tc_fence_after();
+        const unsigned tmem_d = tmem_base + buf * (unsigned)p.bn;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const unsigned sa = smem_base + stage * stage_bytes;
+          const unsigned sb = sa + p.a_bytes;
+          unsigned long long da = p.a_desc | (unsigned long long)((sa >> 4) & 0x3fff);
+          unsigned long long db = p.b_desc | (unsigned long long)((sb >> 4) & 0x3fff);
+          for (int k = 0; k < p.ksteps; ++k) {
+            tc_mma_i8(tmem_d, da, db, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+            da += p.a_kstep16;
+            db += p.b_kstep16;
+          }
+          tc_commit(empty0 + 8 * stage);        // frees the stage once these MMAs have read it
+          if (++stage == p.stages) { stage = 0; phase ^= 1; }
+        }
+        if (ok) tc_commit(tfull0 + 8 * buf);    // accumulator complete
+      }
+    }
+  } else {
+    // ================= epilogue: TMEM -> int32 accumulators + max magnitude =================
+    const int quarter = warp & 3;               // TMEM lanes [32 * quarter, +32)
+    const int row_in_tile = quarter * 32 + lane;
+    unsigned use = 0;
+    unsigned mx = 0;
+    bool ok = true;
+    for (long long item = blockIdx.x; ok && item < p.items; item += gridDim.x, ++use) {
+      const long long tile = item / p.splits;
+      const int mt = (int)(tile / p.n_tiles_n), nt = (int)(tile % p.n_tiles_n);
+      const unsigned buf = use & 1u;
+      // output row / column base of this thread
+      long long out_row;
+      bool row_ok;
+      long long col0;
+      int ncols_valid;
+      if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) {
+        int w0, h0, b0;
+        pixel_box(p, mt, w0, h0, b0);
+        int ww = row_in_tile % p.Wt, t = row_in_tile / p.Wt;
+        int hh = t % p.Ht, bb = t / p.Ht;
+        int w = w0 + ww, h = h0 + hh, b = b0 + bb;
+        row_ok = w < p.PW && h < p.PH && b < p.PB;
+        out_row = ((long long)b * p.PH + h) * p.PW + w;
+        col0 = (long long)nt * p.bn;
+        long long rem = p.gn - col0;
+        ncols_valid = rem < p.bn ? (int)rem : p.bn;
+      } else if (p.kind == GK_CONV_WGRAD) {
+        out_row = (long long)mt * BM + row_in_tile;
+        row_ok = out_row < p.gm;
+        int tap = nt / p.n_chunks, ci0 = (nt % p.n_chunks) * p.bn;
+        col0 = (long long)tap * p.Cn + ci0;
+        int rem = p.Cn - ci0;
+        ncols_valid = rem < p.bn ? rem : p.bn;
+      } else {
+        out_row = (long long)mt * BM + row_in_tile;
+        row_ok = out_row < p.gm;
+        col0 = (long long)nt * p.bn;
+        long long rem = p.gn - col0;
+        ncols_valid = rem < p.bn ? (int)rem : p.bn;
+      }
+      if (!mbar_wait(tfull0 + 8 * buf, (use >> 1) & 1u, &abort_flag, status)) { ok = false; break; }
+      tc_fence_after();
+      int32_t *dst = acc + out_row * p.gn + col0;
+      const bool vec_ok = ((p.gn & 3) == 0) && ((col0 & 3) == 0);
+      for (int c = 0; c < p.bn; c += 32) {
+        int v[32];
+        tc_ld32(tmem_base + ((unsigned)(quarter * 32) << 16) + buf * (unsigned)p.bn + (unsigned)c, v);
+        if (row_ok && c < ncols_valid) {
+          if (p.atomic_out) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c + j < ncols_valid && v[j] != 0) atomicAdd(dst + c + j, v[j]);
+          } else {
+            if (vec_ok && c + 32 <= ncols_valid) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                *reinterpret_cast<int4 *>(dst + c + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+              }
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                unsigned a = v[j] < 0 ? 0u - (unsigned)v[j] : (unsigned)v[j];
+                mx = a > mx ? a : mx;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (c + j < ncols_valid) {
+                  dst[c + j] = v[j];
+                  unsigned a = v[j] < 0 ? 0u - (unsigned)v[j] : (unsigned)v[j];
+                  mx = a > mx ? a : mx;
+                }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8 * buf);
+    }
+    if (!p.atomic_out) {
+      for (int o = 16; o > 0; o >>= 1) {
+        unsigned u = __shfl_xor_sync(0xffffffffu, mx, o);
+        mx = u > mx ? u : mx;
+      }
+      if (lane == 0 && mx) atomicMax(&hdr->maxabs32, mx);
+    }
+  }
+
+  // ================= common exit =================
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    // give copies and MMAs still in flight time to land before shared and tensor memory go away
+    long long t0 = clock64();
+    while (clock64() - t0 < 20000000LL) {
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side: tensor maps, descriptors, eligibility
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static CUtensorMapSwizzle swizzle_enum(int bytes) {
+  return bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+}
+static unsigned long long layout_bits(int swizzle_bytes) {
+  // matrix-descriptor layout type: 2 = 128-byte swizzle, 4 = 64-byte, 6 = 32-byte
+  unsigned long long t = swizzle_bytes == 128 ? 2 : (swizzle_bytes == 64 ? 4 : 6);
+  return t << 61;
+}
+// Descriptor (without start address) of a K-major operand whose rows are `sw` bytes wide.
+static unsigned long long desc_kmajor(int sw) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)1 << 16;                          // leading byte offset: unused, 1
+  d |= (unsigned long long)((8 * sw) >> 4) << 32;            // stride between 8-row groups
+  d |= (unsigned long long)1 << 46;                          // descriptor version
+  return d | layout_bits(sw);
+}
+// Descriptor of an MN-major operand stored as sub-tiles [kdepth rows][sw bytes].
+static unsigned long long desc_mnmajor(int sw, int kdepth) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((kdepth * sw) >> 4) << 16;       // next sw-wide chunk along M/N
+  d |= (unsigned long long)((8 * sw) >> 4) << 32;            // next group of 8 k-rows
+  d |= (unsigned long long)1 << 46;
+  return d | layout_bits(sw);
+}
+static int pick_swizzle(long long extent) { return extent >= 128 ? 128 : (extent >= 64 ? 64 : (extent >= 32 ? 32 : 0)); }
+
+struct MapSpec {
+  int nd;
+  cuuint64_t dims[4];
+  cuuint64_t strides[3];   // bytes, dims 1..3
+  cuuint32_t box[4];
+  int swizzle;
+  const void *base;
+};
+
+static bool encode(niti_ctx *ctx, CUtensorMap *m, const MapSpec &s) {
+  if (!ctx->encode_tiled) return false;
+  if (((uintptr_t)s.base & 15) != 0) return false;
+  for (int i = 0; i + 1 < s.nd; ++i)
+    if (s.strides[i] % 16 != 0) return false;
+  for (int i = 0; i < s.nd; ++i)
+    if (s.box[i] == 0 || s.box[i] > 256) return false;
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  CUresult r = ((EncodeTiledFn)ctx->encode_tiled)(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)s.nd,
+                                                  const_cast<void *>(s.base), s.dims, s.strides, s.box, es,
+                                                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_enum(s.swizzle),
+                                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// Pixel box with Wt * Ht * Bt == 128 (powers of two).
+static bool pick_pixel_box(int W, int H, int B, int &Wt, int &Ht, int &Bt) {
+  Wt = 1;
+  while (Wt < 128 && W % (Wt * 2) == 0) Wt *= 2;
+  Ht = 1;
+  while (Wt * Ht < 128 && H % (Ht * 2) == 0) Ht *= 2;
+  Bt = 128 / (Wt * Ht);
+  if (Bt > 256) return false;
+  return Wt <= W && Ht <= H && Bt <= B;
+}
+
+static int round_up32(long long n) { return (int)((n + 31) / 32 * 32); }
+
+// Builds params and maps; returns false if the shape is not eligible for this engine.
+static bool plan(niti_ctx *ctx, const GemmProblem &g, TcParams &p, CUtensorMap &ma, CUtensorMap &mb) {
+  memset(&p, 0, sizeof(p));
+  p.kind = g.kind;
+  p.gm = g.gm;
+  p.gn = g.gn;
+  p.splits = 1;
+  MapSpec sa, sb;
+  memset(&sa, 0, sizeof(sa));
+  memset(&sb, 0, sizeof(sb));
+  int a_mn = 0, b_mn = 0;        // 1 = MN-major operand
+  int a_sw = 0, b_sw = 0;
+  long long m_tiles = 0;
+  if (g.gm * g.gn >= (1LL << 31)) return false;
+  switch (g.kind) {
+    case GK_FC_FWD: {
+      p.kdepth = pick_swizzle(g.gk);
+      if (!p.kdepth) return false;
+      p.bn = g.gn >= 256 ? 256 : round_up32(g.gn);
+      a_sw = b_sw = p.kdepth;
+      sa = {2, {(cuuint64_t)g.gk, (cuuint64_t)g.gm}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, BM}, a_sw, g.p0};
+      sb = {2, {(cuuint64_t)g.gk, (cuuint64_t)g.gn}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, (cuuint32_t)p.bn}, b_sw, g.p1};
+      p.kb_total = (int)((g.gk + p.kdepth - 1) / p.kdepth);
+      m_tiles = (g.gm + BM - 1) / BM;
+      p.n_tiles_n = (int)((g.gn + p.bn - 1) / p.bn);
+      break;
+    }
+    case GK_FC_DGRAD: {   // out [M][K'], contraction over N
+      p.kdepth = pick_swizzle(g.gk);
+      if (!p.kdepth) return false;
+      b_mn = 1;
+      b_sw = pick_swizzle(g.gn);
+      if (!b_sw) return false;
+      p.bn = g.gn >= 256 ? 256 : (int)((g.gn + b_sw - 1) / b_sw * b_sw);
+      if (p.bn % 32) return false;
+      a_sw = p.kdepth;
+      sa = {2, {(cuuint64_t)g.gk, (cuuint64_t)g.gm}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, BM}, a_sw, g.p0};
+      sb = {2, {(cuuint64_t)g.gn, (cuuint64_t)g.gk}, {(cuuint64_t)g.gn}, {(cuuint32_t)b_sw, (cuuint32_t)p.kdepth}, b_sw, g.p1};
+      p.kb_total = (int)((g.gk + p.kdepth - 1) / p.kdepth);
+      m_tiles = (g.gm + BM - 1) / BM;
+      p.n_tiles_n = (int)((g.gn + p.bn - 1) / p.bn);
+      break;
+    }
+    case GK_FC_WGRAD: {   // out [N][K'], contraction over M (rows of both operands)
+      a_mn = b_mn = 1;
+      a_sw = pick_swizzle(g.gm);
+      b_sw = pick_swizzle(g.gn);
+      if (!a_sw || !b_sw || g.gk < 32) return false;
+      p.kdepth = g.gk >= 128 ? 128 : (g.gk >= 64 ? 64 : 32);
+      p.bn = g.gn >= 256 ? 256 : (int)((g.gn + b_sw - 1) / b_sw * b_sw);
+      if (p.bn % 32) return false;
+      sa = {2, {(cuuint64_t)g.gm, (cuuint64_t)g.gk}, {(cuuint64_t)g.gm}, {(cuuint32_t)a_sw, (cuuint32_t)p.kdepth}, a_sw, g.p0};
+      sb = {2, {(cuuint64_t)g.gn, (cuuint64_t)g.gk}, {(cuuint64_t)g.gn}, {(cuuint32_t)b_sw, (cuuint32_t)p.kdepth}, b_sw, g.p1};
+      p.kb_total = (int)((g.gk + p.kdepth - 1) / p.kdepth);
+      m_tiles = (g.gm + BM - 1) / BM;
+      p.n_tiles_n = (int)((g.gn + p.bn - 1) / p.bn);
+      break;
+    }
+    case GK_CONV_FWD:
+    case GK_CONV_DGRAD: {
+      // rows run over the pixels of the OUTPUT tensor of this multiply; the shifted operand is the
+      // other activation tensor.  Only "same" geometry (odd taps, pad = (R-1)/2) is taken here.
+      if (g.Ho != g.H || g.Wo != g.W) return false;
+      const bool fwd = g.kind == GK_CONV_FWD;
+      const int Cc = fwd ? g.Ci : g.Co;        // contraction channels
+      const int Cn = fwd ? g.Co : g.Ci;        // output channels of this multiply
+      p.kdepth = pick_swizzle(Cc);
+      if (!p.kdepth || Cc % p.kdepth) return false;
+      if (!pick_pixel_box(g.W, g.H, g.B, p.Wt, p.Ht, p.Bt)) return false;
+      p.w_tiles = (g.W + p.Wt - 1) / p.Wt;
+      p.h_tiles = (g.H + p.Ht - 1) / p.Ht;
+      p.b_tiles = (g.B + p.Bt - 1) / p.Bt;
+      p.PW = g.W; p.PH = g.H; p.PB = g.B;
+      p.R = g.R; p.S = g.S; p.pad = g.pad;
+      p.c_chunks = Cc / p.kdepth;
+      p.Cn = Cn;
+      a_sw = p.kdepth;
+      sa = {4, {(cuuint64_t)Cc, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.B},
+            {(cuuint64_t)Cc, (cuuint64_t)Cc * g.W, (cuuint64_t)Cc * g.W * g.H},
+            {(cuuint32_t)p.kdepth, (cuuint32_t)p.Wt, (cuuint32_t)p.Ht, (cuuint32_t)p.Bt}, a_sw, g.p0};
+      if (fwd) {
+        p.bn = Cn >= 256 ? 256 : round_up32(Cn);
+        b_sw = p.kdepth;
+        sb = {2, {(cuuint64_t)g.gk, (cuuint64_t)Cn}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, (cuuint32_t)p.bn}, b_sw, g.p1};
+      } else {
+        b_mn = 1;
+        b_sw = pick_swizzle(Cn);
+        if (!b_sw || Cn % b_sw) return false;
+        p.bn = Cn >= 256 ? 256 : Cn;
+        if (p.bn % 32 || Cn % p.bn) return false;
+        // w viewed as [Co rows][R*S*Ci]: column = tap * Ci + ci
+        sb = {2, {(cuuint64_t)g.R * g.S * g.Ci, (cuuint64_t)g.Co}, {(cuuint64_t)g.R * g.S * g.Ci},
+              {(cuuint32_t)b_sw, (cuuint32_t)p.kdepth}, b_sw, g.p1};
+      }
+      p.kb_total = g.R * g.S * p.c_chunks;
+      m_tiles = (long long)p.w_tiles * p.h_tiles * p.b_tiles;
+      p.n_tiles_n = (Cn + p.bn - 1) / p.bn;
+      break;
+    }
+    case GK_CONV_WGRAD: {
+      if (g.Ho != g.H || g.Wo != g.W) return false;
+      a_mn = b_mn = 1;
+      a_sw = pick_swizzle(g.Co);
+      b_sw = pick_swizzle(g.Ci);
+      if (!a_sw || !b_sw || g.Co % a_sw || g.Ci % b_sw) return false;
+      if (!pick_pixel_box(g.W, g.H, g.B, p.Wt, p.Ht, p.Bt)) return false;
+      p.kdepth = 128;
+      p.w_tiles = (g.W + p.Wt - 1) / p.Wt;
+      p.h_tiles = (g.H + p.Ht - 1) / p.Ht;
+      p.b_tiles = (g.B + p.Bt - 1) / p.Bt;
+      p.PW = g.W; p.PH = g.H; p.PB = g.B;
+      p.R = g.R; p.S = g.S; p.pad = g.pad;
+      p.Cn = g.Ci;
+      p.bn = g.Ci >= 256 ? 256 : g.Ci;
+      if (p.bn % 32 || g.Ci % p.bn) return false;
+      p.n_chunks = g.Ci / p.bn;
+      sa = {4, {(cuuint64_t)g.Co, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.B},
+            {(cuuint64_t)g.Co, (cuuint64_t)g.Co * g.W, (cuuint64_t)g.Co * g.W * g.H},
+            {(cuuint32_t)a_sw, (cuuint32_t)p.Wt, (cuuint32_t)p.Ht, (cuuint32_t)p.Bt}, a_sw, g.p0};
+      sb = {4, {(cuuint64_t)g.Ci, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.B},
+            {(cuuint64_t)g.Ci, (cuuint64_t)g.Ci * g.W, (cuuint64_t)g.Ci * g.W * g.H},
+            {(cuuint32_t)b_sw, (cuuint32_t)p.Wt, (cuuint32_t)p.Ht, (cuuint32_t)p.Bt}, b_sw, g.p1};
+      p.kb_total = p.w_tiles * p.h_tiles * p.b_tiles;
+      m_tiles = (g.Co + BM - 1) / BM;
+      p.n_tiles_n = g.R * g.S * p.n_chunks;
+      break;
+    }
+    default:
+      return false;
+  }
+  p.ksteps = p.kdepth / 32;
+  // operand staging
+  if (a_mn) {
+    p.a_boxes = BM / a_sw;
+    if ((long long)p.a_boxes * a_sw > (g.gm + a_sw - 1) / a_sw * a_sw) p.a_boxes = (int)((g.gm + a_sw - 1) / a_sw);
+    p.a_box_bytes = p.kdepth * a_sw;
+    p.a_box_step = a_sw;
+    p.a_bytes = (BM / a_sw) * p.a_box_bytes;
+    p.a_desc = desc_mnmajor(a_sw, p.kdepth);
+    p.a_kstep16 = (unsigned)((32 * a_sw) >> 4);
+  } else {
+    p.a_boxes = 1;
+    p.a_box_bytes = BM * p.kdepth;
+    p.a_bytes = p.a_box_bytes;
+    p.a_desc = desc_kmajor(a_sw);
+    p.a_kstep16 = 2;
+  }
+  if (b_mn) {
+    p.b_boxes = p.bn / b_sw;
+    p.b_box_bytes = p.kdepth * b_sw;
+    p.b_box_step = b_sw;
+    p.b_bytes = p.b_boxes * p.b_box_bytes;
+    p.b_desc = desc_mnmajor(b_sw, p.kdepth);
+    p.b_kstep16 = (unsigned)((32 * b_sw) >> 4);
+  } else {
+    p.b_boxes = 1;
+    p.b_box_bytes = p.bn * p.kdepth;
+    p.b_bytes = p.b_box_bytes;
+    p.b_desc = desc_kmajor(b_sw);
+    p.b_kstep16 = 2;
+  }
+  // stage buffers must start on the swizzle period (1024 bytes)
+  p.a_bytes = (p.a_bytes + 1023) / 1024 * 1024;
+  p.b_bytes = (p.b_bytes + 1023) / 1024 * 1024;
+  int stage_bytes = p.a_bytes + p.b_bytes;
+  p.stages = (200 * 1024) / stage_bytes;
+  if (p.stages > MAX_STAGES) p.stages = MAX_STAGES;
+  if (p.stages < 2) return false;
+  // instruction descriptor: s32 accumulate, signed 8-bit operands, majorness, N, M
+  p.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((unsigned)a_mn << 15) | ((unsigned)b_mn << 16) |
+            ((unsigned)(p.bn >> 3) << 17) | ((unsigned)(BM >> 4) << 24);
+  long long tiles = m_tiles * p.n_tiles_n;
+  // split the contraction when the tiles alone cannot fill the SMs
+  if (tiles < ctx->sm_count && p.kb_total >= 8) {
+    long long s = (ctx->sm_count + tiles - 1) / tiles;
+    if (s > p.kb_total / 4) s = p.kb_total / 4;
+    if (s < 1) s = 1;
+    p.splits = (int)s;
+  }
+  p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
+  p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+  p.atomic_out = p.splits > 1;
+  p.items = tiles * p.splits;
+  if (!encode(ctx, &ma, sa) || !encode(ctx, &mb, sb)) return false;
+  return true;
+}
+
+}  // namespace
+
+int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr);
+
+size_t niti_tc_scratch_bytes(const GemmProblem &) { return 0; }
+
+int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, int32_t *acc, WsHeader *hdr, void *,
+                 size_t) {
+  TcParams p;
+  CUtensorMap ma, mb;
+  if (!plan(ctx, g, p, ma, mb)) return NITI_ERR_SHAPE;
+  size_t smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + 1024;
+  static size_t attr_smem = 0;
+  if (smem > attr_smem) {
+    NITI_CUDA_TRY(ctx, cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_smem = smem;
+  }
+  if (p.atomic_out) {
+    NITI_CUDA_TRY(ctx, cudaMemsetAsync(acc, 0, sizeof(int32_t) * (size_t)(g.gm * g.gn), st));
+    ctx->launches++;
+  }
+  long long grid = p.items < ctx->sm_count ? p.items : ctx->sm_count;
+  tc_gemm_kernel<<<(unsigned)grid, NUM_THREADS, smem, st>>>(ma, mb, p, acc, hdr, ctx->d_status);
+  ctx->launches++;
+  ctx->tc_launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  if (p.atomic_out) return niti_launch_maxabs(ctx, st, acc, g.gm * g.gn, hdr);
+  return NITI_OK;
+}

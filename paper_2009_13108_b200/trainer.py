@@ -1,0 +1,136 @@
+"""One integer training step (Algorithm 1 of the paper) as a fixed sequence of library calls.
+
+All tensors are allocated once; a step enqueues kernels on the current stream and never
+synchronises with the host, so it can be captured in a CUDA graph.  ReLU is fused into the
+forward epilogue, the ReLU mask into the dgrad epilogue, and the ReLU mask of a pooled layer
+into the max-pool backward."""
+from __future__ import annotations
+
+import torch
+
+from .api import Niti, ROUND_PSR
+
+
+class NitiTrainer:
+    def __init__(self, niti: Niti, net, weights, round_mode: int = ROUND_PSR):
+        """``net``: an object with ``batch``, ``in_shape``, ``s_in``, ``m_u`` and ``layers`` (dicts
+        with op in {"conv", "pool", "fc"}); ``weights``: int8 host arrays / tensors per weight
+        layer ([Cout,3,3,Cin] or [N,K])."""
+        self.n = niti
+        self.net = net
+        self.round_mode = round_mode
+        dev = niti.device
+        i8 = dict(dtype=torch.int8, device=dev)
+        self.weights = [torch.as_tensor(w).to(dev).contiguous() for w in weights]
+        self.s_in = niti.scalar(net.s_in)
+        self.x = torch.empty((net.batch,) + tuple(net.in_shape), **i8)
+        self.labels = torch.empty((net.batch,), dtype=torch.int32, device=dev)
+        # forward buffers
+        self.acts, self.s_act, self.b_fwd, self.s_w = [], [], [], []
+        shape = self.x.shape
+        wi = 0
+        max_act, max_w = 0, 0
+        for L in net.layers:
+            if L["op"] == "conv":
+                shape = (shape[0], shape[1], shape[2], L["cout"])
+            elif L["op"] == "pool":
+                shape = (shape[0], shape[1] // 2, shape[2] // 2, shape[3])
+            else:
+                shape = (shape[0], L["n"])
+            self.acts.append(torch.empty(shape, **i8))
+            self.s_act.append(niti.scalar())
+            self.b_fwd.append(niti.scalar(-1))
+            if L["op"] != "pool":
+                self.s_w.append(niti.scalar(L["s_w"]))
+                max_w = max(max_w, self.weights[wi].numel())
+                wi += 1
+            else:
+                self.s_w.append(None)
+            max_act = max(max_act, self.acts[-1].numel())
+        max_act = max(max_act, self.x.numel())
+        # backward buffers: two ping-pong error buffers and one gradient buffer
+        self.e_buf = [torch.empty(max_act, **i8), torch.empty(max_act, **i8)]
+        self.g_buf = torch.empty(max_w, **i8)
+        self.b_e = [niti.scalar(-1) for _ in net.layers]
+        self.b_g = [niti.scalar(-1) for _ in net.layers]
+        self.b_loss = niti.scalar()
+        self.n_correct = niti.scalar()
+        self.first_weight_layer = next(i for i, L in enumerate(net.layers) if L["op"] != "pool")
+
+    def load_batch(self, x, labels):
+        """Copies one batch (host or device tensors) into the resident input buffers."""
+        self.x.copy_(torch.as_tensor(x).reshape(self.x.shape), non_blocking=True)
+        self.labels.copy_(torch.as_tensor(labels), non_blocking=True)
+
+    def _view(self, buf, shape):
+        n = 1
+        for d in shape:
+            n *= d
+        return buf[:n].view(shape)
+
+    def forward(self):
+        n, net = self.n, self.net
+        a, s = self.x, self.s_in
+        wi = 0
+        for li, L in enumerate(net.layers):
+            out = self.acts[li]
+            if L["op"] == "conv":
+                n.conv_fwd(a, s, self.weights[wi], self.s_w[li], y=out, s_y=self.s_act[li],
+                           b_y=self.b_fwd[li], pad=1, relu=L["relu"], round_mode=self.round_mode)
+                s = self.s_act[li]
+                wi += 1
+            elif L["op"] == "fc":
+                n.linear_fwd(a.reshape(a.shape[0], -1), s, self.weights[wi], self.s_w[li], out=out,
+                             s_out=self.s_act[li], b_out=self.b_fwd[li], relu=L["relu"],
+                             round_mode=self.round_mode)
+                s = self.s_act[li]
+                wi += 1
+            else:
+                n.maxpool2_fwd(a, y=out)
+            a = out
+        return a, s
+
+    def step(self):
+        """Forward, integer loss gradient, backward with in-place weight update."""
+        n, net = self.n, self.net
+        logits, s_out = self.forward()
+        cur = 0
+        e = self._view(self.e_buf[cur], logits.shape)
+        n.int_xent(logits, s_out, self.labels, e=e, b_e=self.b_loss, n_correct=self.n_correct,
+                   round_mode=self.round_mode)
+        wi = len(self.weights)
+        for li in range(len(net.layers) - 1, -1, -1):
+            L = net.layers[li]
+            a_in = self.x if li == 0 else self.acts[li - 1]
+            if L["op"] == "pool":
+                nxt = self._view(self.e_buf[cur ^ 1], a_in.shape)
+                relu = bool(li > 0 and net.layers[li - 1].get("relu"))
+                n.maxpool2_bwd(a_in, e.view(self.acts[li].shape), e_in=nxt, relu=relu)
+                e, cur = nxt, cur ^ 1
+                continue
+            wi -= 1
+            w = self.weights[wi]
+            need_e = li != self.first_weight_layer
+            mask = None
+            if need_e and net.layers[li - 1]["op"] != "pool" and net.layers[li - 1].get("relu"):
+                mask = a_in
+            g = self._view(self.g_buf, w.shape)
+            nxt = self._view(self.e_buf[cur ^ 1], a_in.shape) if need_e else None
+            if L["op"] == "conv":
+                ev = e.view(self.acts[li].shape)
+                n.conv_wgrad(a_in, ev, (3, 3), g=g, b_g=self.b_g[li], pad=1, m_u=net.m_u,
+                             round_mode=self.round_mode)
+                if need_e:
+                    n.conv_dgrad(ev, w, a_in.shape[1:3], e_prev=nxt, relu_mask_src=mask,
+                                 b_e=self.b_e[li], pad=1, round_mode=self.round_mode)
+            else:
+                a2 = a_in.reshape(a_in.shape[0], -1)
+                n.linear_bwd(a2, e.view(a2.shape[0], -1), w, need_e_prev=need_e,
+                             relu_mask_src=None if mask is None else mask.reshape(a2.shape),
+                             e_prev=None if nxt is None else nxt.view(a2.shape), g=g,
+                             b_e=self.b_e[li], b_g=self.b_g[li], m_u=net.m_u,
+                             round_mode=self.round_mode)
+            n.int_sgd_update(w, g)
+            if need_e:
+                e, cur = nxt, cur ^ 1
+        return self.n_correct
