@@ -97,6 +97,14 @@ uint64_t niti_launch_count(niti_ctx *ctx);
 /* Of those, launches of the tensor-core (tcgen05) matrix-multiply kernel. */
 uint64_t niti_tc_launch_count(niti_ctx *ctx);
 
+/* Timing of the tensor-core matrix-multiply kernel.  While enabled, every launch of that
+ * kernel is bracketed by a pair of CUDA events on its stream (up to 8192 launches are kept).
+ * niti_profile_read() waits for the recorded events, returns their summed duration in
+ * milliseconds, their count and the summed algorithmic int8 operations (2*M*N*K of each
+ * multiply), and starts a new record.  Host pointers. */
+int niti_profile_enable(niti_ctx *ctx, int on);
+int niti_profile_read(niti_ctx *ctx, double *tc_ms, uint64_t *tc_launches, double *tc_ops);
+
 /* Fully connected forward (Algorithm 1, forward loop; Section 3.2):
  *   acc[m][n] = sum_k a[m][k] * w[n][k];  b = B(acc);  bp = max(0, b - 7);
  *   out = Round(acc, bp) (then max(.,0) if relu);  *s_out = *s_a + *s_w + bp.

@@ -486,5 +486,9 @@ int niti_ref_int_xent(const int8_t *a, int32_t s_a, const int32_t *labels, int8_
     return rc;
   }
   if (n_correct) *n_correct = niti_ref_count_correct(a, labels, B, N);
-  return finish(e32, B * N, 7, round_mode, e, b_e, NULL);
+  /* the loss accumulators are 64-bit quantities (up to 2^45 at s_a = -22): the int32 contract of
+   * the matrix multiplies does not apply to them */
+  rc = niti_ref_shift_round(e32, B * N, 7, round_mode, e, b_e, NULL);
+  free(e32);
+  return rc;
 }

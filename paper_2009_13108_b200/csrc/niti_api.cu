@@ -39,6 +39,11 @@ extern "C" int niti_create(niti_ctx **out, int device) {
 
 extern "C" int niti_destroy(niti_ctx *ctx) {
   if (!ctx) return NITI_ERR_ARG;
+  if (ctx->prof_ev) {
+    for (int i = 0; i < 2 * NITI_PROF_MAX; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+    delete[] ctx->prof_ev;
+    delete[] ctx->prof_ops;
+  }
   cudaFree(ctx->d_status);
   delete ctx;
   return NITI_OK;
@@ -55,6 +60,35 @@ extern "C" int niti_set_engine(niti_ctx *ctx, int engine) {
 
 extern "C" uint64_t niti_launch_count(niti_ctx *ctx) { return ctx ? ctx->launches : 0; }
 extern "C" uint64_t niti_tc_launch_count(niti_ctx *ctx) { return ctx ? ctx->tc_launches : 0; }
+
+extern "C" int niti_profile_enable(niti_ctx *ctx, int on) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (on && !ctx->prof_ev) {
+    ctx->prof_ev = new cudaEvent_t[2 * NITI_PROF_MAX];
+    ctx->prof_ops = new double[NITI_PROF_MAX];
+    for (int i = 0; i < 2 * NITI_PROF_MAX; ++i) NITI_CUDA_TRY(ctx, cudaEventCreate(&ctx->prof_ev[i]));
+  }
+  ctx->profile_on = on ? 1 : 0;
+  ctx->prof_used = 0;
+  return NITI_OK;
+}
+
+extern "C" int niti_profile_read(niti_ctx *ctx, double *tc_ms, uint64_t *tc_launches, double *tc_ops) {
+  if (!ctx || !tc_ms || !tc_launches || !tc_ops) return NITI_ERR_ARG;
+  double ms = 0, ops = 0;
+  for (int i = 0; i < ctx->prof_used; ++i) {
+    float t = 0;
+    NITI_CUDA_TRY(ctx, cudaEventSynchronize(ctx->prof_ev[2 * i + 1]));
+    NITI_CUDA_TRY(ctx, cudaEventElapsedTime(&t, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]));
+    ms += t;
+    ops += ctx->prof_ops[i];
+  }
+  *tc_ms = ms;
+  *tc_launches = (uint64_t)ctx->prof_used;
+  *tc_ops = ops;
+  ctx->prof_used = 0;
+  return NITI_OK;
+}
 
 extern "C" int niti_check(niti_ctx *ctx, void *stream, uint32_t *status) {
   if (!ctx) return NITI_ERR_ARG;

@@ -16,10 +16,16 @@ struct niti_ctx {
   uint64_t launches;
   uint64_t tc_launches;     // launches of the tensor-core matrix-multiply kernel
   char err[256];
+  // optional timing of the tensor-core kernel: event pairs recorded around each launch
+  int profile_on;
+  int prof_used;
+  cudaEvent_t *prof_ev;     // 2 * NITI_PROF_MAX events
+  double *prof_ops;         // algorithmic int8 operations (2*M*N*K) of each recorded launch
   // cuTensorMapEncodeTiled, fetched through the runtime so that libcuda is not a link dependency
   void *encode_tiled;
 };
 
+#define NITI_PROF_MAX 8192
 #define NITI_WS_HEADER 256  // bytes reserved at the start of every workspace for reduction scalars
 
 // Scalars at the start of a workspace.

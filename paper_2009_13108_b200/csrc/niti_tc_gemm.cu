@@ -682,7 +682,14 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, int32_t *
     ctx->launches++;
   }
   long long grid = p.items < ctx->sm_count ? p.items : ctx->sm_count;
+  const bool prof = ctx->profile_on && ctx->prof_ev && ctx->prof_used < NITI_PROF_MAX;
+  if (prof) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st);
   tc_gemm_kernel<<<(unsigned)grid, NUM_THREADS, smem, st>>>(ma, mb, p, acc, hdr, ctx->d_status);
+  if (prof) {
+    cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st);
+    ctx->prof_ops[ctx->prof_used] = 2.0 * (double)g.gm * (double)g.gn * (double)g.gk;
+    ctx->prof_used++;
+  }
   ctx->launches++;
   ctx->tc_launches++;
   NITI_CUDA_TRY(ctx, cudaGetLastError());

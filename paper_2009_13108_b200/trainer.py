@@ -22,6 +22,7 @@ class NitiTrainer:
         dev = niti.device
         i8 = dict(dtype=torch.int8, device=dev)
         self.weights = [torch.as_tensor(w).to(dev).contiguous() for w in weights]
+        self._initial = None
         self.s_in = niti.scalar(net.s_in)
         self.x = torch.empty((net.batch,) + tuple(net.in_shape), **i8)
         self.labels = torch.empty((net.batch,), dtype=torch.int32, device=dev)
@@ -56,6 +57,15 @@ class NitiTrainer:
         self.b_loss = niti.scalar()
         self.n_correct = niti.scalar()
         self.first_weight_layer = next(i for i, L in enumerate(net.layers) if L["op"] != "pool")
+
+    def snapshot_weights(self):
+        """Keeps a device copy of the current weights for reset_weights()."""
+        self._initial = [w.clone() for w in self.weights]
+
+    def reset_weights(self):
+        """Restores the snapshot (device-to-device copies on the current stream)."""
+        for w, w0 in zip(self.weights, self._initial):
+            w.copy_(w0, non_blocking=True)
 
     def load_batch(self, x, labels):
         """Copies one batch (host or device tensors) into the resident input buffers."""

@@ -8,6 +8,7 @@ from .workloads import (  # noqa: F401
     config_net,
     gaussian_like_int8,
     gemm_operands,
+    gemm_grad_operands,
     he_like_exponent,
     make_net_inputs,
     uniform_int8,

@@ -158,3 +158,11 @@ def gemm_operands(M: int, N: int, K: int, dist: str = "uniform", seed: int = 1):
     rng = np.random.Generator(np.random.PCG64([seed, M, N, K, 0 if dist == "uniform" else 1]))
     gen = uniform_int8 if dist == "uniform" else gaussian_like_int8
     return gen(rng, (M, K)), gen(rng, (N, K))
+
+
+def gemm_grad_operands(M: int, N: int, K: int, dist: str = "uniform", seed: int = 1):
+    """Operands of the sweep's gradient variant: e[K,M] and a[K,N]; the product
+    g[M,N] = sum_k e[k,m] a[k,n] contracts over the rows of both (a weight-gradient multiply)."""
+    rng = np.random.Generator(np.random.PCG64([seed, M, N, K, 2 if dist == "uniform" else 3]))
+    gen = uniform_int8 if dist == "uniform" else gaussian_like_int8
+    return gen(rng, (K, M)), gen(rng, (K, N))

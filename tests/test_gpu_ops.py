@@ -1,0 +1,233 @@
+"""Bit-exact parity of every C-ABI op against the CPU oracle on seeded inputs (GPU only).
+
+Sizes are chosen so the oracle finishes in seconds while the tensor-core engine still sees
+several tiles, ragged tails, every operand layout (K-major / MN-major, 32/64/128-byte swizzle),
+split contractions and the fallback engine."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def niti():
+    from paper_2009_13108_b200 import Niti
+    n = Niti(0)
+    yield n
+    n.check()
+    n.close()
+
+
+def _i8(rng, shape):
+    return rng.integers(-127, 128, size=shape, dtype=np.int8)
+
+
+def _T(niti, a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(niti.device)
+
+
+def _eq(t, want):
+    got = t.cpu().numpy()
+    assert got.shape == want.shape
+    assert np.array_equal(got, want), "mismatch at %s" % np.argwhere(got != want)[:4].tolist()
+
+
+FC_SHAPES = [(64, 256, 784), (64, 10, 256), (300, 520, 384), (128, 256, 128), (130, 70, 100),
+             (257, 300, 96), (1, 32, 32), (64, 1000, 512), (512, 384, 2048)]
+
+
+@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("M,N,K", FC_SHAPES)
+def test_linear_fwd(niti, oref, M, N, K, engine):
+    rng = np.random.default_rng(M * 7 + N * 3 + K)
+    a, w = _i8(rng, (M, K)), _i8(rng, (N, K))
+    niti.set_engine(engine)
+    try:
+        for relu, mode in [(False, 0), (True, 0), (False, 1)]:
+            want, s, b = oref.linear_fwd(a, -7, w, -10, relu, mode)
+            out, s_out, b_out = niti.linear_fwd(_T(niti, a), niti.scalar(-7), _T(niti, w),
+                                                niti.scalar(-10), relu=relu, round_mode=mode)
+            _eq(out, want)
+            assert (int(s_out), int(b_out)) == (s, b)
+    finally:
+        niti.set_engine(0)
+    niti.check()
+
+
+@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("M,N,K", FC_SHAPES[:7] + [(640, 256, 512)])
+def test_linear_bwd(niti, oref, M, N, K, engine):
+    rng = np.random.default_rng(M * 5 + N * 11 + K)
+    a, w, e = _i8(rng, (M, K)), _i8(rng, (N, K)), _i8(rng, (M, N))
+    mask = np.maximum(a, 0)
+    niti.set_engine(engine)
+    try:
+        for m_u, use_mask in [(5, True), (3, False)]:
+            we, wg, be, bg = oref.linear_bwd(a, e, w, True, mask if use_mask else None, m_u)
+            ep, g, b_e, b_g = niti.linear_bwd(_T(niti, a), _T(niti, e), _T(niti, w), True,
+                                              _T(niti, mask) if use_mask else None, m_u=m_u)
+            _eq(ep, we)
+            _eq(g, wg)
+            assert (int(b_e), int(b_g)) == (be, bg)
+            assert int(g.abs().max()) <= 2 ** m_u - 1
+        # first layer: no error to propagate
+        _, wg, _, bg = oref.linear_bwd(a, e, w, False, None, 5)
+        ep, g, _, b_g = niti.linear_bwd(_T(niti, a), _T(niti, e), _T(niti, w), False)
+        assert ep is None
+        _eq(g, wg)
+    finally:
+        niti.set_engine(0)
+    niti.check()
+
+
+CONV_SHAPES = [(2, 8, 8, 3, 16), (2, 16, 16, 64, 64), (4, 8, 8, 128, 256), (8, 4, 4, 256, 128),
+               (2, 32, 32, 32, 64), (3, 28, 28, 1, 32), (2, 28, 28, 32, 64), (32, 2, 2, 512, 512),
+               (1, 56, 56, 64, 128), (2, 12, 20, 96, 160)]
+
+
+@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("B,H,W,Ci,Co", CONV_SHAPES)
+def test_conv_ops(niti, oref, B, H, W, Ci, Co, engine):
+    rng = np.random.default_rng(B + H * 3 + W * 5 + Ci * 7 + Co * 11)
+    x, w, e = _i8(rng, (B, H, W, Ci)), _i8(rng, (Co, 3, 3, Ci)), _i8(rng, (B, H, W, Co))
+    xm = np.maximum(x, 0)
+    niti.set_engine(engine)
+    try:
+        wy, s, b = oref.conv_fwd(x, -7, w, -9, 1, True)
+        y, s_y, b_y = niti.conv_fwd(_T(niti, x), niti.scalar(-7), _T(niti, w), niti.scalar(-9),
+                                    relu=True)
+        _eq(y, wy)
+        assert (int(s_y), int(b_y)) == (s, b)
+        wd, bd = oref.conv_dgrad(e, w, (H, W), 1, xm)
+        ep, b_e = niti.conv_dgrad(_T(niti, e), _T(niti, w), (H, W), relu_mask_src=_T(niti, xm))
+        _eq(ep, wd)
+        assert int(b_e) == bd
+        wg, bg = oref.conv_wgrad(x, e, (3, 3), 1, 5)
+        g, b_g = niti.conv_wgrad(_T(niti, x), _T(niti, e))
+        _eq(g, wg)
+        assert int(b_g) == bg
+    finally:
+        niti.set_engine(0)
+    niti.check()
+
+
+def test_tensor_core_engine_is_the_one_that_runs(niti):
+    rng = np.random.default_rng(1)
+    before = niti.tc_launch_count()
+    a, w = _T(niti, _i8(rng, (256, 512))), _T(niti, _i8(rng, (256, 512)))
+    niti.linear_fwd(a, niti.scalar(-7), w, niti.scalar(-10))
+    x, wc = _T(niti, _i8(rng, (2, 16, 16, 64))), _T(niti, _i8(rng, (64, 3, 3, 64)))
+    e = _T(niti, _i8(rng, (2, 16, 16, 64)))
+    niti.conv_fwd(x, niti.scalar(-7), wc, niti.scalar(-9))
+    niti.conv_dgrad(e, wc, (16, 16))
+    niti.conv_wgrad(x, e)
+    niti.linear_bwd(a, _T(niti, _i8(rng, (256, 256))), w)
+    assert niti.tc_launch_count() - before == 6
+    niti.check()
+
+
+def test_general_taps_and_padding_use_the_fallback(niti, oref):
+    rng = np.random.default_rng(2)
+    x, w = _i8(rng, (2, 9, 9, 4)), _i8(rng, (6, 5, 5, 4))
+    for pad in (0, 2):
+        wy, s, b = oref.conv_fwd(x, -7, w, -9, pad, False)
+        y, s_y, b_y = niti.conv_fwd(_T(niti, x), niti.scalar(-7), _T(niti, w), niti.scalar(-9),
+                                    pad=pad)
+        _eq(y, wy)
+        e = _i8(rng, wy.shape)
+        wd, _ = oref.conv_dgrad(e, w, (9, 9), pad)
+        _eq(niti.conv_dgrad(_T(niti, e), _T(niti, w), (9, 9), pad=pad)[0], wd)
+        wg, _ = oref.conv_wgrad(x, e, (5, 5), pad, 5)
+        _eq(niti.conv_wgrad(_T(niti, x), _T(niti, e), (5, 5), pad=pad)[0], wg)
+    niti.check()
+
+
+def test_saturation_and_zero_tensor(niti, oref):
+    # all-zero accumulators: b = 0, output zero, exponent = s_a + s_w
+    a = np.zeros((32, 64), np.int8)
+    w = _i8(np.random.default_rng(3), (32, 64))
+    out, s_out, b_out = niti.linear_fwd(_T(niti, a), niti.scalar(-7), _T(niti, w), niti.scalar(-3))
+    assert int(out.abs().max()) == 0 and int(b_out) == 0 and int(s_out) == -10
+    # an accumulator whose integer part is already 127 and whose fraction asks for +1
+    a = np.zeros((32, 64), np.int8)
+    w = np.zeros((32, 64), np.int8)
+    a[0, :4] = [127, 127, 1, 0]
+    w[0, :4] = [127, 127, 127, 0]      # 32385: 15 bits, bp = 8, q = 126 ... generic check below
+    a[1, :3] = [127, 127, 127]
+    w[1, :3] = [86, 0, 0]
+    want, s, b = oref.linear_fwd(a, 0, w, 0)
+    out, s_out, b_out = niti.linear_fwd(_T(niti, a), niti.scalar(0), _T(niti, w), niti.scalar(0))
+    _eq(out, want)
+    assert int(out.max()) <= 127 and int(out.min()) >= -127
+
+
+@pytest.mark.parametrize("s_a", [-22, -9, -7, -6, -4, 0, 24])
+@pytest.mark.parametrize("B,N", [(64, 10), (64, 1000), (7, 33), (256, 10)])
+def test_int_xent(niti, oref, s_a, B, N):
+    rng = np.random.default_rng(1000 + s_a + B + N)
+    a = _i8(rng, (B, N))
+    labels = rng.integers(0, N, size=B).astype(np.int32)
+    for mode in (0, 1):
+        want, b, nc = oref.int_xent(a, s_a, labels, mode)
+        e, b_e, n_correct = niti.int_xent(_T(niti, a), niti.scalar(s_a), _T(niti, labels),
+                                          round_mode=mode)
+        _eq(e, want)
+        assert (int(b_e), int(n_correct)) == (b, nc)
+    niti.check()
+
+
+def test_int_xent_flags_bad_domain(niti):
+    from paper_2009_13108_b200 import NitiError
+    a = torch.zeros((4, 8), dtype=torch.int8, device=niti.device)
+    labels = torch.zeros(4, dtype=torch.int32, device=niti.device)
+    niti.int_xent(a, niti.scalar(30), labels)
+    with pytest.raises(NitiError):
+        niti.check()
+    labels[2] = 8
+    niti.int_xent(a, niti.scalar(-4), labels)
+    with pytest.raises(NitiError):
+        niti.check()
+    assert niti.check() == 0
+
+
+@pytest.mark.parametrize("n", [1, 15, 16, 17, 4096, 100003, 1 << 22])
+def test_sgd_update_and_relu(niti, oref, n):
+    rng = np.random.default_rng(n)
+    w, g = _i8(rng, n), _i8(rng, n)
+    wt = _T(niti, w)
+    niti.int_sgd_update(wt, _T(niti, g))
+    _eq(wt, oref.sgd_update(w, g))
+    x, e = _i8(rng, n), _i8(rng, n)
+    y = niti.relu_fwd(_T(niti, x))
+    _eq(y, oref.relu_fwd(x))
+    _eq(niti.relu_bwd(y, _T(niti, e)), oref.relu_bwd(oref.relu_fwd(x), e))
+
+
+@pytest.mark.parametrize("B,H,W,C", [(2, 4, 6, 16), (3, 8, 8, 5), (2, 28, 28, 64), (1, 2, 2, 1),
+                                     (4, 6, 10, 48)])
+def test_maxpool(niti, oref, B, H, W, C):
+    rng = np.random.default_rng(B + H + W + C)
+    x = np.maximum(rng.integers(-40, 40, size=(B, H, W, C)), 0).astype(np.int8)   # many ties
+    e = _i8(rng, (B, H // 2, W // 2, C))
+    y = niti.maxpool2_fwd(_T(niti, x))
+    _eq(y, oref.maxpool2_fwd(x))
+    _eq(niti.maxpool2_bwd(_T(niti, x), _T(niti, e), relu=False), oref.maxpool2_bwd(x, e))
+    _eq(niti.maxpool2_bwd(_T(niti, x), _T(niti, e), relu=True),
+        oref.relu_bwd(x, oref.maxpool2_bwd(x, e)))
+    xs = _i8(rng, (B, H, W, C))
+    _eq(niti.maxpool2_bwd(_T(niti, xs), _T(niti, e)), oref.maxpool2_bwd(xs, e))
+
+
+def test_argument_errors(niti):
+    from paper_2009_13108_b200 import NitiError
+    a = torch.zeros((4, 32), dtype=torch.int8, device=niti.device)
+    with pytest.raises(NitiError) as ei:
+        niti.linear_bwd(a, a, a, m_u=9)
+    assert ei.value.code == 1
+    # too small a workspace is refused
+    import ctypes
+    rc = niti.lib.niti_linear_fwd(niti.h, None, a.data_ptr(), niti.scalar().data_ptr(), a.data_ptr(),
+                                  niti.scalar().data_ptr(), a.data_ptr(), None, None, 4, 4, 32, 0, 0,
+                                  niti._ws.data_ptr(), ctypes.c_size_t(16))
+    assert rc == 3
