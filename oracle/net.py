@@ -88,6 +88,8 @@ def oracle_train_step(net, x, labels, state: OracleNetState, round_mode=ref.ROUN
                                                  net.m_u, round_mode, allow_overflow)
             if e_prev is not None:
                 e_prev = e_prev.reshape(a_in.shape)
+            else:
+                b_e = -1
         rec["b_e"].append(b_e)
         rec["b_g"].append(b_g)
         if keep_tensors:
