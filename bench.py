@@ -298,7 +298,17 @@ def main():
     ap.add_argument("--config", type=int, default=4, choices=[0, 2, 3, 4])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-gemm", dest="gemm", action="store_false")
+    ap.add_argument("--gemm-shape", default=None,
+                    help="MxNxK: time only the fused GEMM at this shape (for profiling a small case)")
+    ap.add_argument("--iters", type=int, default=10)
     args = ap.parse_args()
+    if args.gemm_shape:
+        from paper_2009_13108_b200 import Niti
+        niti = Niti(0)
+        M, N, K = (int(v) for v in args.gemm_shape.lower().split("x"))
+        print(json.dumps(gemm_point(niti, M, N, K, iters=args.iters)), flush=True)
+        niti.check()
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
