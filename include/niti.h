@@ -88,14 +88,19 @@ int niti_check(niti_ctx *ctx, void *stream, uint32_t *status);
 size_t niti_workspace_bytes(int op, const int64_t *dims, int ndims);
 
 /* Selects the matrix-multiply engine: 0 = automatic (tensor cores whenever
- * the shape allows, default), 1 = force the plain CUDA-core kernels (used by
- * tests to cross-check the two engines).  Returns the previous value. */
+ * the shape allows; pairs of CTAs on 256-row tiles when there are enough of
+ * them; default), 1 = plain CUDA-core kernels only, 2 = tensor cores with the
+ * single-CTA kernel only, 3 = tensor cores with the paired-CTA kernel only
+ * (falls back to CUDA cores where that kernel does not apply).  1-3 exist so
+ * that tests can cross-check the engines.  Returns the previous value. */
 int niti_set_engine(niti_ctx *ctx, int engine);
 
 /* Number of kernels / memsets this context has enqueued so far. */
 uint64_t niti_launch_count(niti_ctx *ctx);
 /* Of those, launches of the tensor-core (tcgen05) matrix-multiply kernel. */
 uint64_t niti_tc_launch_count(niti_ctx *ctx);
+/* Of those, launches of the paired-CTA (cta_group::2) variant. */
+uint64_t niti_tc_pair_launch_count(niti_ctx *ctx);
 
 /* Timing of the tensor-core matrix-multiply kernel.  While enabled, every launch of that
  * kernel is bracketed by a pair of CUDA events on its stream (up to 8192 launches are kept).

@@ -60,6 +60,7 @@ extern "C" int niti_set_engine(niti_ctx *ctx, int engine) {
 
 extern "C" uint64_t niti_launch_count(niti_ctx *ctx) { return ctx ? ctx->launches : 0; }
 extern "C" uint64_t niti_tc_launch_count(niti_ctx *ctx) { return ctx ? ctx->tc_launches : 0; }
+extern "C" uint64_t niti_tc_pair_launch_count(niti_ctx *ctx) { return ctx ? ctx->tc2_launches : 0; }
 
 extern "C" int niti_profile_enable(niti_ctx *ctx, int on) {
   if (!ctx) return NITI_ERR_ARG;
@@ -189,7 +190,7 @@ static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, 
   NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, sizeof(WsHeader), st));
   ctx->launches++;
   int rc = NITI_ERR_SHAPE;
-  if (ctx->engine == 0) rc = niti_tc_gemm(ctx, st, p, acc, hdr, scratch, scratch_bytes);
+  if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, acc, hdr, scratch, scratch_bytes);
   if (rc == NITI_ERR_SHAPE) rc = niti_simt_gemm(ctx, st, p, acc, hdr);
   if (rc != NITI_OK) return rc;
   return niti_launch_round(ctx, st, acc, hdr, out, p.gm * p.gn, mbits, round_mode, relu, mask, s_a, s_w,

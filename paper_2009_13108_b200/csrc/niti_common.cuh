@@ -11,10 +11,11 @@
 struct niti_ctx {
   int device;
   int sm_count;
-  int engine;               // 0 auto, 1 force CUDA-core kernels
+  int engine;               // 0 auto, 1 CUDA-core kernels only, 2 single-CTA tensor-core kernel, 3 paired-CTA only
   uint32_t *d_status;       // device status word
   uint64_t launches;
   uint64_t tc_launches;     // launches of the tensor-core matrix-multiply kernel
+  uint64_t tc2_launches;    // of those, launches of the paired-CTA (cta_group::2) variant
   char err[256];
   // optional timing of the tensor-core kernel: event pairs recorded around each launch
   int profile_on;

@@ -51,6 +51,9 @@ struct TcParams {
   int c_chunks;                 // channel chunks per tap along the contraction (fwd / dgrad)
   int Cn;                       // wgrad: input channels Ci (columns per tap)
   int n_chunks;                 // wgrad: column chunks per tap
+  int ctas;                     // CTAs per tile: 1, or 2 (cta_group::2, 256-row tiles)
+  int m_units;                  // row units: 128-row tiles (ctas = 1) or 256-row pairs (ctas = 2)
+  int raster_g;                 // row units per rasterisation group (0: row-major order)
 };
 
 // ------------------------------------------------------------------------------------------
@@ -146,8 +149,87 @@ __device__ __forceinline__ void pixel_box(const TcParams &p, int idx, int &w0, i
 }
 
 // ------------------------------------------------------------------------------------------
+// Cluster helpers (CTAS == 2: a pair of CTAs on neighbouring SMs works on one 256-row tile with
+// tcgen05 cta_group::2; the even CTA of the pair issues the MMAs and owns the barriers).
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned cluster_ctarank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ unsigned map_to_cta(unsigned local_addr, unsigned rank) {
+  unsigned r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(unsigned cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1,
+                                                 int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(unsigned bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((unsigned short)3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_i8_pair(unsigned tmem_d, unsigned long long da, unsigned long long db,
+                                               unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+template <int CTAS>
+__device__ __forceinline__ void load2(unsigned dst, const CUtensorMap *m, unsigned bar, int c0, int c1) {
+  if (CTAS == 2) tma_load_2d_pair(dst, m, bar, c0, c1); else tma_load_2d(dst, m, bar, c0, c1);
+}
+template <int CTAS>
+__device__ __forceinline__ void load4(unsigned dst, const CUtensorMap *m, unsigned bar, int c0, int c1, int c2, int c3) {
+  if (CTAS == 2) tma_load_4d_pair(dst, m, bar, c0, c1, c2, c3); else tma_load_4d(dst, m, bar, c0, c1, c2, c3);
+}
+
+// item -> (row unit, column tile, split).  Row units (one CTA's 128 rows, or a pair's 256) are
+// visited in groups of raster_g so that the CTAs running at the same time share operand tiles in L2.
+__device__ __forceinline__ void decode_item(const TcParams &p, long long item, int &mu, int &nt, int &split) {
+  const long long tile = item / p.splits;
+  split = (int)(item % p.splits);
+  if (p.raster_g <= 0) {
+    mu = (int)(tile / p.n_tiles_n);
+    nt = (int)(tile % p.n_tiles_n);
+    return;
+  }
+  const long long per_group = (long long)p.raster_g * p.n_tiles_n;
+  const int g = (int)(tile / per_group);
+  const int rem = (int)(tile % per_group);
+  int in_group = p.m_units - g * p.raster_g;
+  if (in_group > p.raster_g) in_group = p.raster_g;
+  mu = g * p.raster_g + rem % in_group;
+  nt = rem / in_group;
+}
+
+// ------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------
+template <int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const TcParams p, int32_t *__restrict__ acc, WsHeader *hdr, uint32_t *status) {
@@ -157,12 +239,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ volatile int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned rank = CTAS == 2 ? cluster_ctarank() : 0u;
   const unsigned smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int stage_bytes = p.a_bytes + p.b_bytes;
   const unsigned full0 = smem_u32(&bars[0]);
   const unsigned empty0 = smem_u32(&bars[MAX_STAGES]);
   const unsigned tfull0 = smem_u32(&bars[2 * MAX_STAGES]);
   const unsigned tempty0 = smem_u32(&bars[2 * MAX_STAGES + 2]);
+  // barriers of the leader CTA as seen from this CTA
+  const unsigned lead_full0 = CTAS == 2 ? map_to_cta(full0, 0) : full0;
+  const unsigned lead_tempty0 = CTAS == 2 ? map_to_cta(tempty0, 0) : tempty0;
+  const long long first_item = blockIdx.x / CTAS;
+  const long long item_step = gridDim.x / CTAS;
 
   // TMEM columns: two accumulator buffers of bn columns, rounded up to a power of two >= 32
   unsigned tmem_cols = 32;
@@ -176,72 +264,86 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull0 + 8 * b, 1);
-      mbar_init(tempty0 + 8 * b, 4);     // one arrival per epilogue warp
+      mbar_init(tempty0 + 8 * b, 4 * CTAS);     // one arrival per epilogue warp of every CTA
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CTAS == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();   // the peer's barriers exist before anyone signals them
   tc_fence_after();
   const unsigned tmem_base = tmem_base_slot;
 
   if (warp == 0) {
-    // ================= TMA producer =================
+    // ================= TMA producer (every CTA loads its own rows of A and its share of B) ========
     if (lane == 0) {
       int stage = 0;
       unsigned phase = 0;
       bool ok = true;
-      for (long long item = blockIdx.x; ok && item < p.items; item += gridDim.x) {
-        const long long tile = item / p.splits;
-        const int split = (int)(item % p.splits);
-        const int mt = (int)(tile / p.n_tiles_n), nt = (int)(tile % p.n_tiles_n);
+      const int bn_cta = p.bn / CTAS;             // B rows (output columns) staged by this CTA
+      for (long long item = first_item; ok && item < p.items; item += item_step) {
+        int mu, nt, split;
+        decode_item(p, item, mu, nt, split);
+        const int mt = mu * CTAS + (int)rank;     // this CTA's 128-row tile
+        const int nb = nt * p.bn + (int)rank * bn_cta;
         const int kb0 = split * p.kb_per_split;
         int kb1 = kb0 + p.kb_per_split;
         if (kb1 > p.kb_total) kb1 = p.kb_total;
         int w0 = 0, h0 = 0, b0 = 0, tap_n = 0, ci0 = 0;
         if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) pixel_box(p, mt, w0, h0, b0);
-        if (p.kind == GK_CONV_WGRAD) { tap_n = nt / p.n_chunks; ci0 = (nt % p.n_chunks) * p.bn; }
+        if (p.kind == GK_CONV_WGRAD) {
+          tap_n = nt / p.n_chunks;
+          ci0 = (nt % p.n_chunks) * p.bn + (int)rank * bn_cta;
+        }
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
-          const unsigned full = full0 + 8 * stage;
+          const unsigned full = lead_full0 + 8 * stage;
           const unsigned sa = smem_base + stage * stage_bytes;
           const unsigned sb = sa + p.a_bytes;
-          mbar_expect_tx(full, (unsigned)(p.a_boxes * p.a_box_bytes + p.b_boxes * p.b_box_bytes));
+          if (rank == 0)
+            mbar_expect_tx(full0 + 8 * stage,
+                           (unsigned)(CTAS * (p.a_boxes * p.a_box_bytes + p.b_boxes * p.b_box_bytes)));
           switch (p.kind) {
             case GK_FC_FWD:       // A [M][K] K-major, B [N][K] K-major
-              tma_load_2d(sa, &map_a, full, kb * p.kdepth, mt * BM);
-              tma_load_2d(sb, &map_b, full, kb * p.kdepth, nt * p.bn);
+              load2<CTAS>(sa, &map_a, full, kb * p.kdepth, mt * BM);
+              load2<CTAS>(sb, &map_b, full, kb * p.kdepth, nb);
               break;
             case GK_FC_DGRAD:     // A = e [M][N] K-major; B(k', n) = w[n][k'] MN-major
-              tma_load_2d(sa, &map_a, full, kb * p.kdepth, mt * BM);
+              load2<CTAS>(sa, &map_a, full, kb * p.kdepth, mt * BM);
               for (int j = 0; j < p.b_boxes; ++j)
-                tma_load_2d(sb + j * p.b_box_bytes, &map_b, full, nt * p.bn + j * p.b_box_step, kb * p.kdepth);
+                load2<CTAS>(sb + j * p.b_box_bytes, &map_b, full, nb + j * p.b_box_step, kb * p.kdepth);
               break;
             case GK_FC_WGRAD:     // A(n, m) = e[m][n] MN-major; B(k', m) = a[m][k'] MN-major
               for (int j = 0; j < p.a_boxes; ++j)
-                tma_load_2d(sa + j * p.a_box_bytes, &map_a, full, mt * BM + j * p.a_box_step, kb * p.kdepth);
+                load2<CTAS>(sa + j * p.a_box_bytes, &map_a, full, mt * BM + j * p.a_box_step, kb * p.kdepth);
               for (int j = 0; j < p.b_boxes; ++j)
-                tma_load_2d(sb + j * p.b_box_bytes, &map_b, full, nt * p.bn + j * p.b_box_step, kb * p.kdepth);
+                load2<CTAS>(sb + j * p.b_box_bytes, &map_b, full, nb + j * p.b_box_step, kb * p.kdepth);
               break;
             case GK_CONV_FWD: {   // k-block = (tap, channel chunk)
               int tap = kb / p.c_chunks, cc = kb % p.c_chunks;
               int r = tap / p.S, s = tap % p.S;
-              tma_load_4d(sa, &map_a, full, cc * p.kdepth, w0 + s - p.pad, h0 + r - p.pad, b0);
-              tma_load_2d(sb, &map_b, full, kb * p.kdepth, nt * p.bn);
+              load4<CTAS>(sa, &map_a, full, cc * p.kdepth, w0 + s - p.pad, h0 + r - p.pad, b0);
+              load2<CTAS>(sb, &map_b, full, kb * p.kdepth, nb);
               break;
             }
             case GK_CONV_DGRAD: { // A = e shifted the other way; B(ci, (tap, co)) = w[co][tap][ci]
               int tap = kb / p.c_chunks, cc = kb % p.c_chunks;
               int r = tap / p.S, s = tap % p.S;
-              tma_load_4d(sa, &map_a, full, cc * p.kdepth, w0 - s + p.pad, h0 - r + p.pad, b0);
+              load4<CTAS>(sa, &map_a, full, cc * p.kdepth, w0 - s + p.pad, h0 - r + p.pad, b0);
               for (int j = 0; j < p.b_boxes; ++j)
-                tma_load_2d(sb + j * p.b_box_bytes, &map_b, full, tap * p.Cn + nt * p.bn + j * p.b_box_step,
+                load2<CTAS>(sb + j * p.b_box_bytes, &map_b, full, tap * p.Cn + nb + j * p.b_box_step,
                             cc * p.kdepth);
               break;
             }
@@ -250,9 +352,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               pixel_box(p, kb, kw0, kh0, kbb0);
               int r = tap_n / p.S, s = tap_n % p.S;
               for (int j = 0; j < p.a_boxes; ++j)
-                tma_load_4d(sa + j * p.a_box_bytes, &map_a, full, mt * BM + j * p.a_box_step, kw0, kh0, kbb0);
+                load4<CTAS>(sa + j * p.a_box_bytes, &map_a, full, mt * BM + j * p.a_box_step, kw0, kh0, kbb0);
               for (int j = 0; j < p.b_boxes; ++j)
-                tma_load_4d(sb + j * p.b_box_bytes, &map_b, full, ci0 + j * p.b_box_step, kw0 + s - p.pad,
+                load4<CTAS>(sb + j * p.b_box_bytes, &map_b, full, ci0 + j * p.b_box_step, kw0 + s - p.pad,
                             kh0 + r - p.pad, kbb0);
               break;
             }
@@ -262,13 +364,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    // ================= MMA issuer =================
-    if (lane == 0) {
+    // ================= MMA issuer (leader CTA only) =================
+    if (lane == 0 && rank == 0) {
       int stage = 0;
       unsigned phase = 0;
-      unsigned use = 0;                 // tiles processed by this CTA
+      unsigned use = 0;                 // tiles processed by this CTA (pair)
       bool ok = true;
-      for (long long item = blockIdx.x; ok && item < p.items; item += gridDim.x, ++use) {
+      for (long long item = first_item; ok && item < p.items; item += item_step, ++use) {
         const int split = (int)(item % p.splits);
         const int kb0 = split * p.kb_per_split;
         int kb1 = kb0 + p.kb_per_split;
@@ -286,14 +388,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           unsigned long long da = p.a_desc | (unsigned long long)((sa >> 4) & 0x3fff);
           unsigned long long db = p.b_desc | (unsigned long long)((sb >> 4) & 0x3fff);
           for (int k = 0; k < p.ksteps; ++k) {
-            tc_mma_i8(tmem_d, da, db, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+            const unsigned accum = (kb > kb0 || k > 0) ? 1u : 0u;
+            if (CTAS == 2) tc_mma_i8_pair(tmem_d, da, db, p.idesc, accum);
+            else tc_mma_i8(tmem_d, da, db, p.idesc, accum);
             da += p.a_kstep16;
             db += p.b_kstep16;
           }
-          tc_commit(empty0 + 8 * stage);        // frees the stage once these MMAs have read it
+          // frees the stage (in every CTA of the pair) once these MMAs have read it
+          if (CTAS == 2) tc_commit_pair(empty0 + 8 * stage); else tc_commit(empty0 + 8 * stage);
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
         }
-        if (ok) tc_commit(tfull0 + 8 * buf);    // accumulator complete
+        if (ok) {                               // accumulator complete
+          if (CTAS == 2) tc_commit_pair(tfull0 + 8 * buf); else tc_commit(tfull0 + 8 * buf);
+        }
       }
     }
   } else {
@@ -303,9 +410,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     unsigned use = 0;
     unsigned mx = 0;
     bool ok = true;
-    for (long long item = blockIdx.x; ok && item < p.items; item += gridDim.x, ++use) {
-      const long long tile = item / p.splits;
-      const int mt = (int)(tile / p.n_tiles_n), nt = (int)(tile % p.n_tiles_n);
+    for (long long item = first_item; ok && item < p.items; item += item_step, ++use) {
+      int mu, nt, split;
+      decode_item(p, item, mu, nt, split);
+      const int mt = mu * CTAS + (int)rank;
       const unsigned buf = use & 1u;
       // output row / column base of this thread
       long long out_row;
@@ -374,7 +482,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty0 + 8 * buf);
+      if (lane == 0) {
+        if (CTAS == 2 && rank != 0) mbar_arrive_cluster(lead_tempty0 + 8 * buf);
+        else mbar_arrive(tempty0 + 8 * buf);
+      }
     }
     if (!p.atomic_out) {
       for (int o = 16; o > 0; o >>= 1) {
@@ -395,9 +506,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     __syncthreads();
   }
+  if (CTAS == 2) cluster_sync_all();   // nobody leaves while the peer may still touch this CTA
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    if (CTAS == 2)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
   }
 }
 
@@ -474,8 +589,9 @@ static bool pick_pixel_box(int W, int H, int B, int &Wt, int &Ht, int &Bt) {
 static int round_up32(long long n) { return (int)((n + 31) / 32 * 32); }
 
 // Builds params and maps; returns false if the shape is not eligible for this engine.
-static bool plan(niti_ctx *ctx, const GemmProblem &g, TcParams &p, CUtensorMap &ma, CUtensorMap &mb) {
+static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, TcParams &p, CUtensorMap &ma, CUtensorMap &mb) {
   memset(&p, 0, sizeof(p));
+  p.ctas = ctas;
   p.kind = g.kind;
   p.gm = g.gm;
   p.gn = g.gn;
@@ -494,7 +610,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, TcParams &p, CUtensorMap &
       p.bn = g.gn >= 256 ? 256 : round_up32(g.gn);
       a_sw = b_sw = p.kdepth;
       sa = {2, {(cuuint64_t)g.gk, (cuuint64_t)g.gm}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, BM}, a_sw, g.p0};
-      sb = {2, {(cuuint64_t)g.gk, (cuuint64_t)g.gn}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, (cuuint32_t)p.bn}, b_sw, g.p1};
+      sb = {2, {(cuuint64_t)g.gk, (cuuint64_t)g.gn}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, (cuuint32_t)(p.bn / ctas)}, b_sw, g.p1};
       p.kb_total = (int)((g.gk + p.kdepth - 1) / p.kdepth);
       m_tiles = (g.gm + BM - 1) / BM;
       p.n_tiles_n = (int)((g.gn + p.bn - 1) / p.bn);
@@ -556,7 +672,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, TcParams &p, CUtensorMap &
       if (fwd) {
         p.bn = Cn >= 256 ? 256 : round_up32(Cn);
         b_sw = p.kdepth;
-        sb = {2, {(cuuint64_t)g.gk, (cuuint64_t)Cn}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, (cuuint32_t)p.bn}, b_sw, g.p1};
+        sb = {2, {(cuuint64_t)g.gk, (cuuint64_t)Cn}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, (cuuint32_t)(p.bn / ctas)}, b_sw, g.p1};
       } else {
         b_mn = 1;
         b_sw = pick_swizzle(Cn);
@@ -620,8 +736,11 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, TcParams &p, CUtensorMap &
     p.a_desc = desc_kmajor(a_sw);
     p.a_kstep16 = 2;
   }
+  const int bn_cta = p.bn / ctas;               // output columns staged by each CTA
+  if (bn_cta % 16) return false;
   if (b_mn) {
-    p.b_boxes = p.bn / b_sw;
+    if (bn_cta % b_sw) return false;
+    p.b_boxes = bn_cta / b_sw;
     p.b_box_bytes = p.kdepth * b_sw;
     p.b_box_step = b_sw;
     p.b_bytes = p.b_boxes * p.b_box_bytes;
@@ -629,7 +748,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, TcParams &p, CUtensorMap &
     p.b_kstep16 = (unsigned)((32 * b_sw) >> 4);
   } else {
     p.b_boxes = 1;
-    p.b_box_bytes = p.bn * p.kdepth;
+    p.b_box_bytes = bn_cta * p.kdepth;
     p.b_bytes = p.b_box_bytes;
     p.b_desc = desc_kmajor(b_sw);
     p.b_kstep16 = 2;
@@ -643,11 +762,16 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, TcParams &p, CUtensorMap &
   if (p.stages < 2) return false;
   // instruction descriptor: s32 accumulate, signed 8-bit operands, majorness, N, M
   p.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((unsigned)a_mn << 15) | ((unsigned)b_mn << 16) |
-            ((unsigned)(p.bn >> 3) << 17) | ((unsigned)(BM >> 4) << 24);
-  long long tiles = m_tiles * p.n_tiles_n;
+            ((unsigned)(p.bn >> 3) << 17) | ((unsigned)((BM * ctas) >> 4) << 24);
+  p.m_units = (int)((m_tiles + ctas - 1) / ctas);
+  long long tiles = (long long)p.m_units * p.n_tiles_n;
+  const int units = ctx->sm_count / ctas;       // CTAs (or CTA pairs) that run at the same time
+  // visit row units in groups so that concurrently running tiles share operands in L2
+  if ((g.kind == GK_FC_FWD || g.kind == GK_FC_DGRAD || g.kind == GK_FC_WGRAD) && p.n_tiles_n > 1 && p.m_units > 1)
+    p.raster_g = ctas == 2 ? 8 : 12;
   // split the contraction when the tiles alone cannot fill the SMs
-  if (tiles < ctx->sm_count && p.kb_total >= 8) {
-    long long s = (ctx->sm_count + tiles - 1) / tiles;
+  if (tiles < units && p.kb_total >= 8) {
+    long long s = (units + tiles - 1) / tiles;
     if (s > p.kb_total / 4) s = p.kb_total / 4;
     if (s < 1) s = 1;
     p.splits = (int)s;
@@ -666,25 +790,71 @@ int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long 
 
 size_t niti_tc_scratch_bytes(const GemmProblem &) { return 0; }
 
+template <int CTAS>
+static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CUtensorMap &ma, const CUtensorMap &mb,
+                     int32_t *acc, WsHeader *hdr) {
+  size_t smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + 1024;
+  static size_t attr_smem = 0;
+  if (smem > attr_smem) {
+    NITI_CUDA_TRY(ctx, cudaFuncSetAttribute(tc_gemm_kernel<CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_smem = smem;
+  }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)(ctx->sm_count / CTAS * CTAS), 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTAS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  // CTA pairs that can be resident at the same time (SMs pair up inside a GPC, so this can be
+  // fewer than sm_count / 2); a persistent grid larger than that would run a second, short wave
+  static int units_cached = 0;
+  if (!units_cached) {
+    units_cached = ctx->sm_count / CTAS;
+    if (CTAS == 2) {
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, tc_gemm_kernel<CTAS>, &cfg) == cudaSuccess && n > 0 && n < units_cached)
+        units_cached = n;
+      else
+        (void)cudaGetLastError();
+    }
+  }
+  const int units = units_cached;
+  long long grid = (p.items < units ? p.items : units) * CTAS;
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  NITI_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, tc_gemm_kernel<CTAS>, ma, mb, p, acc, hdr, ctx->d_status));
+  return NITI_OK;
+}
+
 int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, int32_t *acc, WsHeader *hdr, void *,
                  size_t) {
   TcParams p;
   CUtensorMap ma, mb;
-  if (!plan(ctx, g, p, ma, mb)) return NITI_ERR_SHAPE;
-  size_t smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + 1024;
-  static size_t attr_smem = 0;
-  if (smem > attr_smem) {
-    NITI_CUDA_TRY(ctx, cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_smem = smem;
+  // engine 0: pairs of CTAs (cta_group::2) when there are enough 256-row tiles to fill the GPU;
+  // engine 2 / 3 force the single-CTA / paired kernel (tests)
+  bool planned = false;
+  if (ctx->engine != 2 && g.gm >= 2 * BM) {
+    planned = plan(ctx, g, 2, p, ma, mb);
+    if (planned && ctx->engine != 3 && p.items < ctx->sm_count / 2) planned = false;
+  }
+  if (!planned) {
+    if (ctx->engine == 3) return NITI_ERR_SHAPE;
+    if (!plan(ctx, g, 1, p, ma, mb)) return NITI_ERR_SHAPE;
   }
   if (p.atomic_out) {
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(acc, 0, sizeof(int32_t) * (size_t)(g.gm * g.gn), st));
     ctx->launches++;
   }
-  long long grid = p.items < ctx->sm_count ? p.items : ctx->sm_count;
   const bool prof = ctx->profile_on && ctx->prof_ev && ctx->prof_used < NITI_PROF_MAX;
   if (prof) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st);
-  tc_gemm_kernel<<<(unsigned)grid, NUM_THREADS, smem, st>>>(ma, mb, p, acc, hdr, ctx->d_status);
+  int rc = p.ctas == 2 ? launch_tc<2>(ctx, st, p, ma, mb, acc, hdr) : launch_tc<1>(ctx, st, p, ma, mb, acc, hdr);
+  if (rc != NITI_OK) return rc;
   if (prof) {
     cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st);
     ctx->prof_ops[ctx->prof_used] = 2.0 * (double)g.gm * (double)g.gn * (double)g.gk;
@@ -692,7 +862,7 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, int32_t *
   }
   ctx->launches++;
   ctx->tc_launches++;
-  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  if (p.ctas == 2) ctx->tc2_launches++;
   if (p.atomic_out) return niti_launch_maxabs(ctx, st, acc, g.gm * g.gn, hdr);
   return NITI_OK;
 }

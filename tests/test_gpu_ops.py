@@ -37,7 +37,7 @@ FC_SHAPES = [(64, 256, 784), (64, 10, 256), (300, 520, 384), (128, 256, 128), (1
              (257, 300, 96), (1, 32, 32), (64, 1000, 512), (512, 384, 2048)]
 
 
-@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("engine", [0, 1, 2, 3])
 @pytest.mark.parametrize("M,N,K", FC_SHAPES)
 def test_linear_fwd(niti, oref, M, N, K, engine):
     rng = np.random.default_rng(M * 7 + N * 3 + K)
@@ -55,7 +55,7 @@ def test_linear_fwd(niti, oref, M, N, K, engine):
     niti.check()
 
 
-@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("engine", [0, 1, 2, 3])
 @pytest.mark.parametrize("M,N,K", FC_SHAPES[:7] + [(640, 256, 512)])
 def test_linear_bwd(niti, oref, M, N, K, engine):
     rng = np.random.default_rng(M * 5 + N * 11 + K)
@@ -86,7 +86,7 @@ CONV_SHAPES = [(2, 8, 8, 3, 16), (2, 16, 16, 64, 64), (4, 8, 8, 128, 256), (8, 4
                (1, 56, 56, 64, 128), (2, 12, 20, 96, 160)]
 
 
-@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("engine", [0, 1, 2, 3])
 @pytest.mark.parametrize("B,H,W,Ci,Co", CONV_SHAPES)
 def test_conv_ops(niti, oref, B, H, W, Ci, Co, engine):
     rng = np.random.default_rng(B + H * 3 + W * 5 + Ci * 7 + Co * 11)
