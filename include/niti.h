@@ -91,8 +91,10 @@ size_t niti_workspace_bytes(int op, const int64_t *dims, int ndims);
  * the shape allows; pairs of CTAs on 256-row tiles when there are enough of
  * them; default), 1 = plain CUDA-core kernels only, 2 = tensor cores with the
  * single-CTA kernel only, 3 = tensor cores with the paired-CTA kernel only
- * (falls back to CUDA cores where that kernel does not apply).  1-3 exist so
- * that tests can cross-check the engines.  Returns the previous value. */
+ * (falls back to CUDA cores where that kernel does not apply), 4 = tensor
+ * cores with the two-pass epilogue (int32 accumulators spilled to the
+ * workspace, rounded by a second kernel) instead of the fused one.  1-4 exist
+ * so that tests can cross-check the engines.  Returns the previous value. */
 int niti_set_engine(niti_ctx *ctx, int engine);
 
 /* Number of kernels / memsets this context has enqueued so far. */

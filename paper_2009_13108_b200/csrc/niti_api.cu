@@ -184,15 +184,14 @@ static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, 
     return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
   WsHeader *hdr = (WsHeader *)ws;
   int32_t *acc = (int32_t *)((char *)ws + NITI_WS_HEADER);
-  size_t acc_bytes = round_up((size_t)(p.gm * p.gn) * 4, 256);
-  void *scratch = (char *)ws + NITI_WS_HEADER + acc_bytes;
-  size_t scratch_bytes = ws_bytes - NITI_WS_HEADER - acc_bytes;
   NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, sizeof(WsHeader), st));
   ctx->launches++;
   int rc = NITI_ERR_SHAPE;
-  if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, acc, hdr, scratch, scratch_bytes);
+  bool fused = false;
+  RoundSpec rs = {out, mask, mbits, round_mode, relu, s_a, s_w, s_out, b_out};
+  if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, rs, acc, hdr, &fused);
   if (rc == NITI_ERR_SHAPE) rc = niti_simt_gemm(ctx, st, p, acc, hdr);
-  if (rc != NITI_OK) return rc;
+  if (rc != NITI_OK || fused) return rc;
   return niti_launch_round(ctx, st, acc, hdr, out, p.gm * p.gn, mbits, round_mode, relu, mask, s_a, s_w,
                            s_out, b_out);
 }

@@ -32,7 +32,7 @@ struct niti_ctx {
 // Scalars at the start of a workspace.
 struct WsHeader {
   unsigned int maxabs32;            // max |acc| of an int32 accumulator tensor
-  unsigned int pad0;
+  unsigned int est_max;             // max |acc| over the first tile of every CTA (speculative shift)
   unsigned long long maxabs64;      // same for the 64-bit loss accumulators
   unsigned int tile_counter;        // dynamic tile scheduler / arrival counter
   unsigned int pad1[3];
@@ -102,9 +102,19 @@ struct GemmProblem {
 
 // Plain CUDA-core engine: writes int32 accumulators to acc[gm][gn] and max|acc| to hdr->maxabs32.
 int niti_simt_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t *acc, WsHeader *hdr);
-// Tensor-core engine (tcgen05); returns NITI_ERR_SHAPE if the shape is not eligible.
-int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t *acc, WsHeader *hdr,
-                 void *scratch, size_t scratch_bytes);
+// What follows the multiply: rounding target and the scalars of Algorithm 2.
+struct RoundSpec {
+  int8_t *out;
+  const int8_t *mask;      // optional ReLU mask source (zero the output where mask <= 0)
+  int mbits, round_mode, relu;
+  const int32_t *s_a, *s_w;
+  int32_t *s_out, *b_out;
+};
+// Tensor-core engine (tcgen05); returns NITI_ERR_SHAPE if the shape is not eligible.  *fused is set
+// when the kernel also did the bit-width / shift / round / store (nothing is left to do); otherwise
+// acc holds the int32 accumulators and hdr->maxabs32 their max magnitude.
+int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, const RoundSpec &r, int32_t *acc,
+                 WsHeader *hdr, bool *fused);
 size_t niti_tc_scratch_bytes(const GemmProblem &p);
 
 // Epilogue pass: b from hdr->maxabs32, bp = max(0, b - mbits), out = Round(acc) with optional ReLU

@@ -33,7 +33,6 @@ struct TcParams {
   int kdepth;                   // contraction elements per k-block (32, 64 or 128)
   int ksteps;                   // kdepth / 32 MMAs per k-block
   int stages;
-  int atomic_out;               // 1: add into acc (split contraction), 0: store + max
   // shared-memory layout of one stage
   int a_bytes, b_bytes;         // bytes of the A and B parts of a stage
   int a_boxes, b_boxes;         // TMA copies per operand per stage
@@ -54,7 +53,24 @@ struct TcParams {
   int ctas;                     // CTAs per tile: 1, or 2 (cta_group::2, 256-row tiles)
   int m_units;                  // row units: 128-row tiles (ctas = 1) or 256-row pairs (ctas = 2)
   int raster_g;                 // row units per rasterisation group (0: row-major order)
+  // epilogue
+  int epi_mode;                 // EPI_SPILL / EPI_ATOMIC / EPI_SPECULATE / EPI_KNOWN_B
+  int mbits, round_mode, relu;
 };
+
+// Epilogue modes.  The shift of Algorithm 2 needs the bit-width of the WHOLE accumulator tensor:
+//  EPI_SPILL      store int32 accumulators + max; a second kernel rounds (always exact, 8 B / output
+//                 of extra traffic)
+//  EPI_ATOMIC     split contraction: add partial sums into a zeroed int32 tensor
+//  EPI_SPECULATE  every CTA computes its first tile, the grid agrees on the max over those tiles
+//                 (one bounded grid-wide wait), and all tiles are rounded and stored as int8 with the
+//                 shift that max implies, while the true max is tracked.  If the true bit-width turns
+//                 out larger, the EPI_KNOWN_B pass recomputes everything with it (exact in all cases;
+//                 the common case costs one multiply and no int32 traffic)
+//  EPI_KNOWN_B    bit-width known (hdr->maxabs32): round and store directly.  The kernel returns at
+//                 once when the speculative pass was right.
+enum { EPI_SPILL = 0, EPI_ATOMIC = 1, EPI_SPECULATE = 2, EPI_KNOWN_B = 3 };
+
 
 // ------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -232,7 +248,23 @@ __device__ __forceinline__ void decode_item(const TcParams &p, long long item, i
 template <int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const TcParams p, int32_t *__restrict__ acc, WsHeader *hdr, uint32_t *status) {
+               const TcParams p, int32_t *__restrict__ acc, WsHeader *hdr, uint32_t *status,
+               int8_t *__restrict__ out8, const int8_t *__restrict__ mask8, const int32_t *s_a,
+               const int32_t *s_w, int32_t *s_out, int32_t *b_out) {
+  if (p.epi_mode == EPI_KNOWN_B) {
+    // follow-up of a speculative pass: publish the scalars, then leave unless the guess was wrong
+    const int b_true = niti_bitlen32(hdr->maxabs32), b_est = niti_bitlen32(hdr->est_max);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      const int bp = b_true > p.mbits ? b_true - p.mbits : 0;
+      if (b_out) *b_out = b_true;
+      if (s_out) {
+        int s = bp + (s_a ? *s_a : 0) + (s_w ? *s_w : 0);
+        *s_out = s;
+        if (s < -128 || s > 127) atomicOr(status, NITI_DEV_EXP_RANGE);
+      }
+    }
+    if (b_true == b_est) return;
+  }
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 4];
   __shared__ unsigned tmem_base_slot;
@@ -409,6 +441,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int row_in_tile = quarter * 32 + lane;
     unsigned use = 0;
     unsigned mx = 0;
+    unsigned spec_max = 0;
+    int bp = 0;
+    if (p.epi_mode == EPI_KNOWN_B) {
+      const int b = niti_bitlen32(hdr->maxabs32);
+      bp = b > p.mbits ? b - p.mbits : 0;
+    }
     bool ok = true;
     for (long long item = first_item; ok && item < p.items; item += item_step, ++use) {
       int mu, nt, split;
@@ -447,34 +485,126 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       if (!mbar_wait(tfull0 + 8 * buf, (use >> 1) & 1u, &abort_flag, status)) { ok = false; break; }
       tc_fence_after();
-      int32_t *dst = acc + out_row * p.gn + col0;
-      const bool vec_ok = ((p.gn & 3) == 0) && ((col0 & 3) == 0);
-      for (int c = 0; c < p.bn; c += 32) {
-        int v[32];
-        tc_ld32(tmem_base + ((unsigned)(quarter * 32) << 16) + buf * (unsigned)p.bn + (unsigned)c, v);
-        if (row_ok && c < ncols_valid) {
-          if (p.atomic_out) {
+      const unsigned tm_row = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * (unsigned)p.bn;
+      if (p.epi_mode <= EPI_ATOMIC) {
+        int32_t *dst = acc + out_row * p.gn + col0;
+        const bool vec_ok = ((p.gn & 3) == 0) && ((col0 & 3) == 0);
+        for (int c = 0; c < p.bn; c += 32) {
+          int v[32];
+          tc_ld32(tm_row + (unsigned)c, v);
+          if (row_ok && c < ncols_valid) {
+            if (p.epi_mode == EPI_ATOMIC) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c + j < ncols_valid && v[j] != 0) atomicAdd(dst + c + j, v[j]);
-          } else {
+              for (int j = 0; j < 32; ++j)
+                if (c + j < ncols_valid && v[j] != 0) atomicAdd(dst + c + j, v[j]);
+            } else {
+              if (vec_ok && c + 32 <= ncols_valid) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                  *reinterpret_cast<int4 *>(dst + c + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  unsigned a = v[j] < 0 ? 0u - (unsigned)v[j] : (unsigned)v[j];
+                  mx = a > mx ? a : mx;
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (c + j < ncols_valid) {
+                    dst[c + j] = v[j];
+                    unsigned a = v[j] < 0 ? 0u - (unsigned)v[j] : (unsigned)v[j];
+                    mx = a > mx ? a : mx;
+                  }
+              }
+            }
+          }
+        }
+      } else {
+        if (p.epi_mode == EPI_SPECULATE && use == 0) {
+          // first tile of this CTA: max only, then agree on the estimate with the whole grid
+          unsigned m0 = 0;
+          for (int c = 0; c < p.bn; c += 32) {
+            int v[32];
+            tc_ld32(tm_row + (unsigned)c, v);
+            if (row_ok) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (c + j < ncols_valid) {
+                  unsigned a = v[j] < 0 ? 0u - (unsigned)v[j] : (unsigned)v[j];
+                  m0 = a > m0 ? a : m0;
+                }
+            }
+          }
+          for (int o = 16; o > 0; o >>= 1) {
+            unsigned u = __shfl_xor_sync(0xffffffffu, m0, o);
+            m0 = u > m0 ? u : m0;
+          }
+          if (lane == 0) {
+            if (m0) atomicMax(&hdr->est_max, m0);
+            __threadfence();
+            atomicAdd(&hdr->tile_counter, 1u);
+            const unsigned expected = gridDim.x * 4u;      // four epilogue warps per CTA
+            long long t0 = clock64();
+            while (*(volatile unsigned *)&hdr->tile_counter < expected) {
+              if (abort_flag) break;
+              if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                abort_flag = 1;
+                atomicOr(status, NITI_DEV_TIMEOUT);
+                break;
+              }
+            }
+            __threadfence();
+          }
+          __syncwarp();
+          if (abort_flag) { ok = false; break; }
+          if (lane == 0) spec_max = *(volatile unsigned *)&hdr->est_max;
+          spec_max = __shfl_sync(0xffffffffu, spec_max, 0);
+          const int b = niti_bitlen32(spec_max);
+          bp = b > p.mbits ? b - p.mbits : 0;
+        }
+        int8_t *dst8 = out8 + out_row * p.gn + col0;
+        const int8_t *msk = mask8 ? mask8 + out_row * p.gn + col0 : nullptr;
+        const bool vec_ok = ((p.gn & 15) == 0) && ((col0 & 15) == 0);
+        const unsigned qmax = (1u << p.mbits) - 1u;
+        for (int c = 0; c < p.bn; c += 32) {
+          int v[32];
+          tc_ld32(tm_row + (unsigned)c, v);
+          if (row_ok && c < ncols_valid) {
+            unsigned w8[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              unsigned word = 0;
+#pragma unroll
+              for (int t = 0; t < 4; ++t) {
+                const int x = v[4 * j + t];
+                unsigned a = x < 0 ? 0u - (unsigned)x : (unsigned)x;
+                if (c + 4 * j + t < ncols_valid) mx = a > mx ? a : mx;
+                int q = (int)niti_round_mag<unsigned>(a, bp, qmax, p.round_mode);
+                q = x < 0 ? -q : q;
+                if (p.relu && q < 0) q = 0;
+                word |= (unsigned)(q & 0xff) << (8 * t);
+              }
+              w8[j] = word;
+            }
             if (vec_ok && c + 32 <= ncols_valid) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                *reinterpret_cast<int4 *>(dst + c + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+              if (msk) {
+                const int4 m0v = *reinterpret_cast<const int4 *>(msk + c);
+                const int4 m1v = *reinterpret_cast<const int4 *>(msk + c + 16);
+                w8[0] &= __vcmpgts4(m0v.x, 0); w8[1] &= __vcmpgts4(m0v.y, 0);
+                w8[2] &= __vcmpgts4(m0v.z, 0); w8[3] &= __vcmpgts4(m0v.w, 0);
+                w8[4] &= __vcmpgts4(m1v.x, 0); w8[5] &= __vcmpgts4(m1v.y, 0);
+                w8[6] &= __vcmpgts4(m1v.z, 0); w8[7] &= __vcmpgts4(m1v.w, 0);
               }
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                unsigned a = v[j] < 0 ? 0u - (unsigned)v[j] : (unsigned)v[j];
-                mx = a > mx ? a : mx;
-              }
+              *reinterpret_cast<int4 *>(dst8 + c) = make_int4(w8[0], w8[1], w8[2], w8[3]);
+              *reinterpret_cast<int4 *>(dst8 + c + 16) = make_int4(w8[4], w8[5], w8[6], w8[7]);
             } else {
 #pragma unroll
               for (int j = 0; j < 32; ++j)
                 if (c + j < ncols_valid) {
-                  dst[c + j] = v[j];
-                  unsigned a = v[j] < 0 ? 0u - (unsigned)v[j] : (unsigned)v[j];
-                  mx = a > mx ? a : mx;
+                  int8_t q = (int8_t)((w8[j >> 2] >> (8 * (j & 3))) & 0xff);
+                  if (msk && msk[c + j] <= 0) q = 0;
+                  dst8[c + j] = q;
                 }
             }
           }
@@ -487,7 +617,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         else mbar_arrive(tempty0 + 8 * buf);
       }
     }
-    if (!p.atomic_out) {
+    if (p.epi_mode == EPI_SPILL || p.epi_mode == EPI_SPECULATE) {
       for (int o = 16; o > 0; o >>= 1) {
         unsigned u = __shfl_xor_sync(0xffffffffu, mx, o);
         mx = u > mx ? u : mx;
@@ -778,7 +908,6 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, TcParams &p, CUt
   }
   p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
   p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
-  p.atomic_out = p.splits > 1;
   p.items = tiles * p.splits;
   if (!encode(ctx, &ma, sa) || !encode(ctx, &mb, sb)) return false;
   return true;
@@ -792,7 +921,7 @@ size_t niti_tc_scratch_bytes(const GemmProblem &) { return 0; }
 
 template <int CTAS>
 static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CUtensorMap &ma, const CUtensorMap &mb,
-                     int32_t *acc, WsHeader *hdr) {
+                     int32_t *acc, WsHeader *hdr, const RoundSpec &r) {
   size_t smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + 1024;
   static size_t attr_smem = 0;
   if (smem > attr_smem) {
@@ -828,16 +957,21 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
   const int units = units_cached;
   long long grid = (p.items < units ? p.items : units) * CTAS;
   cfg.gridDim = dim3((unsigned)grid, 1, 1);
-  NITI_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, tc_gemm_kernel<CTAS>, ma, mb, p, acc, hdr, ctx->d_status));
+  NITI_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, tc_gemm_kernel<CTAS>, ma, mb, p, acc, hdr, ctx->d_status, r.out, r.mask,
+                                        r.s_a, r.s_w, r.s_out, r.b_out));
+  ctx->launches++;
+  ctx->tc_launches++;
+  if (CTAS == 2) ctx->tc2_launches++;
   return NITI_OK;
 }
 
-int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, int32_t *acc, WsHeader *hdr, void *,
-                 size_t) {
+int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const RoundSpec &r, int32_t *acc,
+                 WsHeader *hdr, bool *fused) {
   TcParams p;
   CUtensorMap ma, mb;
-  // engine 0: pairs of CTAs (cta_group::2) when there are enough 256-row tiles to fill the GPU;
-  // engine 2 / 3 force the single-CTA / paired kernel (tests)
+  *fused = false;
+  // engine 0: pairs of CTAs (cta_group::2) when there are enough 256-row tiles to fill the GPU.
+  // Test switches: 2 / 3 force the single-CTA / paired kernel, 4 keeps the int32 spill epilogue.
   bool planned = false;
   if (ctx->engine != 2 && g.gm >= 2 * BM) {
     planned = plan(ctx, g, 2, p, ma, mb);
@@ -847,22 +981,30 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, int32_t *
     if (ctx->engine == 3) return NITI_ERR_SHAPE;
     if (!plan(ctx, g, 1, p, ma, mb)) return NITI_ERR_SHAPE;
   }
-  if (p.atomic_out) {
+  p.mbits = r.mbits;
+  p.round_mode = r.round_mode;
+  p.relu = r.relu;
+  p.epi_mode = p.splits > 1 ? EPI_ATOMIC : (ctx->engine == 4 ? EPI_SPILL : EPI_SPECULATE);
+  if (p.epi_mode == EPI_ATOMIC) {
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(acc, 0, sizeof(int32_t) * (size_t)(g.gm * g.gn), st));
     ctx->launches++;
   }
   const bool prof = ctx->profile_on && ctx->prof_ev && ctx->prof_used < NITI_PROF_MAX;
   if (prof) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st);
-  int rc = p.ctas == 2 ? launch_tc<2>(ctx, st, p, ma, mb, acc, hdr) : launch_tc<1>(ctx, st, p, ma, mb, acc, hdr);
+  int rc = p.ctas == 2 ? launch_tc<2>(ctx, st, p, ma, mb, acc, hdr, r) : launch_tc<1>(ctx, st, p, ma, mb, acc, hdr, r);
   if (rc != NITI_OK) return rc;
+  if (p.epi_mode == EPI_SPECULATE) {
+    // publishes b and the exponent; recomputes with the true bit-width only if the guess was low
+    p.epi_mode = EPI_KNOWN_B;
+    rc = p.ctas == 2 ? launch_tc<2>(ctx, st, p, ma, mb, acc, hdr, r) : launch_tc<1>(ctx, st, p, ma, mb, acc, hdr, r);
+    if (rc != NITI_OK) return rc;
+    *fused = true;
+  }
   if (prof) {
     cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st);
     ctx->prof_ops[ctx->prof_used] = 2.0 * (double)g.gm * (double)g.gn * (double)g.gk;
     ctx->prof_used++;
   }
-  ctx->launches++;
-  ctx->tc_launches++;
-  if (p.ctas == 2) ctx->tc2_launches++;
-  if (p.atomic_out) return niti_launch_maxabs(ctx, st, acc, g.gm * g.gn, hdr);
+  if (p.epi_mode == EPI_ATOMIC) return niti_launch_maxabs(ctx, st, acc, g.gm * g.gn, hdr);
   return NITI_OK;
 }

@@ -37,7 +37,7 @@ FC_SHAPES = [(64, 256, 784), (64, 10, 256), (300, 520, 384), (128, 256, 128), (1
              (257, 300, 96), (1, 32, 32), (64, 1000, 512), (512, 384, 2048)]
 
 
-@pytest.mark.parametrize("engine", [0, 1, 2, 3])
+@pytest.mark.parametrize("engine", [0, 1, 2, 3, 4])
 @pytest.mark.parametrize("M,N,K", FC_SHAPES)
 def test_linear_fwd(niti, oref, M, N, K, engine):
     rng = np.random.default_rng(M * 7 + N * 3 + K)
@@ -55,7 +55,7 @@ def test_linear_fwd(niti, oref, M, N, K, engine):
     niti.check()
 
 
-@pytest.mark.parametrize("engine", [0, 1, 2, 3])
+@pytest.mark.parametrize("engine", [0, 1, 2, 3, 4])
 @pytest.mark.parametrize("M,N,K", FC_SHAPES[:7] + [(640, 256, 512)])
 def test_linear_bwd(niti, oref, M, N, K, engine):
     rng = np.random.default_rng(M * 5 + N * 11 + K)
@@ -86,7 +86,7 @@ CONV_SHAPES = [(2, 8, 8, 3, 16), (2, 16, 16, 64, 64), (4, 8, 8, 128, 256), (8, 4
                (1, 56, 56, 64, 128), (2, 12, 20, 96, 160)]
 
 
-@pytest.mark.parametrize("engine", [0, 1, 2, 3])
+@pytest.mark.parametrize("engine", [0, 1, 2, 3, 4])
 @pytest.mark.parametrize("B,H,W,Ci,Co", CONV_SHAPES)
 def test_conv_ops(niti, oref, B, H, W, Ci, Co, engine):
     rng = np.random.default_rng(B + H * 3 + W * 5 + Ci * 7 + Co * 11)
@@ -123,7 +123,37 @@ def test_tensor_core_engine_is_the_one_that_runs(niti):
     niti.conv_dgrad(e, wc, (16, 16))
     niti.conv_wgrad(x, e)
     niti.linear_bwd(a, _T(niti, _i8(rng, (256, 256))), w)
-    assert niti.tc_launch_count() - before == 6
+    assert niti.tc_launch_count() - before >= 6
+    niti.check()
+
+
+@pytest.mark.parametrize("engine", [0, 2, 3])
+def test_speculative_shift_is_corrected(niti, oref, engine):
+    """The fused epilogue rounds with the bit-width of the first tile of every CTA and redoes the
+    multiply when the whole tensor needs a larger shift: here only the last rows are large."""
+    rng = np.random.default_rng(77)
+    M, N, K = 128 * 400, 64, 128
+    a = rng.integers(-3, 4, size=(M, K), dtype=np.int8)
+    a[-5:] = rng.integers(100, 128, size=(5, K), dtype=np.int8)
+    w = rng.integers(64, 128, size=(N, K), dtype=np.int8)
+    want, s, b = oref.linear_fwd(a, -7, w, -10, True)
+    niti.set_engine(engine)
+    try:
+        out, s_out, b_out = niti.linear_fwd(_T(niti, a), niti.scalar(-7), _T(niti, w),
+                                            niti.scalar(-10), relu=True)
+        _eq(out, want)
+        assert (int(s_out), int(b_out)) == (s, b)
+        # and the mirrored case through the masked dgrad epilogue
+        e = rng.integers(-2, 3, size=(M, N), dtype=np.int8)
+        e[-3:] = 127
+        mask = rng.integers(-5, 6, size=(M, K), dtype=np.int8)
+        we, wg, be, bg = oref.linear_bwd(a, e, w, True, mask, 5)
+        ep, g, b_e, b_g = niti.linear_bwd(_T(niti, a), _T(niti, e), _T(niti, w), True, _T(niti, mask))
+        _eq(ep, we)
+        _eq(g, wg)
+        assert (int(b_e), int(b_g)) == (be, bg)
+    finally:
+        niti.set_engine(0)
     niti.check()
 
 
