@@ -104,6 +104,12 @@ uint64_t niti_tc_launch_count(niti_ctx *ctx);
 /* Of those, launches of the paired-CTA (cta_group::2) variant. */
 uint64_t niti_tc_pair_launch_count(niti_ctx *ctx);
 
+/* The fused epilogue of the tensor-core kernel rounds with a bit-width guessed from the first
+ * tile of every CTA and recomputes the multiply when the whole tensor turns out to need a larger
+ * shift (results are exact either way).  Returns how many such recomputations this context has
+ * run so far (synchronises `stream`; -1 on error). */
+int64_t niti_redo_count(niti_ctx *ctx, void *stream);
+
 /* Timing of the tensor-core matrix-multiply kernel.  While enabled, every launch of that
  * kernel is bracketed by a pair of CUDA events on its stream (up to 8192 launches are kept).
  * niti_profile_read() waits for the recorded events, returns their summed duration in

@@ -20,7 +20,7 @@ OP_LINEAR_FWD, OP_LINEAR_BWD, OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_INT_
 EXPORTS = [
     "niti_create", "niti_destroy", "niti_last_error", "niti_check", "niti_workspace_bytes",
     "niti_set_engine", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
-    "niti_profile_enable",
+    "niti_redo_count", "niti_profile_enable",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
     "niti_conv_dgrad", "niti_conv_wgrad", "niti_int_xent", "niti_int_sgd_update", "niti_relu_fwd",
     "niti_relu_bwd", "niti_maxpool2_fwd", "niti_maxpool2_bwd",
@@ -57,6 +57,8 @@ def load_library():
     lib.niti_tc_launch_count.restype = C.c_uint64
     lib.niti_tc_pair_launch_count.argtypes = [vp]
     lib.niti_tc_pair_launch_count.restype = C.c_uint64
+    lib.niti_redo_count.argtypes = [vp, vp]
+    lib.niti_redo_count.restype = C.c_int64
     lib.niti_profile_enable.argtypes = [vp, i32]
     lib.niti_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64),
                                       C.POINTER(C.c_double)]
@@ -142,6 +144,9 @@ class Niti:
 
     def tc_pair_launch_count(self) -> int:
         return int(self.lib.niti_tc_pair_launch_count(self.h))
+
+    def redo_count(self) -> int:
+        return int(self.lib.niti_redo_count(self.h, self._stream()))
 
     def profile_enable(self, on: bool):
         self._ck(self.lib.niti_profile_enable(self.h, int(on)))

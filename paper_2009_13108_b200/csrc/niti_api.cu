@@ -62,6 +62,14 @@ extern "C" uint64_t niti_launch_count(niti_ctx *ctx) { return ctx ? ctx->launche
 extern "C" uint64_t niti_tc_launch_count(niti_ctx *ctx) { return ctx ? ctx->tc_launches : 0; }
 extern "C" uint64_t niti_tc_pair_launch_count(niti_ctx *ctx) { return ctx ? ctx->tc2_launches : 0; }
 
+extern "C" int64_t niti_redo_count(niti_ctx *ctx, void *stream) {
+  if (!ctx) return -1;
+  uint32_t h = 0;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return -1;
+  if (cudaMemcpy(&h, ctx->d_status + 1, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  return (int64_t)h;
+}
+
 extern "C" int niti_profile_enable(niti_ctx *ctx, int on) {
   if (!ctx) return NITI_ERR_ARG;
   if (on && !ctx->prof_ev) {

@@ -31,7 +31,7 @@ struct niti_ctx {
 
 // Scalars at the start of a workspace.
 struct WsHeader {
-  unsigned int maxabs32;            // max |acc| of an int32 accumulator tensor
+  unsigned int maxabs32;            // a value with the bit length of max |acc| (a max, or an OR of magnitudes)
   unsigned int est_max;             // max |acc| over the first tile of every CTA (speculative shift)
   unsigned long long maxabs64;      // same for the 64-bit loss accumulators
   unsigned int tile_counter;        // dynamic tile scheduler / arrival counter

@@ -17,7 +17,8 @@
 namespace {
 
 constexpr int BM = 128;               // rows of an output tile = TMEM lanes
-constexpr int NUM_THREADS = 192;
+constexpr int EPI_WARPS = 8;           // two per TMEM lane quarter, alternating 32-column chunks
+constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int MAX_STAGES = 8;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;
 
@@ -155,6 +156,58 @@ __device__ __forceinline__ void tc_ld32(unsigned taddr, int (&v)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// The same load without the wait, and a wait that names the registers so that no use of them can be
+// scheduled before it.
+__device__ __forceinline__ void tc_ld32_issue(unsigned taddr, int (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld_wait(int (&v)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                 "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
+                 "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
+                 "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+               :
+               : "memory");
+}
+
+// Shift-and-round of four accumulators (Algorithm 2 + 3, or round-to-nearest) packed into four int8.
+// The discarded fraction has bp bits; with an odd bp its lowest bit is dropped; top and bottom
+// halves are h = bp / 2 bits wide: top = bits [odd + h, odd + 2h), bottom = bits [odd, odd + h).
+// `orv` collects the OR of the magnitudes: its bit length equals that of the maximum.
+template <int ROUND_MODE>
+__device__ __forceinline__ unsigned round_pack4(int x0, int x1, int x2, int x3, int bp, int sh_top, int sh_bot,
+                                                unsigned hmask, unsigned qmax, int relu, unsigned &orv) {
+  const unsigned a0 = (unsigned)abs(x0), a1 = (unsigned)abs(x1), a2 = (unsigned)abs(x2), a3 = (unsigned)abs(x3);
+  orv |= a0 | a1;
+  orv |= a2 | a3;
+  unsigned q0 = a0 >> bp, q1 = a1 >> bp, q2 = a2 >> bp, q3 = a3 >> bp;
+  if (ROUND_MODE == NITI_ROUND_PSR) {
+    q0 += ((a0 >> sh_top) & hmask) > ((a0 >> sh_bot) & hmask);
+    q1 += ((a1 >> sh_top) & hmask) > ((a1 >> sh_bot) & hmask);
+    q2 += ((a2 >> sh_top) & hmask) > ((a2 >> sh_bot) & hmask);
+    q3 += ((a3 >> sh_top) & hmask) > ((a3 >> sh_bot) & hmask);
+  } else {
+    // sh_top = bp - 1, hmask = (bp > 0): the highest discarded bit
+    q0 += (a0 >> sh_top) & hmask; q1 += (a1 >> sh_top) & hmask;
+    q2 += (a2 >> sh_top) & hmask; q3 += (a3 >> sh_top) & hmask;
+  }
+  q0 = min(q0, qmax); q1 = min(q1, qmax); q2 = min(q2, qmax); q3 = min(q3, qmax);
+  const unsigned mag = __byte_perm(__byte_perm(q0, q1, 0x4040), __byte_perm(q2, q3, 0x4040), 0x5410);
+  const unsigned sgn = __byte_perm(__byte_perm((unsigned)(x0 >> 31), (unsigned)(x1 >> 31), 0x4040),
+                                   __byte_perm((unsigned)(x2 >> 31), (unsigned)(x3 >> 31), 0x4040), 0x5410);
+  return relu ? (mag & ~sgn) : __vsub4(mag ^ sgn, sgn);
+}
+
 // Coordinates of an output tile / k-block in the pixel grid of a convolution.
 __device__ __forceinline__ void pixel_box(const TcParams &p, int idx, int &w0, int &h0, int &b0) {
   int wt = idx % p.w_tiles;
@@ -264,6 +317,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
     if (b_true == b_est) return;
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(status + 1, 1u);   // count of recomputations
   }
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 4];
@@ -296,7 +350,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull0 + 8 * b, 1);
-      mbar_init(tempty0 + 8 * b, 4 * CTAS);     // one arrival per epilogue warp of every CTA
+      mbar_init(tempty0 + 8 * b, EPI_WARPS * CTAS);     // one arrival per epilogue warp of every CTA
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -438,6 +492,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else {
     // ================= epilogue: TMEM -> int32 accumulators + max magnitude =================
     const int quarter = warp & 3;               // TMEM lanes [32 * quarter, +32)
+    const int chunk_phase = (warp - 2) >> 2;    // this warp takes 32-column chunks phase, phase + 2, ...
     const int row_in_tile = quarter * 32 + lane;
     unsigned use = 0;
     unsigned mx = 0;
@@ -489,7 +544,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (p.epi_mode <= EPI_ATOMIC) {
         int32_t *dst = acc + out_row * p.gn + col0;
         const bool vec_ok = ((p.gn & 3) == 0) && ((col0 & 3) == 0);
-        for (int c = 0; c < p.bn; c += 32) {
+        for (int c = 32 * chunk_phase; c < p.bn; c += 64) {
           int v[32];
           tc_ld32(tm_row + (unsigned)c, v);
           if (row_ok && c < ncols_valid) {
@@ -524,7 +579,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (p.epi_mode == EPI_SPECULATE && use == 0) {
           // first tile of this CTA: max only, then agree on the estimate with the whole grid
           unsigned m0 = 0;
-          for (int c = 0; c < p.bn; c += 32) {
+          for (int c = 32 * chunk_phase; c < p.bn; c += 64) {
             int v[32];
             tc_ld32(tm_row + (unsigned)c, v);
             if (row_ok) {
@@ -544,7 +599,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (m0) atomicMax(&hdr->est_max, m0);
             __threadfence();
             atomicAdd(&hdr->tile_counter, 1u);
-            const unsigned expected = gridDim.x * 4u;      // four epilogue warps per CTA
+            const unsigned expected = gridDim.x * (unsigned)EPI_WARPS;
             long long t0 = clock64();
             while (*(volatile unsigned *)&hdr->tile_counter < expected) {
               if (abort_flag) break;
@@ -567,27 +622,36 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int8_t *msk = mask8 ? mask8 + out_row * p.gn + col0 : nullptr;
         const bool vec_ok = ((p.gn & 15) == 0) && ((col0 & 15) == 0);
         const unsigned qmax = (1u << p.mbits) - 1u;
-        for (int c = 0; c < p.bn; c += 32) {
-          int v[32];
-          tc_ld32(tm_row + (unsigned)c, v);
+        // constants of the rounding rule for this binary point
+        const int odd = bp & 1, h = bp >> 1;
+        int sh_top, sh_bot;
+        unsigned hmask;
+        if (p.round_mode == NITI_ROUND_PSR) { sh_top = odd + h; sh_bot = odd; hmask = (1u << h) - 1u; }
+        else { sh_top = bp > 0 ? bp - 1 : 0; sh_bot = 0; hmask = bp > 0 ? 1u : 0u; }
+        int va[32], vb[32];
+        int c = 32 * chunk_phase;
+        if (c < p.bn) tc_ld32_issue(tm_row + (unsigned)c, va);
+        for (int it = 0; c < p.bn; c += 64, ++it) {
+          int (&v)[32] = (it & 1) ? vb : va;
+          int (&vn)[32] = (it & 1) ? va : vb;
+          tc_ld_wait(v);
+          if (c + 64 < p.bn) tc_ld32_issue(tm_row + (unsigned)(c + 64), vn);   // overlaps the math below
           if (row_ok && c < ncols_valid) {
             unsigned w8[8];
+            unsigned orv = 0;
+            if (p.round_mode == NITI_ROUND_PSR) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              unsigned word = 0;
+              for (int j = 0; j < 8; ++j)
+                w8[j] = round_pack4<NITI_ROUND_PSR>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], bp, sh_top,
+                                                    sh_bot, hmask, qmax, p.relu, orv);
+            } else {
 #pragma unroll
-              for (int t = 0; t < 4; ++t) {
-                const int x = v[4 * j + t];
-                unsigned a = x < 0 ? 0u - (unsigned)x : (unsigned)x;
-                if (c + 4 * j + t < ncols_valid) mx = a > mx ? a : mx;
-                int q = (int)niti_round_mag<unsigned>(a, bp, qmax, p.round_mode);
-                q = x < 0 ? -q : q;
-                if (p.relu && q < 0) q = 0;
-                word |= (unsigned)(q & 0xff) << (8 * t);
-              }
-              w8[j] = word;
+              for (int j = 0; j < 8; ++j)
+                w8[j] = round_pack4<NITI_ROUND_NEAREST>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], bp,
+                                                        sh_top, sh_bot, hmask, qmax, p.relu, orv);
             }
             if (vec_ok && c + 32 <= ncols_valid) {
+              mx |= orv;
               if (msk) {
                 const int4 m0v = *reinterpret_cast<const int4 *>(msk + c);
                 const int4 m1v = *reinterpret_cast<const int4 *>(msk + c + 16);
@@ -602,6 +666,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
               for (int j = 0; j < 32; ++j)
                 if (c + j < ncols_valid) {
+                  mx |= (unsigned)abs(v[j]);
                   int8_t q = (int8_t)((w8[j >> 2] >> (8 * (j & 3))) & 0xff);
                   if (msk && msk[c + j] <= 0) q = 0;
                   dst8[c + j] = q;
