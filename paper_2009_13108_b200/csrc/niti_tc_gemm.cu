@@ -17,7 +17,8 @@
 namespace {
 
 constexpr int BM = 128;               // rows of an output tile = TMEM lanes
-constexpr int EPI_WARPS = 8;           // two per TMEM lane quarter, alternating 32-column chunks
+constexpr int EPI_WARPS = 16;          // four per TMEM lane quarter, interleaved 32-column chunks
+constexpr int EPI_PER_Q = EPI_WARPS / 4;
 constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int MAX_STAGES = 8;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;
@@ -181,31 +182,58 @@ __device__ __forceinline__ void tc_ld_wait(int (&v)[32]) {
 }
 
 // Shift-and-round of four accumulators (Algorithm 2 + 3, or round-to-nearest) packed into four int8.
-// The discarded fraction has bp bits; with an odd bp its lowest bit is dropped; top and bottom
-// halves are h = bp / 2 bits wide: top = bits [odd + h, odd + 2h), bottom = bits [odd, odd + h).
-// `orv` collects the OR of the magnitudes: its bit length equals that of the maximum.
-template <int ROUND_MODE>
-__device__ __forceinline__ unsigned round_pack4(int x0, int x1, int x2, int x3, int bp, int sh_top, int sh_bot,
-                                                unsigned hmask, unsigned qmax, int relu, unsigned &orv) {
+//
+// Pseudo-stochastic rule on a magnitude a with bp discarded bits (h = bp / 2, odd = bp & 1):
+// y = a >> odd drops the lowest bit when bp is odd; its low 2h bits are top * 2^h + bot, and the
+// integer part is incremented iff top > bot.  Adding C - bot * 2^h with C = 2^(2h) - 2^h carries
+// into bit 2h exactly in that case:  q = (y + C - (y & (2^h - 1)) * 2^h) >> 2h.
+// Round-to-nearest is the same expression with odd = 0, mask = 0, C = 2^(bp-1) (0 if bp = 0) and
+// a final shift by bp.  `orv` collects the OR of the magnitudes (same bit length as their maximum).
+struct RoundConst {
+  int odd;        // pre-shift
+  unsigned mask;  // 2^h - 1
+  unsigned negp;  // -(2^h) as an unsigned multiplier
+  unsigned c;     // additive constant
+  int shift;      // final shift
+  unsigned qmax;  // saturation 2^mbits - 1
+};
+__device__ __forceinline__ RoundConst make_round_const(int bp, int mbits, int round_mode) {
+  RoundConst k;
+  k.qmax = (1u << mbits) - 1u;
+  if (round_mode == NITI_ROUND_PSR) {
+    const int h = bp >> 1;
+    k.odd = bp & 1;
+    k.mask = (1u << h) - 1u;
+    k.negp = 0u - (1u << h);
+    k.c = (1u << (2 * h)) - (1u << h);
+    k.shift = 2 * h;
+  } else {
+    k.odd = 0;
+    k.mask = 0;
+    k.negp = 0;
+    k.c = bp > 0 ? 1u << (bp - 1) : 0u;
+    k.shift = bp;
+  }
+  return k;
+}
+__device__ __forceinline__ unsigned round_mag1(unsigned a, const RoundConst &k) {
+  const unsigned y = a >> k.odd;
+  const unsigned q = ((y & k.mask) * k.negp + (y + k.c)) >> k.shift;
+  return min(q, k.qmax);
+}
+template <bool RELU>
+__device__ __forceinline__ unsigned round_pack4(int x0, int x1, int x2, int x3, const RoundConst &k, unsigned &orv) {
   const unsigned a0 = (unsigned)abs(x0), a1 = (unsigned)abs(x1), a2 = (unsigned)abs(x2), a3 = (unsigned)abs(x3);
   orv |= a0 | a1;
   orv |= a2 | a3;
-  unsigned q0 = a0 >> bp, q1 = a1 >> bp, q2 = a2 >> bp, q3 = a3 >> bp;
-  if (ROUND_MODE == NITI_ROUND_PSR) {
-    q0 += ((a0 >> sh_top) & hmask) > ((a0 >> sh_bot) & hmask);
-    q1 += ((a1 >> sh_top) & hmask) > ((a1 >> sh_bot) & hmask);
-    q2 += ((a2 >> sh_top) & hmask) > ((a2 >> sh_bot) & hmask);
-    q3 += ((a3 >> sh_top) & hmask) > ((a3 >> sh_bot) & hmask);
+  unsigned q0 = round_mag1(a0, k), q1 = round_mag1(a1, k), q2 = round_mag1(a2, k), q3 = round_mag1(a3, k);
+  const unsigned s0 = (unsigned)(x0 >> 31), s1 = (unsigned)(x1 >> 31), s2 = (unsigned)(x2 >> 31), s3 = (unsigned)(x3 >> 31);
+  if (RELU) {
+    q0 &= ~s0; q1 &= ~s1; q2 &= ~s2; q3 &= ~s3;
   } else {
-    // sh_top = bp - 1, hmask = (bp > 0): the highest discarded bit
-    q0 += (a0 >> sh_top) & hmask; q1 += (a1 >> sh_top) & hmask;
-    q2 += (a2 >> sh_top) & hmask; q3 += (a3 >> sh_top) & hmask;
+    q0 = (q0 ^ s0) - s0; q1 = (q1 ^ s1) - s1; q2 = (q2 ^ s2) - s2; q3 = (q3 ^ s3) - s3;
   }
-  q0 = min(q0, qmax); q1 = min(q1, qmax); q2 = min(q2, qmax); q3 = min(q3, qmax);
-  const unsigned mag = __byte_perm(__byte_perm(q0, q1, 0x4040), __byte_perm(q2, q3, 0x4040), 0x5410);
-  const unsigned sgn = __byte_perm(__byte_perm((unsigned)(x0 >> 31), (unsigned)(x1 >> 31), 0x4040),
-                                   __byte_perm((unsigned)(x2 >> 31), (unsigned)(x3 >> 31), 0x4040), 0x5410);
-  return relu ? (mag & ~sgn) : __vsub4(mag ^ sgn, sgn);
+  return __byte_perm(__byte_perm(q0, q1, 0x4040), __byte_perm(q2, q3, 0x4040), 0x5410);
 }
 
 // Coordinates of an output tile / k-block in the pixel grid of a convolution.
@@ -492,7 +520,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else {
     // ================= epilogue: TMEM -> int32 accumulators + max magnitude =================
     const int quarter = warp & 3;               // TMEM lanes [32 * quarter, +32)
-    const int chunk_phase = (warp - 2) >> 2;    // this warp takes 32-column chunks phase, phase + 2, ...
+    const int chunk_phase = (warp - 2) >> 2;    // this warp takes 32-column chunks phase, phase + EPI_PER_Q, ...
     const int row_in_tile = quarter * 32 + lane;
     unsigned use = 0;
     unsigned mx = 0;
@@ -544,7 +572,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (p.epi_mode <= EPI_ATOMIC) {
         int32_t *dst = acc + out_row * p.gn + col0;
         const bool vec_ok = ((p.gn & 3) == 0) && ((col0 & 3) == 0);
-        for (int c = 32 * chunk_phase; c < p.bn; c += 64) {
+        for (int c = 32 * chunk_phase; c < p.bn; c += 32 * EPI_PER_Q) {
           int v[32];
           tc_ld32(tm_row + (unsigned)c, v);
           if (row_ok && c < ncols_valid) {
@@ -579,7 +607,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (p.epi_mode == EPI_SPECULATE && use == 0) {
           // first tile of this CTA: max only, then agree on the estimate with the whole grid
           unsigned m0 = 0;
-          for (int c = 32 * chunk_phase; c < p.bn; c += 64) {
+          for (int c = 32 * chunk_phase; c < p.bn; c += 32 * EPI_PER_Q) {
             int v[32];
             tc_ld32(tm_row + (unsigned)c, v);
             if (row_ok) {
@@ -621,34 +649,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int8_t *dst8 = out8 + out_row * p.gn + col0;
         const int8_t *msk = mask8 ? mask8 + out_row * p.gn + col0 : nullptr;
         const bool vec_ok = ((p.gn & 15) == 0) && ((col0 & 15) == 0);
-        const unsigned qmax = (1u << p.mbits) - 1u;
-        // constants of the rounding rule for this binary point
-        const int odd = bp & 1, h = bp >> 1;
-        int sh_top, sh_bot;
-        unsigned hmask;
-        if (p.round_mode == NITI_ROUND_PSR) { sh_top = odd + h; sh_bot = odd; hmask = (1u << h) - 1u; }
-        else { sh_top = bp > 0 ? bp - 1 : 0; sh_bot = 0; hmask = bp > 0 ? 1u : 0u; }
-        int va[32], vb[32];
-        int c = 32 * chunk_phase;
-        if (c < p.bn) tc_ld32_issue(tm_row + (unsigned)c, va);
-        for (int it = 0; c < p.bn; c += 64, ++it) {
-          int (&v)[32] = (it & 1) ? vb : va;
-          int (&vn)[32] = (it & 1) ? va : vb;
-          tc_ld_wait(v);
-          if (c + 64 < p.bn) tc_ld32_issue(tm_row + (unsigned)(c + 64), vn);   // overlaps the math below
+        const RoundConst rk = make_round_const(bp, p.mbits, p.round_mode);
+        for (int c = 32 * chunk_phase; c < p.bn; c += 32 * EPI_PER_Q) {
+          int v[32];
+          tc_ld32(tm_row + (unsigned)c, v);
           if (row_ok && c < ncols_valid) {
             unsigned w8[8];
             unsigned orv = 0;
-            if (p.round_mode == NITI_ROUND_PSR) {
+            if (p.relu) {
 #pragma unroll
               for (int j = 0; j < 8; ++j)
-                w8[j] = round_pack4<NITI_ROUND_PSR>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], bp, sh_top,
-                                                    sh_bot, hmask, qmax, p.relu, orv);
+                w8[j] = round_pack4<true>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, orv);
             } else {
 #pragma unroll
               for (int j = 0; j < 8; ++j)
-                w8[j] = round_pack4<NITI_ROUND_NEAREST>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], bp,
-                                                        sh_top, sh_bot, hmask, qmax, p.relu, orv);
+                w8[j] = round_pack4<false>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, orv);
             }
             if (vec_ok && c + 32 <= ncols_valid) {
               mx |= orv;
