@@ -93,8 +93,10 @@ size_t niti_workspace_bytes(int op, const int64_t *dims, int ndims);
  * single-CTA kernel only, 3 = tensor cores with the paired-CTA kernel only
  * (falls back to CUDA cores where that kernel does not apply), 4 = tensor
  * cores with the two-pass epilogue (int32 accumulators spilled to the
- * workspace, rounded by a second kernel) instead of the fused one.  1-4 exist
- * so that tests can cross-check the engines.  Returns the previous value. */
+ * workspace, rounded by a second kernel) instead of the fused one, 5 = tensor
+ * cores without the weights-resident mode of small-channel 3x3 convolutions.
+ * 1-5 exist so that tests can cross-check the engines.  Returns the previous
+ * value. */
 int niti_set_engine(niti_ctx *ctx, int engine);
 
 /* Number of kernels / memsets this context has enqueued so far. */
@@ -117,6 +119,9 @@ int64_t niti_redo_count(niti_ctx *ctx, void *stream);
  * multiply), and starts a new record.  Host pointers. */
 int niti_profile_enable(niti_ctx *ctx, int on);
 int niti_profile_read(niti_ctx *ctx, double *tc_ms, uint64_t *tc_launches, double *tc_ops);
+/* Per-launch view of the same record (does not reset it): fills ms[i] and ops[i] for the first
+ * min(recorded, max_n) launches in launch order and returns that count (-1 on error). */
+int niti_profile_read_launches(niti_ctx *ctx, double *ms, double *ops, int max_n);
 
 /* Fully connected forward (Algorithm 1, forward loop; Section 3.2):
  *   acc[m][n] = sum_k a[m][k] * w[n][k];  b = B(acc);  bp = max(0, b - 7);

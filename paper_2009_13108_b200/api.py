@@ -20,7 +20,7 @@ OP_LINEAR_FWD, OP_LINEAR_BWD, OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_INT_
 EXPORTS = [
     "niti_create", "niti_destroy", "niti_last_error", "niti_check", "niti_workspace_bytes",
     "niti_set_engine", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
-    "niti_redo_count", "niti_profile_enable",
+    "niti_redo_count", "niti_profile_enable", "niti_profile_read_launches",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
     "niti_conv_dgrad", "niti_conv_wgrad", "niti_int_xent", "niti_int_sgd_update", "niti_relu_fwd",
     "niti_relu_bwd", "niti_maxpool2_fwd", "niti_maxpool2_bwd",
@@ -57,6 +57,7 @@ def load_library():
     lib.niti_tc_launch_count.restype = C.c_uint64
     lib.niti_tc_pair_launch_count.argtypes = [vp]
     lib.niti_tc_pair_launch_count.restype = C.c_uint64
+    lib.niti_profile_read_launches.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), i32]
     lib.niti_redo_count.argtypes = [vp, vp]
     lib.niti_redo_count.restype = C.c_int64
     lib.niti_profile_enable.argtypes = [vp, i32]
@@ -150,6 +151,15 @@ class Niti:
 
     def profile_enable(self, on: bool):
         self._ck(self.lib.niti_profile_enable(self.h, int(on)))
+
+    def profile_read_launches(self, max_n: int = 8192):
+        """[(ms, int8 ops)] of every recorded tensor-core launch, in launch order."""
+        ms = (C.c_double * max_n)()
+        ops = (C.c_double * max_n)()
+        n = self.lib.niti_profile_read_launches(self.h, ms, ops, max_n)
+        if n < 0:
+            raise NitiError(ERR_CUDA, "niti_profile_read_launches failed")
+        return [(ms[i], ops[i]) for i in range(n)]
 
     def profile_read(self):
         """(summed ms, launches, summed int8 ops) of the tensor-core kernel since the last read."""

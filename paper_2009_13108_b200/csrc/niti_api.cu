@@ -82,6 +82,19 @@ extern "C" int niti_profile_enable(niti_ctx *ctx, int on) {
   return NITI_OK;
 }
 
+extern "C" int niti_profile_read_launches(niti_ctx *ctx, double *ms, double *ops, int max_n) {
+  if (!ctx || !ms || !ops || max_n < 0) return -1;
+  int n = ctx->prof_used < max_n ? ctx->prof_used : max_n;
+  for (int i = 0; i < n; ++i) {
+    float t = 0;
+    if (cudaEventSynchronize(ctx->prof_ev[2 * i + 1]) != cudaSuccess) return -1;
+    if (cudaEventElapsedTime(&t, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]) != cudaSuccess) return -1;
+    ms[i] = t;
+    ops[i] = ctx->prof_ops[i];
+  }
+  return n;
+}
+
 extern "C" int niti_profile_read(niti_ctx *ctx, double *tc_ms, uint64_t *tc_launches, double *tc_ops) {
   if (!ctx || !tc_ms || !tc_launches || !tc_ops) return NITI_ERR_ARG;
   double ms = 0, ops = 0;

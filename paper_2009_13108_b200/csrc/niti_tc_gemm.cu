@@ -21,6 +21,7 @@ constexpr int EPI_WARPS = 16;          // four per TMEM lane quarter, interleave
 constexpr int EPI_PER_Q = EPI_WARPS / 4;
 constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int MAX_STAGES = 8;
+constexpr int MAX_TBUF = 8;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;
 
 struct TcParams {
@@ -55,6 +56,15 @@ struct TcParams {
   int ctas;                     // CTAs per tile: 1, or 2 (cta_group::2, 256-row tiles)
   int m_units;                  // row units: 128-row tiles (ctas = 1) or 256-row pairs (ctas = 2)
   int raster_g;                 // row units per rasterisation group (0: row-major order)
+  int blocked;                  // 1: every CTA takes a contiguous range of items (its first tile then
+                                //    samples the tensor evenly), 0: items strided over the grid
+  int nbuf;                     // accumulator buffers in tensor memory (2..8)
+  // halo mode (3x3 convolutions with few channels): the weights of all nine taps stay in shared
+  // memory for the whole kernel, every tile loads its 8 x 16 pixel patch once with a one-pixel
+  // halo (10 x 18 pixels), and the nine taps are nine row offsets into that patch
+  int halo;
+  int b_tile_bytes;             // bytes of one tap's weight tile
+  int b_res_bytes;              // bytes of the resident weights (all taps), multiple of 1024
   // epilogue
   int epi_mode;                 // EPI_SPILL / EPI_ATOMIC / EPI_SPECULATE / EPI_KNOWN_B
   int mbits, round_mode, relu;
@@ -155,30 +165,6 @@ __device__ __forceinline__ void tc_ld32(unsigned taddr, int (&v)[32]) {
       : "r"(taddr)
       : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// The same load without the wait, and a wait that names the registers so that no use of them can be
-// scheduled before it.
-__device__ __forceinline__ void tc_ld32_issue(unsigned taddr, int (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tc_ld_wait(int (&v)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
-                 "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
-                 "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
-                 "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
-               :
-               : "memory");
 }
 
 // Shift-and-round of four accumulators (Algorithm 2 + 3, or round-to-nearest) packed into four int8.
@@ -348,7 +334,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(status + 1, 1u);   // count of recomputations
   }
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 4];
+  __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 2 * MAX_TBUF + 1];
   __shared__ unsigned tmem_base_slot;
   __shared__ volatile int abort_flag;
 
@@ -359,16 +345,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const unsigned full0 = smem_u32(&bars[0]);
   const unsigned empty0 = smem_u32(&bars[MAX_STAGES]);
   const unsigned tfull0 = smem_u32(&bars[2 * MAX_STAGES]);
-  const unsigned tempty0 = smem_u32(&bars[2 * MAX_STAGES + 2]);
+  const unsigned tempty0 = smem_u32(&bars[2 * MAX_STAGES + MAX_TBUF]);
+  const unsigned bres_bar = smem_u32(&bars[2 * MAX_STAGES + 2 * MAX_TBUF]);   // resident weights landed
   // barriers of the leader CTA as seen from this CTA
   const unsigned lead_full0 = CTAS == 2 ? map_to_cta(full0, 0) : full0;
   const unsigned lead_tempty0 = CTAS == 2 ? map_to_cta(tempty0, 0) : tempty0;
-  const long long first_item = blockIdx.x / CTAS;
-  const long long item_step = gridDim.x / CTAS;
+  // items of this CTA (pair): first_item, first_item + item_step, ... below item_end
+  long long first_item = blockIdx.x / CTAS, item_step = gridDim.x / CTAS, item_end = p.items;
+  if (p.blocked) {
+    const long long units = gridDim.x / CTAS, u = blockIdx.x / CTAS;
+    const long long per = p.items / units, extra = p.items % units;
+    first_item = u * per + (u < extra ? u : extra);
+    item_end = first_item + per + (u < extra ? 1 : 0);
+    item_step = 1;
+  }
 
-  // TMEM columns: two accumulator buffers of bn columns, rounded up to a power of two >= 32
+  // TMEM columns: nbuf accumulator buffers of bn columns, rounded up to a power of two >= 32
   unsigned tmem_cols = 32;
-  while (tmem_cols < 2u * (unsigned)p.bn) tmem_cols <<= 1;
+  while (tmem_cols < (unsigned)(p.nbuf * p.bn)) tmem_cols <<= 1;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -376,7 +370,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    mbar_init(bres_bar, 1);
+    for (int b = 0; b < p.nbuf; ++b) {
       mbar_init(tfull0 + 8 * b, 1);
       mbar_init(tempty0 + 8 * b, EPI_WARPS * CTAS);     // one arrival per epilogue warp of every CTA
     }
@@ -407,7 +402,31 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       unsigned phase = 0;
       bool ok = true;
       const int bn_cta = p.bn / CTAS;             // B rows (output columns) staged by this CTA
-      for (long long item = first_item; ok && item < p.items; item += item_step) {
+      if (p.halo) {
+        // resident weights: one tile per tap, [bn rows][kdepth] K-major (forward) or
+        // [kdepth rows][bn] MN-major in b_boxes column chunks (dgrad)
+        mbar_expect_tx(bres_bar, (unsigned)(9 * p.b_boxes * p.b_box_bytes));
+        for (int tap = 0; tap < 9; ++tap) {
+          const unsigned dst = smem_base + tap * p.b_tile_bytes;
+          if (p.kind == GK_CONV_FWD) {
+            tma_load_2d(dst, &map_b, bres_bar, tap * p.kdepth, 0);
+          } else {
+            for (int j = 0; j < p.b_boxes; ++j)
+              tma_load_2d(dst + j * p.b_box_bytes, &map_b, bres_bar, tap * p.Cn + j * p.b_box_step, 0);
+          }
+        }
+        for (long long item = first_item; ok && item < item_end; item += item_step) {
+          int w0, h0, b0;
+          pixel_box(p, (int)item, w0, h0, b0);
+          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
+          const unsigned full = full0 + 8 * stage;
+          mbar_expect_tx(full, (unsigned)p.a_box_bytes);
+          tma_load_4d(smem_base + p.b_res_bytes + stage * p.a_bytes, &map_a, full, 0, w0 - 1, h0 - 1, b0);
+          if (++stage == p.stages) { stage = 0; phase ^= 1; }
+        }
+        item_end = first_item;                    // nothing left for the generic loop
+      }
+      for (long long item = first_item; ok && item < item_end; item += item_step) {
         int mu, nt, split;
         decode_item(p, item, mu, nt, split);
         const int mt = mu * CTAS + (int)rank;     // this CTA's 128-row tile
@@ -484,14 +503,42 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       unsigned phase = 0;
       unsigned use = 0;                 // tiles processed by this CTA (pair)
       bool ok = true;
-      for (long long item = first_item; ok && item < p.items; item += item_step, ++use) {
+      if (p.halo) {
+        ok = mbar_wait(bres_bar, 0, &abort_flag, status);
+        for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
+          const unsigned buf = use % (unsigned)p.nbuf;
+          if (!mbar_wait(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
+          if (!mbar_wait(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const unsigned tmem_d = tmem_base + buf * (unsigned)p.bn;
+          const unsigned sa = smem_base + p.b_res_bytes + stage * p.a_bytes;
+          for (int tap = 0; tap < 9; ++tap) {
+            const int r = tap / 3, t = tap % 3;
+            // patch row of the tile's first pixel for this tap: forward reads x[i + r - 1][j + t - 1],
+            // dgrad reads e[i - r + 1][j - t + 1]; the patch starts one pixel up and left
+            const int rowoff = p.kind == GK_CONV_FWD ? r * 10 + t : (2 - r) * 10 + (2 - t);
+            unsigned long long da = p.a_desc | (unsigned long long)(((sa + rowoff * p.kdepth) >> 4) & 0x3fff);
+            unsigned long long db = p.b_desc | (unsigned long long)(((smem_base + tap * p.b_tile_bytes) >> 4) & 0x3fff);
+            for (int k = 0; k < p.ksteps; ++k) {
+              tc_mma_i8(tmem_d, da, db, p.idesc, (tap > 0 || k > 0) ? 1u : 0u);
+              da += p.a_kstep16;
+              db += p.b_kstep16;
+            }
+          }
+          tc_commit(empty0 + 8 * stage);
+          tc_commit(tfull0 + 8 * buf);
+          if (++stage == p.stages) { stage = 0; phase ^= 1; }
+        }
+        item_end = first_item;
+      }
+      for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
         const int split = (int)(item % p.splits);
         const int kb0 = split * p.kb_per_split;
         int kb1 = kb0 + p.kb_per_split;
         if (kb1 > p.kb_total) kb1 = p.kb_total;
-        const unsigned buf = use & 1u;
-        // wait until the epilogue has drained this accumulator buffer (first two uses pass at once)
-        if (!mbar_wait(tempty0 + 8 * buf, ((use >> 1) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
+        const unsigned buf = use % (unsigned)p.nbuf;
+        // wait until the epilogue has drained this accumulator buffer (the first nbuf uses pass at once)
+        if (!mbar_wait(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
         tc_fence_after();
         const unsigned tmem_d = tmem_base + buf * (unsigned)p.bn;
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -531,11 +578,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bp = b > p.mbits ? b - p.mbits : 0;
     }
     bool ok = true;
-    for (long long item = first_item; ok && item < p.items; item += item_step, ++use) {
+    for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
       int mu, nt, split;
       decode_item(p, item, mu, nt, split);
       const int mt = mu * CTAS + (int)rank;
-      const unsigned buf = use & 1u;
+      const unsigned buf = use % (unsigned)p.nbuf;
       // output row / column base of this thread
       long long out_row;
       bool row_ok;
@@ -566,7 +613,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         long long rem = p.gn - col0;
         ncols_valid = rem < p.bn ? (int)rem : p.bn;
       }
-      if (!mbar_wait(tfull0 + 8 * buf, (use >> 1) & 1u, &abort_flag, status)) { ok = false; break; }
+      if (!mbar_wait(tfull0 + 8 * buf, (use / (unsigned)p.nbuf) & 1u, &abort_flag, status)) { ok = false; break; }
       tc_fence_after();
       const unsigned tm_row = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * (unsigned)p.bn;
       if (p.epi_mode <= EPI_ATOMIC) {
@@ -743,10 +790,10 @@ static unsigned long long layout_bits(int swizzle_bytes) {
   return t << 61;
 }
 // Descriptor (without start address) of a K-major operand whose rows are `sw` bytes wide.
-static unsigned long long desc_kmajor(int sw) {
+static unsigned long long desc_kmajor(int sw, int group_rows = 8) {
   unsigned long long d = 0;
   d |= (unsigned long long)1 << 16;                          // leading byte offset: unused, 1
-  d |= (unsigned long long)((8 * sw) >> 4) << 32;            // stride between 8-row groups
+  d |= (unsigned long long)((group_rows * sw) >> 4) << 32;   // stride between 8-row groups
   d |= (unsigned long long)1 << 46;                          // descriptor version
   return d | layout_bits(sw);
 }
@@ -799,7 +846,8 @@ static bool pick_pixel_box(int W, int H, int B, int &Wt, int &Ht, int &Bt) {
 static int round_up32(long long n) { return (int)((n + 31) / 32 * 32); }
 
 // Builds params and maps; returns false if the shape is not eligible for this engine.
-static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, TcParams &p, CUtensorMap &ma, CUtensorMap &mb) {
+static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, TcParams &p, CUtensorMap &ma,
+                 CUtensorMap &mb) {
   memset(&p, 0, sizeof(p));
   p.ctas = ctas;
   p.kind = g.kind;
@@ -896,6 +944,24 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, TcParams &p, CUt
       p.kb_total = g.R * g.S * p.c_chunks;
       m_tiles = (long long)p.w_tiles * p.h_tiles * p.b_tiles;
       p.n_tiles_n = (Cn + p.bn - 1) / p.bn;
+      // halo mode: one channel chunk, one column tile, weights of all taps fit beside >= 3 patches
+      if (want_halo && ctas == 1 && g.R == 3 && g.S == 3 && g.pad == 1 && p.c_chunks == 1 && p.n_tiles_n == 1 &&
+          g.W >= 10 && g.H >= 18) {
+        const int a_stage = (180 * p.kdepth + 1023) / 1024 * 1024;
+        const int b_res = (9 * p.bn * p.kdepth + 1023) / 1024 * 1024;
+        if (b_res + 3 * a_stage <= 200 * 1024) {
+          p.halo = 1;
+          p.Wt = 8; p.Ht = 16; p.Bt = 1;
+          p.w_tiles = (g.W + 7) / 8;
+          p.h_tiles = (g.H + 15) / 16;
+          p.b_tiles = g.B;
+          m_tiles = (long long)p.w_tiles * p.h_tiles * p.b_tiles;
+          sa.box[1] = 10; sa.box[2] = 18; sa.box[3] = 1;
+          if (fwd) sb.box[1] = (cuuint32_t)p.bn;
+          p.b_tile_bytes = p.bn * p.kdepth;
+          p.b_res_bytes = b_res;
+        }
+      }
       break;
     }
     case GK_CONV_WGRAD: {
@@ -968,6 +1034,15 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, TcParams &p, CUt
   p.b_bytes = (p.b_bytes + 1023) / 1024 * 1024;
   int stage_bytes = p.a_bytes + p.b_bytes;
   p.stages = (200 * 1024) / stage_bytes;
+  if (p.halo) {
+    // a stage is one 10 x 18 pixel patch; consecutive 8-row groups of a tap are one patch row apart
+    p.a_box_bytes = 180 * p.kdepth;
+    p.a_bytes = (p.a_box_bytes + 1023) / 1024 * 1024;
+    p.a_desc = desc_kmajor(a_sw, 10);
+    p.b_bytes = 0;
+    stage_bytes = p.a_bytes;
+    p.stages = (200 * 1024 - p.b_res_bytes) / stage_bytes;
+  }
   if (p.stages > MAX_STAGES) p.stages = MAX_STAGES;
   if (p.stages < 2) return false;
   // instruction descriptor: s32 accumulate, signed 8-bit operands, majorness, N, M
@@ -988,6 +1063,15 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, TcParams &p, CUt
   }
   p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
   p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+  if (p.halo) {
+    p.splits = 1;
+    p.kb_per_split = p.kb_total;
+  }
+  p.nbuf = 512 / p.bn;
+  if (p.nbuf > MAX_TBUF) p.nbuf = MAX_TBUF;
+  // convolution outputs are spatially structured (borders, images): contiguous item ranges make the
+  // first tile of every CTA an even sample of the tensor for the speculative shift
+  p.blocked = (g.kind == GK_CONV_FWD || g.kind == GK_CONV_DGRAD) ? 1 : 0;
   p.items = tiles * p.splits;
   if (!encode(ctx, &ma, sa) || !encode(ctx, &mb, sb)) return false;
   return true;
@@ -1002,7 +1086,7 @@ size_t niti_tc_scratch_bytes(const GemmProblem &) { return 0; }
 template <int CTAS>
 static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CUtensorMap &ma, const CUtensorMap &mb,
                      int32_t *acc, WsHeader *hdr, const RoundSpec &r) {
-  size_t smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + 1024;
+  size_t smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + (size_t)p.b_res_bytes + 1024;
   static size_t attr_smem = 0;
   if (smem > attr_smem) {
     NITI_CUDA_TRY(ctx, cudaFuncSetAttribute(tc_gemm_kernel<CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -1052,14 +1136,17 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
   *fused = false;
   // engine 0: pairs of CTAs (cta_group::2) when there are enough 256-row tiles to fill the GPU.
   // Test switches: 2 / 3 force the single-CTA / paired kernel, 4 keeps the int32 spill epilogue.
+  // Test switches: 5 disables the halo mode of small-channel convolutions.
   bool planned = false;
-  if (ctx->engine != 2 && g.gm >= 2 * BM) {
-    planned = plan(ctx, g, 2, p, ma, mb);
+  if ((g.kind == GK_CONV_FWD || g.kind == GK_CONV_DGRAD) && ctx->engine != 3 && ctx->engine != 5)
+    planned = plan(ctx, g, 1, true, p, ma, mb) && p.halo;
+  if (!planned && ctx->engine != 2 && g.gm >= 2 * BM) {
+    planned = plan(ctx, g, 2, false, p, ma, mb);
     if (planned && ctx->engine != 3 && p.items < ctx->sm_count / 2) planned = false;
   }
   if (!planned) {
     if (ctx->engine == 3) return NITI_ERR_SHAPE;
-    if (!plan(ctx, g, 1, p, ma, mb)) return NITI_ERR_SHAPE;
+    if (!plan(ctx, g, 1, false, p, ma, mb)) return NITI_ERR_SHAPE;
   }
   p.mbits = r.mbits;
   p.round_mode = r.round_mode;

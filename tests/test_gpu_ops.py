@@ -83,10 +83,11 @@ def test_linear_bwd(niti, oref, M, N, K, engine):
 
 CONV_SHAPES = [(2, 8, 8, 3, 16), (2, 16, 16, 64, 64), (4, 8, 8, 128, 256), (8, 4, 4, 256, 128),
                (2, 32, 32, 32, 64), (3, 28, 28, 1, 32), (2, 28, 28, 32, 64), (32, 2, 2, 512, 512),
-               (1, 56, 56, 64, 128), (2, 12, 20, 96, 160)]
+               (1, 56, 56, 64, 128), (2, 12, 20, 96, 160), (2, 24, 40, 128, 128), (1, 64, 48, 64, 64),
+               (2, 18, 10, 128, 64), (3, 30, 22, 32, 96)]
 
 
-@pytest.mark.parametrize("engine", [0, 1, 2, 3, 4])
+@pytest.mark.parametrize("engine", [0, 1, 2, 3, 4, 5])
 @pytest.mark.parametrize("B,H,W,Ci,Co", CONV_SHAPES)
 def test_conv_ops(niti, oref, B, H, W, Ci, Co, engine):
     rng = np.random.default_rng(B + H * 3 + W * 5 + Ci * 7 + Co * 11)
