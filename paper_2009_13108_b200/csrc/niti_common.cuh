@@ -34,8 +34,9 @@ struct WsHeader {
   unsigned int maxabs32;            // a value with the bit length of max |acc| (a max, or an OR of magnitudes)
   unsigned int est_max;             // max |acc| over the first tile of every CTA (speculative shift)
   unsigned long long maxabs64;      // same for the 64-bit loss accumulators
-  unsigned int tile_counter;        // dynamic tile scheduler / arrival counter
-  unsigned int pad1[3];
+  unsigned int tile_counter;        // arrival counter of the grid-wide wait
+  unsigned int spec_b;              // bit-width the speculative epilogue rounded with
+  unsigned int pad1[2];
 };
 
 #define NITI_CUDA_TRY(ctx, expr)                                                        \

@@ -13,6 +13,7 @@
 // NITI_DEV_TIMEOUT in the status word, and all roles drain and leave through the common exit
 // that frees the tensor memory.
 #include "niti_common.cuh"
+#include <math.h>
 
 namespace {
 
@@ -68,6 +69,7 @@ struct TcParams {
   // epilogue
   int epi_mode;                 // EPI_SPILL / EPI_ATOMIC / EPI_SPECULATE / EPI_KNOWN_B
   int mbits, round_mode, relu;
+  unsigned spec_mul256;         // the sampled max is scaled by this / 256 before taking its bit length
 };
 
 // Epilogue modes.  The shift of Algorithm 2 needs the bit-width of the WHOLE accumulator tensor:
@@ -151,6 +153,19 @@ __device__ __forceinline__ void tc_mma_i8(unsigned tmem_d, unsigned long long da
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Same with the two 64-bit matrix descriptors given as 32-bit halves: the issuing thread then does
+// its address arithmetic in 32 bits (the high halves never change inside a kernel).
+__device__ __forceinline__ void tc_mma_i8_lh(unsigned tmem_d, unsigned a_lo, unsigned a_hi, unsigned b_lo,
+                                             unsigned b_hi, unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}"
+      ::"r"(tmem_d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tc_ld32(unsigned taddr, int (&v)[32]) {
@@ -320,7 +335,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                const int32_t *s_w, int32_t *s_out, int32_t *b_out) {
   if (p.epi_mode == EPI_KNOWN_B) {
     // follow-up of a speculative pass: publish the scalars, then leave unless the guess was wrong
-    const int b_true = niti_bitlen32(hdr->maxabs32), b_est = niti_bitlen32(hdr->est_max);
+    const int b_true = niti_bitlen32(hdr->maxabs32), b_est = (int)hdr->spec_b;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       const int bp = b_true > p.mbits ? b_true - p.mbits : 0;
       if (b_out) *b_out = b_true;
@@ -415,14 +430,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               tma_load_2d(dst + j * p.b_box_bytes, &map_b, bres_bar, tap * p.Cn + j * p.b_box_step, 0);
           }
         }
-        for (long long item = first_item; ok && item < item_end; item += item_step) {
-          int w0, h0, b0;
-          pixel_box(p, (int)item, w0, h0, b0);
+        // consecutive items are consecutive tiles (blocked assignment): step the tile coordinates
+        int wt = (int)(first_item % p.w_tiles), ht = (int)((first_item / p.w_tiles) % p.h_tiles);
+        int bt = (int)(first_item / ((long long)p.w_tiles * p.h_tiles));
+        for (long long item = first_item; ok && item < item_end; ++item) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
           const unsigned full = full0 + 8 * stage;
           mbar_expect_tx(full, (unsigned)p.a_box_bytes);
-          tma_load_4d(smem_base + p.b_res_bytes + stage * p.a_bytes, &map_a, full, 0, w0 - 1, h0 - 1, b0);
+          tma_load_4d(smem_base + p.b_res_bytes + stage * p.a_bytes, &map_a, full, 0, wt * 8 - 1, ht * 16 - 1, bt);
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
+          if (++wt == p.w_tiles) { wt = 0; if (++ht == p.h_tiles) { ht = 0; ++bt; } }
         }
         item_end = first_item;                    // nothing left for the generic loop
       }
@@ -505,24 +522,35 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bool ok = true;
       if (p.halo) {
         ok = mbar_wait(bres_bar, 0, &abort_flag, status);
+        // descriptor low words per tap, computed once: the patch row where the tap starts
+        // (forward reads x[i + r - 1][j + t - 1], dgrad reads e[i - r + 1][j - t + 1]; the patch
+        // starts one pixel up and left of the tile) and the tap's resident weight tile
+        const unsigned a_hi = (unsigned)(p.a_desc >> 32), b_hi = (unsigned)(p.b_desc >> 32);
+        const unsigned a_lo0 = (unsigned)p.a_desc, b_lo0 = (unsigned)p.b_desc + ((smem_base >> 4) & 0x3fff);
+        unsigned a_off[9], b_off[9];
+#pragma unroll
+        for (int tap = 0; tap < 9; ++tap) {
+          const int r = tap / 3, t = tap % 3;
+          const int rowoff = p.kind == GK_CONV_FWD ? r * 10 + t : (2 - r) * 10 + (2 - t);
+          a_off[tap] = (unsigned)(rowoff * p.kdepth) >> 4;
+          b_off[tap] = (unsigned)(tap * p.b_tile_bytes) >> 4;
+        }
+        const unsigned a_stage16 = (unsigned)p.a_bytes >> 4;
+        unsigned a_stage_lo = a_lo0 + (((smem_base + p.b_res_bytes) >> 4) & 0x3fff);   // stage 0
         for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
           const unsigned buf = use % (unsigned)p.nbuf;
           if (!mbar_wait(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
           if (!mbar_wait(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
           tc_fence_after();
           const unsigned tmem_d = tmem_base + buf * (unsigned)p.bn;
-          const unsigned sa = smem_base + p.b_res_bytes + stage * p.a_bytes;
+          const unsigned a_lo = a_stage_lo + (unsigned)stage * a_stage16;
+#pragma unroll
           for (int tap = 0; tap < 9; ++tap) {
-            const int r = tap / 3, t = tap % 3;
-            // patch row of the tile's first pixel for this tap: forward reads x[i + r - 1][j + t - 1],
-            // dgrad reads e[i - r + 1][j - t + 1]; the patch starts one pixel up and left
-            const int rowoff = p.kind == GK_CONV_FWD ? r * 10 + t : (2 - r) * 10 + (2 - t);
-            unsigned long long da = p.a_desc | (unsigned long long)(((sa + rowoff * p.kdepth) >> 4) & 0x3fff);
-            unsigned long long db = p.b_desc | (unsigned long long)(((smem_base + tap * p.b_tile_bytes) >> 4) & 0x3fff);
-            for (int k = 0; k < p.ksteps; ++k) {
-              tc_mma_i8(tmem_d, da, db, p.idesc, (tap > 0 || k > 0) ? 1u : 0u);
-              da += p.a_kstep16;
-              db += p.b_kstep16;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              if (k < p.ksteps)
+                tc_mma_i8_lh(tmem_d, a_lo + a_off[tap] + 2 * k, a_hi, b_lo0 + b_off[tap] + k * p.b_kstep16, b_hi,
+                             p.idesc, (tap > 0 || k > 0) ? 1u : 0u);
             }
           }
           tc_commit(empty0 + 8 * stage);
@@ -573,14 +601,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     unsigned mx = 0;
     unsigned spec_max = 0;
     int bp = 0;
+    int h_wt = 0, h_ht = 0, h_bt = 0;
     if (p.epi_mode == EPI_KNOWN_B) {
       const int b = niti_bitlen32(hdr->maxabs32);
       bp = b > p.mbits ? b - p.mbits : 0;
     }
     bool ok = true;
     for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
-      int mu, nt, split;
-      decode_item(p, item, mu, nt, split);
+      int mu = 0, nt = 0, split = 0;
+      if (!p.halo) decode_item(p, item, mu, nt, split);
       const int mt = mu * CTAS + (int)rank;
       const unsigned buf = use % (unsigned)p.nbuf;
       // output row / column base of this thread
@@ -588,7 +617,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bool row_ok;
       long long col0;
       int ncols_valid;
-      if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) {
+      if (p.halo) {
+        // 8 x 16 pixel tiles of one image, visited in order: coordinates are stepped, not divided
+        if (use == 0) {
+          h_wt = (int)(first_item % p.w_tiles);
+          h_ht = (int)((first_item / p.w_tiles) % p.h_tiles);
+          h_bt = (int)(first_item / ((long long)p.w_tiles * p.h_tiles));
+        }
+        const int w = h_wt * 8 + (row_in_tile & 7), h = h_ht * 16 + (row_in_tile >> 3);
+        row_ok = w < p.PW && h < p.PH;
+        out_row = ((long long)h_bt * p.PH + h) * p.PW + w;
+        col0 = 0;
+        ncols_valid = (int)p.gn;
+        if (++h_wt == p.w_tiles) { h_wt = 0; if (++h_ht == p.h_tiles) { h_ht = 0; ++h_bt; } }
+      } else if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) {
         int w0, h0, b0;
         pixel_box(p, mt, w0, h0, b0);
         int ww = row_in_tile % p.Wt, t = row_in_tile / p.Wt;
@@ -690,8 +732,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (abort_flag) { ok = false; break; }
           if (lane == 0) spec_max = *(volatile unsigned *)&hdr->est_max;
           spec_max = __shfl_sync(0xffffffffu, spec_max, 0);
-          const int b = niti_bitlen32(spec_max);
+          // the first tiles are a sample: scale their max by the growth expected from the sample to
+          // the whole tensor before taking the bit length (a wrong guess only costs the redo pass)
+          unsigned long long scaled = ((unsigned long long)spec_max * p.spec_mul256) >> 8;
+          if (scaled > 0x7fffffffull) scaled = 0x7fffffffull;
+          const int b = niti_bitlen32((unsigned)scaled);
           bp = b > p.mbits ? b - p.mbits : 0;
+          if (blockIdx.x == 0 && warp == 2 && lane == 0) hdr->spec_b = (unsigned)b;
         }
         int8_t *dst8 = out8 + out_row * p.gn + col0;
         const int8_t *msk = mask8 ? mask8 + out_row * p.gn + col0 : nullptr;
@@ -949,7 +996,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
           g.W >= 10 && g.H >= 18) {
         const int a_stage = (180 * p.kdepth + 1023) / 1024 * 1024;
         const int b_res = (9 * p.bn * p.kdepth + 1023) / 1024 * 1024;
-        if (b_res + 3 * a_stage <= 200 * 1024) {
+        if (b_res + 3 * a_stage <= 224 * 1024) {
           p.halo = 1;
           p.Wt = 8; p.Ht = 16; p.Bt = 1;
           p.w_tiles = (g.W + 7) / 8;
@@ -1041,7 +1088,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
     p.a_desc = desc_kmajor(a_sw, 10);
     p.b_bytes = 0;
     stage_bytes = p.a_bytes;
-    p.stages = (200 * 1024 - p.b_res_bytes) / stage_bytes;
+    p.stages = (224 * 1024 - p.b_res_bytes) / stage_bytes;
   }
   if (p.stages > MAX_STAGES) p.stages = MAX_STAGES;
   if (p.stages < 2) return false;
@@ -1147,6 +1194,16 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
   if (!planned) {
     if (ctx->engine == 3) return NITI_ERR_SHAPE;
     if (!plan(ctx, g, 1, false, p, ma, mb)) return NITI_ERR_SHAPE;
+  }
+  {
+    // expected ratio between the max of the whole tensor (N values) and the max of the first tile of
+    // every CTA (n values) for roughly Gaussian sums: sqrt(ln N / ln n)
+    const int units = ctx->sm_count / p.ctas;
+    const double n_all = (double)g.gm * (double)g.gn;
+    const double frac = p.items > units ? (double)units / (double)p.items : 1.0;
+    const double n_s = n_all * frac;
+    double f = (n_s > 16.0 && frac < 1.0) ? sqrt(log(n_all) / log(n_s)) : 1.0;
+    p.spec_mul256 = (unsigned)(f * 256.0 + 0.5);
   }
   p.mbits = r.mbits;
   p.round_mode = r.round_mode;
