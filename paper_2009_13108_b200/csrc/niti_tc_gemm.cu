@@ -457,14 +457,27 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tap_n = nt / p.n_chunks;
           ci0 = (nt % p.n_chunks) * p.bn + (int)rank * bn_cta;
         }
+        // k-block counters, stepped instead of divided inside the loop (one thread issues all copies,
+        // so every scalar instruction here is on the critical path):
+        //   forward / dgrad: k-block = (tap row r, tap column s, channel chunk cc)
+        //   wgrad:           k-block = pixel box (kwt, kht, kbt)
+        int cc = 0, ts = 0, tr = 0, kwt = 0, kht = 0, kbt = 0;
+        if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) {
+          const int tap = kb0 / p.c_chunks;
+          cc = kb0 % p.c_chunks; tr = tap / p.S; ts = tap % p.S;
+        } else if (p.kind == GK_CONV_WGRAD) {
+          kwt = kb0 % p.w_tiles;
+          const int t = kb0 / p.w_tiles;
+          kht = t % p.h_tiles; kbt = t / p.h_tiles;
+        }
+        const int wg_r = tap_n / p.S, wg_s = tap_n % p.S;
+        const unsigned tx_bytes = (unsigned)(CTAS * (p.a_boxes * p.a_box_bytes + p.b_boxes * p.b_box_bytes));
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
           const unsigned full = lead_full0 + 8 * stage;
           const unsigned sa = smem_base + stage * stage_bytes;
           const unsigned sb = sa + p.a_bytes;
-          if (rank == 0)
-            mbar_expect_tx(full0 + 8 * stage,
-                           (unsigned)(CTAS * (p.a_boxes * p.a_box_bytes + p.b_boxes * p.b_box_bytes)));
+          if (rank == 0) mbar_expect_tx(full0 + 8 * stage, tx_bytes);
           switch (p.kind) {
             case GK_FC_FWD:       // A [M][K] K-major, B [N][K] K-major
               load2<CTAS>(sa, &map_a, full, kb * p.kdepth, mt * BM);
@@ -481,33 +494,31 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               for (int j = 0; j < p.b_boxes; ++j)
                 load2<CTAS>(sb + j * p.b_box_bytes, &map_b, full, nb + j * p.b_box_step, kb * p.kdepth);
               break;
-            case GK_CONV_FWD: {   // k-block = (tap, channel chunk)
-              int tap = kb / p.c_chunks, cc = kb % p.c_chunks;
-              int r = tap / p.S, s = tap % p.S;
-              load4<CTAS>(sa, &map_a, full, cc * p.kdepth, w0 + s - p.pad, h0 + r - p.pad, b0);
+            case GK_CONV_FWD:     // k-block = (tap, channel chunk)
+              load4<CTAS>(sa, &map_a, full, cc * p.kdepth, w0 + ts - p.pad, h0 + tr - p.pad, b0);
               load2<CTAS>(sb, &map_b, full, kb * p.kdepth, nb);
               break;
-            }
             case GK_CONV_DGRAD: { // A = e shifted the other way; B(ci, (tap, co)) = w[co][tap][ci]
-              int tap = kb / p.c_chunks, cc = kb % p.c_chunks;
-              int r = tap / p.S, s = tap % p.S;
-              load4<CTAS>(sa, &map_a, full, cc * p.kdepth, w0 - s + p.pad, h0 - r + p.pad, b0);
+              load4<CTAS>(sa, &map_a, full, cc * p.kdepth, w0 - ts + p.pad, h0 - tr + p.pad, b0);
+              const int col = (tr * p.S + ts) * p.Cn + nb;
               for (int j = 0; j < p.b_boxes; ++j)
-                load2<CTAS>(sb + j * p.b_box_bytes, &map_b, full, tap * p.Cn + nb + j * p.b_box_step,
-                            cc * p.kdepth);
+                load2<CTAS>(sb + j * p.b_box_bytes, &map_b, full, col + j * p.b_box_step, cc * p.kdepth);
               break;
             }
             default: {            // GK_CONV_WGRAD: k-block = pixel box; A = e, B = x shifted by the tap
-              int kw0, kh0, kbb0;
-              pixel_box(p, kb, kw0, kh0, kbb0);
-              int r = tap_n / p.S, s = tap_n % p.S;
+              const int kw0 = kwt * p.Wt, kh0 = kht * p.Ht, kbb0 = kbt * p.Bt;
               for (int j = 0; j < p.a_boxes; ++j)
                 load4<CTAS>(sa + j * p.a_box_bytes, &map_a, full, mt * BM + j * p.a_box_step, kw0, kh0, kbb0);
               for (int j = 0; j < p.b_boxes; ++j)
-                load4<CTAS>(sb + j * p.b_box_bytes, &map_b, full, ci0 + j * p.b_box_step, kw0 + s - p.pad,
-                            kh0 + r - p.pad, kbb0);
+                load4<CTAS>(sb + j * p.b_box_bytes, &map_b, full, ci0 + j * p.b_box_step, kw0 + wg_s - p.pad,
+                            kh0 + wg_r - p.pad, kbb0);
               break;
             }
+          }
+          if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) {
+            if (++cc == p.c_chunks) { cc = 0; if (++ts == p.S) { ts = 0; ++tr; } }
+          } else if (p.kind == GK_CONV_WGRAD) {
+            if (++kwt == p.w_tiles) { kwt = 0; if (++kht == p.h_tiles) { kht = 0; ++kbt; } }
           }
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
         }
@@ -574,14 +585,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tc_fence_after();
           const unsigned sa = smem_base + stage * stage_bytes;
           const unsigned sb = sa + p.a_bytes;
-          unsigned long long da = p.a_desc | (unsigned long long)((sa >> 4) & 0x3fff);
-          unsigned long long db = p.b_desc | (unsigned long long)((sb >> 4) & 0x3fff);
-          for (int k = 0; k < p.ksteps; ++k) {
-            const unsigned accum = (kb > kb0 || k > 0) ? 1u : 0u;
-            if (CTAS == 2) tc_mma_i8_pair(tmem_d, da, db, p.idesc, accum);
-            else tc_mma_i8(tmem_d, da, db, p.idesc, accum);
-            da += p.a_kstep16;
-            db += p.b_kstep16;
+          if (CTAS == 2) {
+            unsigned long long da = p.a_desc | (unsigned long long)((sa >> 4) & 0x3fff);
+            unsigned long long db = p.b_desc | (unsigned long long)((sb >> 4) & 0x3fff);
+            for (int k = 0; k < p.ksteps; ++k) {
+              tc_mma_i8_pair(tmem_d, da, db, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+              da += p.a_kstep16;
+              db += p.b_kstep16;
+            }
+          } else {
+            unsigned a_lo = (unsigned)p.a_desc + ((sa >> 4) & 0x3fff), b_lo = (unsigned)p.b_desc + ((sb >> 4) & 0x3fff);
+            const unsigned a_hi = (unsigned)(p.a_desc >> 32), b_hi = (unsigned)(p.b_desc >> 32);
+            for (int k = 0; k < p.ksteps; ++k) {
+              tc_mma_i8_lh(tmem_d, a_lo, a_hi, b_lo, b_hi, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+              a_lo += p.a_kstep16;
+              b_lo += p.b_kstep16;
+            }
           }
           // frees the stage (in every CTA of the pair) once these MMAs have read it
           if (CTAS == 2) tc_commit_pair(empty0 + 8 * stage); else tc_commit(empty0 + 8 * stage);
