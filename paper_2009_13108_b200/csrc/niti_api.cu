@@ -3,6 +3,16 @@
 #include "niti_common.cuh"
 
 int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr);
+int niti_launch_im2col32(niti_ctx *ctx, cudaStream_t st, const int8_t *x, int8_t *xcol, int B, int H, int W,
+                         int Ci, int R, int S, int pad, int Ho, int Wo);
+int niti_launch_pad_rows32(niti_ctx *ctx, cudaStream_t st, const int8_t *w, int8_t *wcol, int rows, int k);
+int niti_launch_round_compact32(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, const WsHeader *hdr, int8_t *out,
+                                int rows, int k, int mbits, int round_mode, int32_t *b_out);
+
+// Few-channel convolutions (R*S*Cin <= 32 and Cin not a multiple of 16, i.e. no TMA view of the
+// NHWC tensor): gathered into K = 32 rows and run as a plain matrix multiply.
+static inline bool few_channel_conv(int Ci, int R, int S) { return R * S * Ci <= 32 && (Ci % 16) != 0; }
+static inline size_t round_up(size_t v, size_t a);
 
 extern "C" int niti_create(niti_ctx **out, int device) {
   if (!out) return NITI_ERR_ARG;
@@ -128,6 +138,7 @@ extern "C" int niti_check(niti_ctx *ctx, void *stream, uint32_t *status) {
 
 static inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+
 static bool fill_conv(GemmProblem &p, int kind, int B, int H, int W, int Ci, int Co, int R, int S,
                       int pad) {
   p.kind = kind;
@@ -183,6 +194,11 @@ extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
         return 0;
       outs = (size_t)(p.gm * p.gn);
       extra = niti_tc_scratch_bytes(p);
+      if (few_channel_conv((int)d[3], (int)d[5], (int)d[6]) && op != NITI_OP_CONV_DGRAD) {
+        const size_t M = (size_t)d[0] * p.Ho * p.Wo;
+        extra += round_up(M * 32, 256) + round_up((size_t)d[4] * 32, 256) + round_up((size_t)d[4] * 32 * 4, 256);
+        if (op == NITI_OP_CONV_FWD && outs < M * (size_t)d[4]) outs = M * (size_t)d[4];
+      }
       break;
     }
     case NITI_OP_INT_XENT:
@@ -275,8 +291,25 @@ extern "C" int niti_conv_fwd(niti_ctx *ctx, void *stream, const int8_t *x, const
     return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_fwd: bad argument (pointers must be 16-byte aligned)");
   p.p0 = x; p.p1 = w;
   int64_t dims[8] = {B, H, W, Cin, Cout, R, S, pad};
-  return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes,
-                        niti_workspace_bytes(NITI_OP_CONV_FWD, dims, 8), y, 7, round_mode, relu, nullptr,
+  const size_t need = niti_workspace_bytes(NITI_OP_CONV_FWD, dims, 8);
+  if (few_channel_conv(Cin, R, S) && ctx->engine != 1) {
+    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
+      return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    // gather the taps into [M][32] rows, pad the weights to [Cout][32], then a K = 32 multiply
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t M = (size_t)p.gm;
+    char *base = (char *)ws + NITI_WS_HEADER + round_up(M * (size_t)Cout * 4, 256);
+    int8_t *xcol = (int8_t *)base;
+    int8_t *wcol = (int8_t *)(base + round_up(M * 32, 256));
+    int rc = niti_launch_im2col32(ctx, st, x, xcol, B, H, W, Cin, R, S, pad, p.Ho, p.Wo);
+    if (rc == NITI_OK) rc = niti_launch_pad_rows32(ctx, st, w, wcol, Cout, R * S * Cin);
+    if (rc != NITI_OK) return rc;
+    GemmProblem q;
+    fill_fc(q, GK_FC_FWD, (int)M, Cout, 32);
+    q.p0 = xcol; q.p1 = wcol;
+    return run_gemm_round(ctx, st, q, ws, ws_bytes, need, y, 7, round_mode, relu, nullptr, s_x, s_w, s_y, b_y);
+  }
+  return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, y, 7, round_mode, relu, nullptr,
                         s_x, s_w, s_y, b_y);
 }
 
@@ -310,7 +343,35 @@ extern "C" int niti_conv_wgrad(niti_ctx *ctx, void *stream, const int8_t *x, con
     return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_wgrad: bad argument (pointers must be 16-byte aligned)");
   p.p0 = e; p.p1 = x;
   int64_t dims[8] = {B, H, W, Cin, Cout, R, S, pad};
-  return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes,
-                        niti_workspace_bytes(NITI_OP_CONV_WGRAD, dims, 8), g, m_u, round_mode, 0, nullptr,
+  const size_t need = niti_workspace_bytes(NITI_OP_CONV_WGRAD, dims, 8);
+  if (few_channel_conv(Cin, R, S) && ctx->engine != 1 && (Cout % 16) == 0) {
+    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
+      return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    // g32[co][k] = sum_pix e[pix][co] * xcol[pix][k] over the gathered rows (k < 32), then the first
+    // R*S*Cin columns are rounded into g
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t M = (size_t)B * p.Ho * p.Wo;
+    WsHeader *hdr = (WsHeader *)ws;
+    char *base = (char *)ws + NITI_WS_HEADER + round_up((size_t)(p.gm * p.gn) * 4, 256);
+    int8_t *xcol = (int8_t *)base;
+    int32_t *acc32 = (int32_t *)(base + round_up(M * 32, 256) + round_up((size_t)Cout * 32, 256));
+    NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, sizeof(WsHeader), st));
+    ctx->launches++;
+    int rc = niti_launch_im2col32(ctx, st, x, xcol, B, H, W, Cin, R, S, pad, p.Ho, p.Wo);
+    if (rc != NITI_OK) return rc;
+    GemmProblem q;
+    fill_fc(q, GK_FC_WGRAD, (int)M, Cout, 32);     // rows M are the contraction
+    q.p0 = e; q.p1 = xcol;
+    bool fused = false;
+    RoundSpec none = {nullptr, nullptr, m_u, round_mode, 0, nullptr, nullptr, nullptr, nullptr};
+    const int saved = ctx->engine;
+    if (saved == 0) ctx->engine = 4;               // int32 accumulators are needed here, not a fused store
+    rc = niti_tc_gemm(ctx, st, q, none, acc32, hdr, &fused);
+    ctx->engine = saved;
+    if (rc == NITI_ERR_SHAPE) rc = niti_simt_gemm(ctx, st, q, acc32, hdr);
+    if (rc != NITI_OK) return rc;
+    return niti_launch_round_compact32(ctx, st, acc32, hdr, g, Cout, R * S * Cin, m_u, round_mode, b_g);
+  }
+  return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, g, m_u, round_mode, 0, nullptr,
                         nullptr, nullptr, nullptr, b_g);
 }

@@ -78,6 +78,91 @@ int niti_launch_round(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, const 
 }
 
 // ---------------------------------------------------------------------------------------------
+// Few-channel convolutions (first layer: 1 or 3 input channels, R*S*Cin <= 32): the taps of every
+// output pixel are gathered into one 32-byte row so that the layer becomes a plain K = 32 matrix
+// multiply for the tensor-core engine.  Column k = (r * S + s) * Cin + ci, zero beyond R*S*Cin.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+im2col32_kernel(const int8_t *__restrict__ x, int8_t *__restrict__ xcol, int B, int H, int W, int Ci, int R,
+                int S, int pad, int Ho, int Wo) {
+  const long long M = (long long)B * Ho * Wo;
+  for (long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x; m < M;
+       m += (long long)gridDim.x * blockDim.x) {
+    const int j = (int)(m % Wo);
+    const long long t = m / Wo;
+    const int i = (int)(t % Ho);
+    const long long b = t / Ho;
+    unsigned w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int k = 0;
+    for (int r = 0; r < R; ++r) {
+      const int ii = i + r - pad;
+      for (int q = 0; q < S; ++q) {
+        const int jj = j + q - pad;
+        const bool in = ii >= 0 && ii < H && jj >= 0 && jj < W;
+        const int8_t *src = x + ((b * H + ii) * W + jj) * Ci;
+        for (int c = 0; c < Ci; ++c, ++k) {
+          const unsigned v = in ? (unsigned)(uint8_t)src[c] : 0u;
+          w[k >> 2] |= v << (8 * (k & 3));
+        }
+      }
+    }
+    int4 *dst = reinterpret_cast<int4 *>(xcol + m * 32);
+    dst[0] = make_int4(w[0], w[1], w[2], w[3]);
+    dst[1] = make_int4(w[4], w[5], w[6], w[7]);
+  }
+}
+
+// weights [Cout][R*S*Cin] -> [Cout][32], zero padded
+__global__ void pad_rows32_kernel(const int8_t *__restrict__ w, int8_t *__restrict__ wcol, int rows, int k) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < rows * 32) {
+    const int r = idx >> 5, c = idx & 31;
+    wcol[idx] = c < k ? w[r * k + c] : (int8_t)0;
+  }
+}
+
+// Rounds acc[rows][32] (int32) and keeps the first k columns: out[rows][k].
+__global__ void round_compact32_kernel(const int32_t *__restrict__ acc, const WsHeader *__restrict__ hdr,
+                                       int8_t *__restrict__ out, int rows, int k, int mbits, int round_mode,
+                                       int32_t *__restrict__ b_out) {
+  const int b = niti_bitlen32(hdr->maxabs32);
+  const int bp = b > mbits ? b - mbits : 0;
+  const unsigned qmax = (1u << mbits) - 1u;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx == 0 && b_out) *b_out = b;
+  if (idx < rows * k) {
+    const int r = idx / k, c = idx % k;
+    out[idx] = (int8_t)niti_round_i32(acc[r * 32 + c], bp, qmax, round_mode);
+  }
+}
+
+int niti_launch_im2col32(niti_ctx *ctx, cudaStream_t st, const int8_t *x, int8_t *xcol, int B, int H, int W,
+                         int Ci, int R, int S, int pad, int Ho, int Wo) {
+  long long M = (long long)B * Ho * Wo;
+  long long blocks = (M + 255) / 256;
+  if (blocks > (long long)ctx->sm_count * 16) blocks = (long long)ctx->sm_count * 16;
+  im2col32_kernel<<<(unsigned)blocks, 256, 0, st>>>(x, xcol, B, H, W, Ci, R, S, pad, Ho, Wo);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+int niti_launch_pad_rows32(niti_ctx *ctx, cudaStream_t st, const int8_t *w, int8_t *wcol, int rows, int k) {
+  pad_rows32_kernel<<<(rows * 32 + 255) / 256, 256, 0, st>>>(w, wcol, rows, k);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+int niti_launch_round_compact32(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, const WsHeader *hdr, int8_t *out,
+                                int rows, int k, int mbits, int round_mode, int32_t *b_out) {
+  round_compact32_kernel<<<(rows * k + 255) / 256, 256, 0, st>>>(acc, hdr, out, rows, k, mbits, round_mode, b_out);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Integer cross-entropy gradient, Section 3.5.  Pass 1: one block per sample computes the integer
 // T_i (Eq. 2 or Eq. 3-4), their sum, e32 = T_i - [i == label] * sum (64-bit), the tensor-wide
 // max magnitude, and the arg-max hit count.  Pass 2: shared binary point, rounding to int8.
