@@ -20,7 +20,13 @@ namespace {
 constexpr int BM = 128;               // rows of an output tile = TMEM lanes
 constexpr int EPI_WARPS = 16;          // four per TMEM lane quarter, interleaved 32-column chunks
 constexpr int EPI_PER_Q = EPI_WARPS / 4;
-constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
+// TMA copies are issued by single threads, and one thread sustains only about one copy per
+// 250 ns (measured: four issuing warps give four times the copy rate), so the k-blocks are dealt
+// round-robin to PROD_WARPS producer warps.
+constexpr int PROD_WARPS = 4;          // each stage of the ring belongs to one producer warp (stage % nprod)
+constexpr int MMA_WARP = PROD_WARPS;
+constexpr int EPI_WARP0 = PROD_WARPS + 1;
+constexpr int NUM_THREADS = 32 * (PROD_WARPS + 1 + EPI_WARPS);
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_TBUF = 8;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;
@@ -60,6 +66,8 @@ struct TcParams {
   int blocked;                  // 1: every CTA takes a contiguous range of items (its first tile then
                                 //    samples the tensor evenly), 0: items strided over the grid
   int nbuf;                     // accumulator buffers in tensor memory (2..8)
+  int nprod;                    // producer warps in use; divides `stages` (each stage has one owner, so
+                                // the waits on a stage's barriers stay in order)
   // halo mode (3x3 convolutions with few channels): the weights of all nine taps stay in shared
   // memory for the whole kernel, every tile loads its 8 x 16 pixel patch once with a one-pixel
   // halo (10 x 18 pixels), and the nine taps are nine row offsets into that patch
@@ -393,7 +401,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {
+  if (warp == MMA_WARP) {
     if (CTAS == 2) {
       asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                    ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
@@ -410,8 +418,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   tc_fence_after();
   const unsigned tmem_base = tmem_base_slot;
 
-  if (warp == 0) {
-    // ================= TMA producer (every CTA loads its own rows of A and its share of B) ========
+  if (warp < PROD_WARPS) {
+    // ================= TMA producers (every CTA loads its own rows of A and its share of B) ========
     if (lane == 0) {
       int stage = 0;
       unsigned phase = 0;
@@ -420,8 +428,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (p.halo) {
         // resident weights: one tile per tap, [bn rows][kdepth] K-major (forward) or
         // [kdepth rows][bn] MN-major in b_boxes column chunks (dgrad)
-        mbar_expect_tx(bres_bar, (unsigned)(9 * p.b_boxes * p.b_box_bytes));
-        for (int tap = 0; tap < 9; ++tap) {
+        if (warp == 0) mbar_expect_tx(bres_bar, (unsigned)(9 * p.b_boxes * p.b_box_bytes));
+        for (int tap = 0; warp == 0 && tap < 9; ++tap) {
           const unsigned dst = smem_base + tap * p.b_tile_bytes;
           if (p.kind == GK_CONV_FWD) {
             tma_load_2d(dst, &map_b, bres_bar, tap * p.kdepth, 0);
@@ -434,10 +442,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int wt = (int)(first_item % p.w_tiles), ht = (int)((first_item / p.w_tiles) % p.h_tiles);
         int bt = (int)(first_item / ((long long)p.w_tiles * p.h_tiles));
         for (long long item = first_item; ok && item < item_end; ++item) {
-          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
-          const unsigned full = full0 + 8 * stage;
-          mbar_expect_tx(full, (unsigned)p.a_box_bytes);
-          tma_load_4d(smem_base + p.b_res_bytes + stage * p.a_bytes, &map_a, full, 0, wt * 8 - 1, ht * 16 - 1, bt);
+          if (stage % p.nprod == warp) {
+            if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
+            const unsigned full = full0 + 8 * stage;
+            mbar_expect_tx(full, (unsigned)p.a_box_bytes);
+            tma_load_4d(smem_base + p.b_res_bytes + stage * p.a_bytes, &map_a, full, 0, wt * 8 - 1, ht * 16 - 1, bt);
+          }
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
           if (++wt == p.w_tiles) { wt = 0; if (++ht == p.h_tiles) { ht = 0; ++bt; } }
         }
@@ -473,6 +483,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int wg_r = tap_n / p.S, wg_s = tap_n % p.S;
         const unsigned tx_bytes = (unsigned)(CTAS * (p.a_boxes * p.a_box_bytes + p.b_boxes * p.b_box_bytes));
         for (int kb = kb0; kb < kb1; ++kb) {
+         if (stage % p.nprod == warp) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
           const unsigned full = lead_full0 + 8 * stage;
           const unsigned sa = smem_base + stage * stage_bytes;
@@ -515,6 +526,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               break;
             }
           }
+         }
           if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) {
             if (++cc == p.c_chunks) { cc = 0; if (++ts == p.S) { ts = 0; ++tr; } }
           } else if (p.kind == GK_CONV_WGRAD) {
@@ -524,7 +536,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == MMA_WARP) {
     // ================= MMA issuer (leader CTA only) =================
     if (lane == 0 && rank == 0) {
       int stage = 0;
@@ -614,7 +626,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else {
     // ================= epilogue: TMEM -> int32 accumulators + max magnitude =================
     const int quarter = warp & 3;               // TMEM lanes [32 * quarter, +32)
-    const int chunk_phase = (warp - 2) >> 2;    // this warp takes 32-column chunks phase, phase + EPI_PER_Q, ...
+    const int chunk_phase = (warp - EPI_WARP0) >> 2;    // this warp takes 32-column chunks phase, phase + EPI_PER_Q, ...
     const int row_in_tile = quarter * 32 + lane;
     unsigned use = 0;
     unsigned mx = 0;
@@ -757,7 +769,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (scaled > 0x7fffffffull) scaled = 0x7fffffffull;
           const int b = niti_bitlen32((unsigned)scaled);
           bp = b > p.mbits ? b - p.mbits : 0;
-          if (blockIdx.x == 0 && warp == 2 && lane == 0) hdr->spec_b = (unsigned)b;
+          if (blockIdx.x == 0 && warp == EPI_WARP0 && lane == 0) hdr->spec_b = (unsigned)b;
         }
         int8_t *dst8 = out8 + out_row * p.gn + col0;
         const int8_t *msk = mask8 ? mask8 + out_row * p.gn + col0 : nullptr;
@@ -830,7 +842,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __syncthreads();
   }
   if (CTAS == 2) cluster_sync_all();   // nobody leaves while the peer may still touch this CTA
-  if (warp == 1) {
+  if (warp == MMA_WARP) {
     tc_fence_after();
     if (CTAS == 2)
       asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
@@ -1133,6 +1145,11 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
     p.splits = 1;
     p.kb_per_split = p.kb_total;
   }
+  // producer warps: the largest count <= PROD_WARPS that divides the number of stages
+  if (p.stages == 5 || p.stages == 7) p.stages -= 1;
+  p.nprod = 1;
+  for (int d = 2; d <= PROD_WARPS; ++d)
+    if (p.stages % d == 0) p.nprod = d;
   p.nbuf = 512 / p.bn;
   if (p.nbuf > MAX_TBUF) p.nbuf = MAX_TBUF;
   // convolution outputs are spatially structured (borders, images): contiguous item ranges make the
