@@ -120,6 +120,19 @@ __device__ __forceinline__ bool mbar_try(unsigned bar, unsigned parity) {
       : "memory");
   return ok != 0;
 }
+// Same, but the thread may sleep in hardware for up to `ns` nanoseconds while the phase is pending
+// (it is woken when the phase completes), so a waiting warp does not burn issue slots polling.
+__device__ __forceinline__ bool mbar_try_sleep(unsigned bar, unsigned parity, unsigned ns) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false (and raises the abort flag) if the barrier did not flip in time or
 // another thread already gave up.
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int *abort_flag,
@@ -127,7 +140,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatil
   if (mbar_try(bar, parity)) return true;
   long long t0 = clock64();
   while (true) {
-    if (mbar_try(bar, parity)) return true;
+    if (mbar_try_sleep(bar, parity, 20000u)) return true;
     if (*abort_flag) return false;
     if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
       *abort_flag = 1;
@@ -383,6 +396,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     item_step = 1;
   }
 
+  // epilogue warps with at least one 32-column chunk of the tile (four per chunk phase)
+  const int epi_phases = (p.bn / 32) < EPI_PER_Q ? (p.bn / 32) : EPI_PER_Q;
+  const int epi_active = 4 * epi_phases;
   // TMEM columns: nbuf accumulator buffers of bn columns, rounded up to a power of two >= 32
   unsigned tmem_cols = 32;
   while (tmem_cols < (unsigned)(p.nbuf * p.bn)) tmem_cols <<= 1;
@@ -396,7 +412,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     mbar_init(bres_bar, 1);
     for (int b = 0; b < p.nbuf; ++b) {
       mbar_init(tfull0 + 8 * b, 1);
-      mbar_init(tempty0 + 8 * b, EPI_WARPS * CTAS);     // one arrival per epilogue warp of every CTA
+      mbar_init(tempty0 + 8 * b, epi_active * CTAS);    // one arrival per working epilogue warp of every CTA
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -623,7 +639,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
       }
     }
-  } else {
+  } else if (warp < EPI_WARP0 + epi_active) {
     // ================= epilogue: TMEM -> int32 accumulators + max magnitude =================
     const int quarter = warp & 3;               // TMEM lanes [32 * quarter, +32)
     const int chunk_phase = (warp - EPI_WARP0) >> 2;    // this warp takes 32-column chunks phase, phase + EPI_PER_Q, ...
@@ -747,7 +763,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (m0) atomicMax(&hdr->est_max, m0);
             __threadfence();
             atomicAdd(&hdr->tile_counter, 1u);
-            const unsigned expected = gridDim.x * (unsigned)EPI_WARPS;
+            const unsigned expected = gridDim.x * (unsigned)epi_active;
             long long t0 = clock64();
             while (*(volatile unsigned *)&hdr->tile_counter < expected) {
               if (abort_flag) break;
