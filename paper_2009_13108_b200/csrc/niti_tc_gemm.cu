@@ -71,7 +71,13 @@ struct TcParams {
   // halo mode (3x3 convolutions with few channels): the weights of all nine taps stay in shared
   // memory for the whole kernel, every tile loads its 8 x 16 pixel patch once with a one-pixel
   // halo (10 x 18 pixels), and the nine taps are nine row offsets into that patch
+  // halo == 2: weight gradient of such a convolution for one (64 output channels, 64 input
+  // channels) block.  Per 8 x 16 pixel tile the CTA loads the error tile and the input patch once;
+  // the nine taps are row offsets into the patch, two taps share one MMA (M = 2 x 64 input
+  // channels through the leading-dimension stride of the MN-major descriptor), N = 64 output
+  // channels, and the five accumulators stay in tensor memory over the CTA's whole pixel range.
   int halo;
+  int wg_nci;                   // 64-channel blocks of the input channels
   int b_tile_bytes;             // bytes of one tap's weight tile
   int b_res_bytes;              // bytes of the resident weights (all taps), multiple of 1024
   // epilogue
@@ -397,7 +403,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 
   // epilogue warps with at least one 32-column chunk of the tile (four per chunk phase)
-  const int epi_phases = (p.bn / 32) < EPI_PER_Q ? (p.bn / 32) : EPI_PER_Q;
+  const int epi_phases = (p.halo == 2 || (p.bn / 32) >= EPI_PER_Q) ? EPI_PER_Q : (p.bn / 32);
   const int epi_active = 4 * epi_phases;
   // TMEM columns: nbuf accumulator buffers of bn columns, rounded up to a power of two >= 32
   unsigned tmem_cols = 32;
@@ -441,7 +447,30 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       unsigned phase = 0;
       bool ok = true;
       const int bn_cta = p.bn / CTAS;             // B rows (output columns) staged by this CTA
-      if (p.halo) {
+      if (p.halo == 2) {
+        for (long long item = first_item; ok && item < item_end; item += item_step) {
+          const int split = (int)(item % p.splits);
+          const int blk = (int)(item / p.splits);
+          const int ci0 = (blk % p.wg_nci) * 64, co0 = (blk / p.wg_nci) * 64;
+          const int t0 = split * p.kb_per_split;
+          int t1 = t0 + p.kb_per_split;
+          if (t1 > p.kb_total) t1 = p.kb_total;
+          int wt = t0 % p.w_tiles, ht = (t0 / p.w_tiles) % p.h_tiles, bt = t0 / (p.w_tiles * p.h_tiles);
+          for (int t = t0; t < t1; ++t) {
+            if (stage % p.nprod == warp) {
+              if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
+              const unsigned full = full0 + 8 * stage;
+              const unsigned sa = smem_base + stage * stage_bytes;
+              mbar_expect_tx(full, (unsigned)(p.a_box_bytes + p.b_box_bytes));
+              tma_load_4d(sa, &map_a, full, ci0, wt * 8 - 1, ht * 16 - 1, bt);          // input patch
+              tma_load_4d(sa + p.a_bytes, &map_b, full, co0, wt * 8, ht * 16, bt);     // error tile
+            }
+            if (++stage == p.stages) { stage = 0; phase ^= 1; }
+            if (++wt == p.w_tiles) { wt = 0; if (++ht == p.h_tiles) { ht = 0; ++bt; } }
+          }
+        }
+        item_end = first_item;
+      } else if (p.halo) {
         // resident weights: one tile per tap, [bn rows][kdepth] K-major (forward) or
         // [kdepth rows][bn] MN-major in b_boxes column chunks (dgrad)
         if (warp == 0) mbar_expect_tx(bres_bar, (unsigned)(9 * p.b_boxes * p.b_box_bytes));
@@ -559,7 +588,46 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       unsigned phase = 0;
       unsigned use = 0;                 // tiles processed by this CTA (pair)
       bool ok = true;
-      if (p.halo) {
+      if (p.halo == 2) {
+        // tap pairs (0,1) (2,3) (4,5) (6,7) (8,-): patch row of the first tap and the row distance to
+        // the second one (the leading-dimension stride between the two 64-channel halves of M)
+        const unsigned a_hi = (unsigned)(p.a_desc >> 32), b_hi = (unsigned)(p.b_desc >> 32);
+        const unsigned b_lo0 = (unsigned)p.b_desc;
+        unsigned a_pair[5];
+#pragma unroll
+        for (int pi = 0; pi < 5; ++pi) {
+          const int ta = 2 * pi, tb = 2 * pi + 1 < 9 ? 2 * pi + 1 : 2 * pi - 1;
+          const int ra = (ta / 3) * 10 + ta % 3, rb = (tb / 3) * 10 + tb % 3;
+          const int lbo_rows = rb > ra ? rb - ra : 1;
+          a_pair[pi] = (unsigned)(ra * 4) | ((unsigned)(lbo_rows * 4) << 16);     // 64-byte rows, 16-byte units
+        }
+        for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
+          const int split = (int)(item % p.splits);
+          const int t0 = split * p.kb_per_split;
+          int t1 = t0 + p.kb_per_split;
+          if (t1 > p.kb_total) t1 = p.kb_total;
+          if (!mbar_wait(tempty0, (use & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          for (int t = t0; t < t1; ++t) {
+            if (!mbar_wait(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
+            tc_fence_after();
+            const unsigned sa16 = ((smem_base + stage * stage_bytes) >> 4) & 0x3fff;
+            const unsigned sb16 = ((smem_base + stage * stage_bytes + p.a_bytes) >> 4) & 0x3fff;
+            const unsigned first = t > t0 ? 1u : 0u;
+#pragma unroll
+            for (int pi = 0; pi < 5; ++pi) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j)      // 32 pixels = four rows of eight per MMA
+                tc_mma_i8_lh(tmem_base + 64u * pi, sa16 + a_pair[pi] + 160u * j, a_hi, b_lo0 + sb16 + 128u * j, b_hi,
+                             p.idesc, j > 0 ? 1u : first);
+            }
+            tc_commit(empty0 + 8 * stage);
+            if (++stage == p.stages) { stage = 0; phase ^= 1; }
+          }
+          if (ok) tc_commit(tfull0);
+        }
+        item_end = first_item;
+      } else if (p.halo) {
         ok = mbar_wait(bres_bar, 0, &abort_flag, status);
         // descriptor low words per tap, computed once: the patch row where the tap starts
         // (forward reads x[i + r - 1][j + t - 1], dgrad reads e[i - r + 1][j - t + 1]; the patch
@@ -654,6 +722,33 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bp = b > p.mbits ? b - p.mbits : 0;
     }
     bool ok = true;
+    if (p.halo == 2) {
+      // lane = (tap of the pair, input channel), column = output channel; partial sums of this
+      // CTA's pixel range are added to g32[co][tap][ci]
+      const int which = row_in_tile >> 6, ci = row_in_tile & 63;
+      for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
+        const int blk = (int)(item / p.splits);
+        const int ci0 = (blk % p.wg_nci) * 64, co0 = (blk / p.wg_nci) * 64;
+        if (!mbar_wait(tfull0, use & 1u, &abort_flag, status)) { ok = false; break; }
+        tc_fence_after();
+        for (int job = chunk_phase; job < 10; job += EPI_PER_Q) {
+          const int pi = job >> 1, c0 = (job & 1) * 32;
+          const int tap = 2 * pi + which;
+          int v[32];
+          tc_ld32(tmem_base + ((unsigned)(quarter * 32) << 16) + 64u * pi + (unsigned)c0, v);
+          if (tap < 9) {
+            int32_t *dst = acc + (long long)(co0 + c0) * p.gn + (long long)tap * p.Cn + ci0 + ci;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (v[j] != 0) atomicAdd(dst + (long long)j * p.gn, v[j]);
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty0);
+      }
+      item_end = first_item;
+    }
     for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
       int mu = 0, nt = 0, split = 0;
       if (!p.halo) decode_item(p, item, mu, nt, split);
@@ -1060,6 +1155,58 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
     }
     case GK_CONV_WGRAD: {
       if (g.Ho != g.H || g.Wo != g.W) return false;
+      if (want_halo && ctas == 1 && g.R == 3 && g.S == 3 && g.pad == 1 && g.Ci % 64 == 0 && g.Co % 64 == 0 &&
+          g.W >= 10 && g.H >= 18) {
+        p.halo = 2;
+        p.kdepth = 128;
+        p.bn = 64;
+        p.Wt = 8; p.Ht = 16; p.Bt = 1;
+        p.w_tiles = (g.W + 7) / 8;
+        p.h_tiles = (g.H + 15) / 16;
+        p.b_tiles = g.B;
+        p.PW = g.W; p.PH = g.H; p.PB = g.B;
+        p.Cn = g.Ci;
+        p.wg_nci = g.Ci / 64;
+        p.kb_total = p.w_tiles * p.h_tiles * p.b_tiles;      // pixel tiles
+        // A = input patch (p1 = x), B = error tile (p0 = e); both MN-major, 64-byte rows
+        sa = {4, {(cuuint64_t)g.Ci, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.B},
+              {(cuuint64_t)g.Ci, (cuuint64_t)g.Ci * g.W, (cuuint64_t)g.Ci * g.W * g.H}, {64, 10, 18, 1}, 64, g.p1};
+        sb = {4, {(cuuint64_t)g.Co, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.B},
+              {(cuuint64_t)g.Co, (cuuint64_t)g.Co * g.W, (cuuint64_t)g.Co * g.W * g.H}, {64, 8, 16, 1}, 64, g.p0};
+        p.a_box_bytes = 180 * 64; p.b_box_bytes = 128 * 64;
+        p.a_bytes = 12288; p.b_bytes = 8192;
+        p.a_boxes = p.b_boxes = 1;
+        p.stages = MAX_STAGES;
+        p.nprod = PROD_WARPS;
+        p.nbuf = 5;                                           // five accumulators of 64 columns
+        p.ksteps = 4;
+        // MN-major, 64-byte swizzle: 8-row groups one patch row (10 pixels) apart for A, contiguous for B;
+        // the leading-dimension field of A is filled per tap pair by the kernel
+        p.a_desc = ((unsigned long long)((10 * 64) >> 4) << 32) | ((unsigned long long)1 << 46) | layout_bits(64);
+        p.b_desc = ((unsigned long long)1 << 16) | ((unsigned long long)((8 * 64) >> 4) << 32) |
+                   ((unsigned long long)1 << 46) | layout_bits(64);
+        p.idesc = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((unsigned)(64 >> 3) << 17) |
+                  ((unsigned)(BM >> 4) << 24);
+        const long long blocks = (long long)(g.Ci / 64) * (g.Co / 64);
+        // split the pixel range so that the items fill whole waves of SMs
+        int best_s = 1;
+        double best_eff = 0;
+        const int max_s = p.kb_total / 4 > 0 ? p.kb_total / 4 : 1;
+        for (int sp = 1; sp <= max_s && sp <= 4 * ctx->sm_count; ++sp) {
+          const long long it = blocks * sp;
+          const long long waves = (it + ctx->sm_count - 1) / ctx->sm_count;
+          const double eff = (double)it / (double)(waves * ctx->sm_count);
+          if (eff > best_eff + 0.02) { best_eff = eff; best_s = sp; }
+        }
+        p.splits = best_s;
+        p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
+        p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+        p.items = blocks * p.splits;
+        p.m_units = 1;
+        p.n_tiles_n = 1;
+        if (!encode(ctx, &ma, sa) || !encode(ctx, &mb, sb)) return false;
+        return true;
+      }
       a_mn = b_mn = 1;
       a_sw = pick_swizzle(g.Co);
       b_sw = pick_swizzle(g.Ci);
@@ -1237,7 +1384,8 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
   // Test switches: 2 / 3 force the single-CTA / paired kernel, 4 keeps the int32 spill epilogue.
   // Test switches: 5 disables the halo mode of small-channel convolutions.
   bool planned = false;
-  if ((g.kind == GK_CONV_FWD || g.kind == GK_CONV_DGRAD) && ctx->engine != 3 && ctx->engine != 5)
+  if ((g.kind == GK_CONV_FWD || g.kind == GK_CONV_DGRAD || g.kind == GK_CONV_WGRAD) && ctx->engine != 3 &&
+      ctx->engine != 5)
     planned = plan(ctx, g, 1, true, p, ma, mb) && p.halo;
   if (!planned && ctx->engine != 2 && g.gm >= 2 * BM) {
     planned = plan(ctx, g, 2, false, p, ma, mb);
@@ -1260,7 +1408,7 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
   p.mbits = r.mbits;
   p.round_mode = r.round_mode;
   p.relu = r.relu;
-  p.epi_mode = p.splits > 1 ? EPI_ATOMIC : (ctx->engine == 4 ? EPI_SPILL : EPI_SPECULATE);
+  p.epi_mode = (p.splits > 1 || p.halo == 2) ? EPI_ATOMIC : (ctx->engine == 4 ? EPI_SPILL : EPI_SPECULATE);
   if (p.epi_mode == EPI_ATOMIC) {
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(acc, 0, sizeof(int32_t) * (size_t)(g.gm * g.gn), st));
     ctx->launches++;
