@@ -1155,8 +1155,10 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
     }
     case GK_CONV_WGRAD: {
       if (g.Ho != g.H || g.Wo != g.W) return false;
+      // (64 x 64)-channel blocks re-read the activations once per block of the other operand, so this
+      // mode is kept for layers with few blocks; wide layers use the per-tap tiles below
       if (want_halo && ctas == 1 && g.R == 3 && g.S == 3 && g.pad == 1 && g.Ci % 64 == 0 && g.Co % 64 == 0 &&
-          g.W >= 10 && g.H >= 18) {
+          g.W >= 10 && g.H >= 18 && (long long)g.Ci * g.Co <= 65536) {
         p.halo = 2;
         p.kdepth = 128;
         p.bn = 64;
