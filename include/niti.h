@@ -51,6 +51,7 @@ extern "C" {
 #define NITI_ERR_RANGE 4     /* exponent outside the supported domain              */
 #define NITI_ERR_CUDA 5      /* a CUDA call failed; see niti_last_error()          */
 #define NITI_ERR_DEVICE 6    /* a kernel raised the device status word             */
+#define NITI_ERR_TOO_LARGE 8 /* beyond the fixed capacity of a no-allocation variant */
 
 #define NITI_ROUND_PSR 0
 #define NITI_ROUND_NEAREST 1
@@ -184,6 +185,30 @@ int niti_conv_wgrad(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *
 int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const int32_t *s_a,
                   const int32_t *labels, int8_t *e, int32_t *b_e, int32_t *n_correct, int B, int N,
                   int round_mode, void *ws, size_t ws_bytes);
+
+/* Integer cross-entropy gradient for callers that must not allocate device memory (the paper has
+ * no counterpart: this is a packaging variant of niti_int_xent, same arithmetic, same outputs).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a latency-critical training loop
+ * that forbids allocator calls after start-up, a host process that has already handed all device
+ * memory to its own pool, or a plug-in that is given tensors and a stream but no allocator.  Such
+ * a caller cannot create a context (niti_create allocates the status word) nor a workspace, so
+ * this call takes neither: its scratch (256 bytes of reduction scalars + 8 bytes per logit) lives
+ * in a fixed array inside the library image, NITI_XENT_NOALLOC_MAX_ELEMS logits at most
+ * (B * N <= 65536, i.e. 512 KiB + 256 B that every GPU loading the library holds until exit).
+ * Larger B * N returns NITI_ERR_TOO_LARGE and enqueues nothing.
+ *
+ * a, labels, e, s_a, b_e, n_correct: device pointers as in niti_int_xent (b_e, n_correct may be
+ * NULL); `stream` is the caller's cudaStream_t.  The call allocates nothing and frees nothing.  The
+ * first call on each device looks up the array's device address (with the current device); make
+ * that first call before any stream capture begins.  All calls on a device share the one array,
+ * which keeps the previous call's contents: the call clears the scalars it needs itself, but two
+ * calls that can overlap on the GPU (different streams without ordering) race on it.  There is
+ * no status word in this variant: an exponent outside [-22, 24] or a label outside [0, N) yields
+ * zeros for the affected rows. */
+#define NITI_XENT_NOALLOC_MAX_ELEMS 65536
+int niti_int_xent_noalloc(void *stream, const int8_t *a, const int32_t *s_a, const int32_t *labels,
+                          int8_t *e, int32_t *b_e, int32_t *n_correct, int B, int N, int round_mode);
 
 /* Weight update (Algorithm 1 last line; Section 3.3): w <- clamp(w - g, -127, 127), in place. */
 int niti_int_sgd_update(niti_ctx *ctx, void *stream, int8_t *w, const int8_t *g, int64_t n);

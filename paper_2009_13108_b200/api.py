@@ -22,7 +22,8 @@ EXPORTS = [
     "niti_set_engine", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
     "niti_redo_count", "niti_profile_enable", "niti_profile_read_launches",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
-    "niti_conv_dgrad", "niti_conv_wgrad", "niti_int_xent", "niti_int_sgd_update", "niti_relu_fwd",
+    "niti_conv_dgrad", "niti_conv_wgrad", "niti_int_xent", "niti_int_xent_noalloc", "niti_int_sgd_update",
+    "niti_relu_fwd",
     "niti_relu_bwd", "niti_maxpool2_fwd", "niti_maxpool2_bwd",
 ]
 
@@ -70,6 +71,7 @@ def load_library():
     lib.niti_conv_dgrad.argtypes = [vp, vp, vp, vp, vp, vp, vp] + [i32] * 9 + [vp, sz]
     lib.niti_conv_wgrad.argtypes = [vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
     lib.niti_int_xent.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, sz]
+    lib.niti_int_xent_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32]
     lib.niti_int_sgd_update.argtypes = [vp, vp, vp, vp, i64]
     lib.niti_relu_fwd.argtypes = [vp, vp, vp, vp, i64]
     lib.niti_relu_bwd.argtypes = [vp, vp, vp, vp, vp, i64]
@@ -254,6 +256,14 @@ class Niti:
                                         _ptr(e), _ptr(b_e), _ptr(n_correct), B, N, round_mode, ws,
                                         wsb))
         return e, b_e, n_correct
+
+    def int_xent_noalloc(self, a, s_a, labels, e, b_e=None, n_correct=None, round_mode=ROUND_PSR):
+        """niti_int_xent_noalloc: the caller passes every buffer (this wrapper allocates nothing
+        either); no context, no workspace.  Returns the library's return code."""
+        B, N = a.shape
+        return int(self.lib.niti_int_xent_noalloc(self._stream(), _ptr(a), _ptr(s_a), _ptr(labels),
+                                                  _ptr(e), _ptr(b_e), _ptr(n_correct), B, N,
+                                                  round_mode))
 
     def int_sgd_update(self, w, g):
         self._ck(self.lib.niti_int_sgd_update(self.h, self._stream(), _ptr(w), _ptr(g), w.numel()))

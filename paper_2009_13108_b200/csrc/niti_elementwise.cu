@@ -1,6 +1,7 @@
 // HBM-bound kernels of the NITI library: the shift-and-round pass (Algorithm 2/3), the integer
 // cross-entropy gradient (Section 3.5), the weight update (Algorithm 1) and the int8 support ops.
 #include "niti_common.cuh"
+#include <mutex>
 
 // ---------------------------------------------------------------------------------------------
 // Shift-and-round pass over an int32 accumulator tensor (Algorithm 2, with Algorithm 3 rounding).
@@ -302,6 +303,52 @@ extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const
   round_i64_kernel<<<(unsigned)blocks, 256, 0, st>>>(e64, hdr, e, n, round_mode, b_e);
   ctx->launches++;
   NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// niti_int_xent_noalloc: the same two kernels with their scratch (reduction header + 64-bit loss
+// accumulators) in a fixed device array that is part of the library image, for callers that must
+// not allocate device memory.  Every GPU that loads the library carries the array until exit.
+// ---------------------------------------------------------------------------------------------
+#define NITI_NOALLOC_BYTES (NITI_WS_HEADER + 8 * NITI_XENT_NOALLOC_MAX_ELEMS)
+static __device__ __align__(256) unsigned char g_xent_scratch[NITI_NOALLOC_BYTES];
+// The name above is only a host-side handle in host code; the device address is looked up once per
+// device (with that device current) and cached here.
+static void *g_xent_scratch_addr[64];
+static std::mutex g_xent_scratch_mutex;
+
+extern "C" int niti_int_xent_noalloc(void *stream, const int8_t *a, const int32_t *s_a, const int32_t *labels,
+                                     int8_t *e, int32_t *b_e, int32_t *n_correct, int B, int N, int round_mode) {
+  if (!a || !s_a || !labels || !e || B <= 0 || N <= 0 || N > 65536 || (round_mode != 0 && round_mode != 1))
+    return NITI_ERR_ARG;
+  if ((long long)B * N > NITI_XENT_NOALLOC_MAX_ELEMS) return NITI_ERR_TOO_LARGE;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NITI_ERR_CUDA;
+  void *base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_xent_scratch_mutex);
+    if (!g_xent_scratch_addr[dev]) {
+      void *ptr = nullptr;
+      if (cudaGetSymbolAddress(&ptr, g_xent_scratch) != cudaSuccess || !ptr) return NITI_ERR_CUDA;
+      g_xent_scratch_addr[dev] = ptr;
+    }
+    base = g_xent_scratch_addr[dev];
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  WsHeader *hdr = (WsHeader *)base;
+  long long *e64 = (long long *)((char *)base + NITI_WS_HEADER);
+  // the array keeps what the previous call left: the reduction scalars must start at zero.  The last
+  // word of the header takes the (unreported) status bits of this variant.
+  uint32_t *status = (uint32_t *)((char *)base + NITI_WS_HEADER - sizeof(uint32_t));
+  if (cudaMemsetAsync(base, 0, NITI_WS_HEADER, st) != cudaSuccess) return NITI_ERR_CUDA;
+  if (n_correct && cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st) != cudaSuccess) return NITI_ERR_CUDA;
+  xent_acc_kernel<<<B, 256, 0, st>>>(a, s_a, labels, e64, hdr, n_correct, N, status);
+  const long long n = (long long)B * N;
+  long long blocks = (n + 255) / 256;
+  if (blocks > 1024) blocks = 1024;
+  round_i64_kernel<<<(unsigned)blocks, 256, 0, st>>>(e64, hdr, e, n, round_mode, b_e);
+  if (cudaGetLastError() != cudaSuccess) return NITI_ERR_CUDA;
   return NITI_OK;
 }
 
