@@ -1299,10 +1299,19 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
     p.raster_g = ctas == 2 ? 8 : 12;
   // split the contraction when the tiles alone cannot fill the SMs
   if (tiles < units && p.kb_total >= 8) {
-    long long s = (units + tiles - 1) / tiles;
-    if (s > p.kb_total / 4) s = p.kb_total / 4;
-    if (s < 1) s = 1;
-    p.splits = (int)s;
+    // pick the split count with the least modelled time: waves of items, each item running its
+    // share of the k-blocks plus a fixed cost (pipeline fill and the atomic epilogue) of about
+    // four k-blocks
+    double best = 1e30;
+    int best_s = 1;
+    const int max_s = p.kb_total / 4;
+    for (int sp = 1; sp <= max_s && sp <= 4 * units; ++sp) {
+      const long long it = tiles * sp;
+      const long long waves = (it + units - 1) / units;
+      const double cost = (double)waves * ((double)((p.kb_total + sp - 1) / sp) + 4.0);
+      if (cost < best * 0.98) { best = cost; best_s = sp; }
+    }
+    p.splits = best_s;
   }
   p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
   p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
