@@ -149,29 +149,67 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-def gemm_point(niti, M, N, K, iters=10):
-    """Fused int8 GEMM (multiply + bit-width + shift + pseudo-stochastic round) at one shape."""
+def gemm_point(niti, M, N, K, iters=10, dist="uniform", variant="act"):
+    """Fused int8 GEMM (multiply + bit-width + shift + pseudo-stochastic round) at one shape.
+    variant "act": out[M,N] = a[M,K] w[N,K]^T rounded to 7 bits (forward entry point);
+    variant "grad": g[M,N] = e[K,M]^T a[K,N] rounded to 5 bits (weight-gradient entry point)."""
     import torch
-    from synth import gemm_operands
-    a, w = gemm_operands(M, N, K)
-    a, w = torch.from_numpy(a).to(niti.device), torch.from_numpy(w).to(niti.device)
-    sa, sw = niti.scalar(-7), niti.scalar(-10)
-    out = torch.empty((M, N), dtype=torch.int8, device=niti.device)
+    from synth import gemm_grad_operands, gemm_operands
+    dev = niti.device
+    if variant == "act":
+        a, w = gemm_operands(M, N, K, dist)
+        a, w = torch.from_numpy(a).to(dev), torch.from_numpy(w).to(dev)
+        sa, sw = niti.scalar(-7), niti.scalar(-10)
+        out = torch.empty((M, N), dtype=torch.int8, device=dev)
+
+        def run():
+            niti.linear_fwd(a, sa, w, sw, out=out)
+    else:
+        e, a2 = gemm_grad_operands(M, N, K, dist)
+        e, a2 = torch.from_numpy(e).to(dev), torch.from_numpy(a2).to(dev)
+        wdummy = torch.zeros((16,), dtype=torch.int8, device=dev)
+        g = torch.empty((M, N), dtype=torch.int8, device=dev)
+        b_g = niti.scalar()
+
+        def run():
+            niti.linear_bwd(a2, e, wdummy, need_e_prev=False, g=g, b_g=b_g, m_u=5)
     for _ in range(3):
-        niti.linear_fwd(a, sa, w, sw, out=out)
+        run()
     torch.cuda.synchronize()
     niti.profile_enable(True)
     e0, e1 = torch.cuda.Event(True), torch.cuda.Event(True)
     e0.record()
     for _ in range(iters):
-        niti.linear_fwd(a, sa, w, sw, out=out)
+        run()
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / iters
     k_ms, k_n, k_ops = niti.profile_read()
     niti.profile_enable(False)
-    return {"shape": [M, N, K], "fused_ms": ms, "fused_tops": 2.0 * M * N * K / ms / 1e9,
+    pk = _peaks()
+    tops = 2.0 * M * N * K / ms / 1e9
+    return {"shape": [M, N, K], "dist": dist, "variant": variant, "fused_ms": ms, "fused_tops": tops,
+            "frac_of_2x_bf16_burst": tops / (2.0 * pk["bf16_burst"]), "frac_of_nominal_4500": tops / 4500.0,
             "mma_kernel_ms": k_ms / max(k_n, 1), "mma_kernel_tops": k_ops / max(k_ms, 1e-9) / 1e9}
+
+
+def run_sweep(args):
+    """Config 1: the 64-shape fused-GEMM sweep, two operand distributions, two rounding targets."""
+    from paper_2009_13108_b200 import Niti
+    from synth import GEMM_SWEEP_DIMS
+    niti = Niti(0)
+    dims = GEMM_SWEEP_DIMS
+    for dist in ("uniform", "gauss"):
+        for variant in ("act", "grad"):
+            for M in dims:
+                for N in dims:
+                    for K in dims:
+                        if dist == "gauss" and min(M, N, K) < 4096 and not args.full_sweep:
+                            continue          # the second operand set is timed on the large shapes
+                        r = gemm_point(niti, M, N, K, iters=5, dist=dist, variant=variant)
+                        print(json.dumps(r), flush=True)
+    print(json.dumps({"redo_passes": niti.redo_count()}), flush=True)
+    niti.check()
 
 
 def run_ours(args):
@@ -221,6 +259,7 @@ def run_ours(args):
     barrier()
     sampler.start()
     l0 = niti.launch_count()
+    redo0 = niti.redo_count()
     e0, e1 = torch.cuda.Event(True), torch.cuda.Event(True)
     e0.record()
     for _ in range(args.steps):
@@ -230,6 +269,7 @@ def run_ours(args):
     clocks = sampler.stop()
     ms = e0.elapsed_time(e1)
     launches = niti.launch_count() - l0
+    redo = niti.redo_count() - redo0
     k_ms, k_n, k_ops = niti.profile_read()
     niti.profile_enable(False)
     # ---- end to end: host batch in, hit count out, every step ----
@@ -277,6 +317,7 @@ def run_ours(args):
         "e2e": {"value": images / (ms_e2e / 1e3), "unit": UNIT, "h2d_bytes_per_step": int(xh.numel() + lh.numel() * 4),
                 "d2h_bytes_per_step": 4},
         "gpu_launches": int(launches),
+        "speculation_redo_passes": int(redo),
         "roofline": {"bound": "tensor", "kernel": "tc_gemm_kernel (tcgen05 kind::i8)", "achieved": achieved,
                      "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
                      "peak_source": "2 x %s bf16 sustained (int8 : bf16 = 2 : 1 nominal); nominal int8 4500" % pk["source"],
@@ -301,7 +342,12 @@ def main():
     ap.add_argument("--gemm-shape", default=None,
                     help="MxNxK: time only the fused GEMM at this shape (for profiling a small case)")
     ap.add_argument("--iters", type=int, default=10)
+    ap.add_argument("--sweep", action="store_true", help="run the fused-GEMM sweep (config 1), one JSON line per point")
+    ap.add_argument("--full-sweep", action="store_true", help="with --sweep: time the second operand set on every shape")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.gemm_shape:
         from paper_2009_13108_b200 import Niti
         niti = Niti(0)
