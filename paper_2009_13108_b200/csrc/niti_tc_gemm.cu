@@ -66,6 +66,7 @@ struct TcParams {
   int blocked;                  // 1: every CTA takes a contiguous range of items (its first tile then
                                 //    samples the tensor evenly), 0: items strided over the grid
   int nbuf;                     // accumulator buffers in tensor memory (2..8)
+  int egroups;                  // epilogue warp groups (1, 2 or 4); tile `use` belongs to group use % egroups
   int nprod;                    // producer warps in use; divides `stages` (each stage has one owner, so
                                 // the waits on a stage's barriers stay in order)
   // halo mode (3x3 convolutions with few channels): the weights of all nine taps stay in shared
@@ -379,6 +380,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ __align__(8) unsigned long long bars[2 * MAX_STAGES + 2 * MAX_TBUF + 1];
   __shared__ unsigned tmem_base_slot;
   __shared__ volatile int abort_flag;
+  __shared__ volatile int spec_bp_ready;      // 0: not yet; else the speculative binary point + 1
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const unsigned rank = CTAS == 2 ? cluster_ctarank() : 0u;
@@ -403,14 +405,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 
   // epilogue warps with at least one 32-column chunk of the tile (four per chunk phase)
-  const int epi_phases = (p.halo == 2 || (p.bn / 32) >= EPI_PER_Q) ? EPI_PER_Q : (p.bn / 32);
-  const int epi_active = 4 * epi_phases;
+  // The 16 epilogue warps are split into `egroups` groups that drain different tiles at the same
+  // time (narrow tiles have too few 32-column chunks to keep every warp busy on one tile).  Inside a
+  // group each TMEM lane quarter has wpq warps that interleave the tile's chunks.
+  const int egroups = p.halo == 2 ? 1 : p.egroups;
+  const int wpq = EPI_PER_Q / egroups;                       // warps per quarter per tile
+  const int chunks_all = p.bn / 32;
+  const int wpq_active = p.halo == 2 ? EPI_PER_Q : (chunks_all < wpq ? chunks_all : wpq);
+  const int epi_active = 4 * wpq_active;                     // warps that drain one tile
   // TMEM columns: nbuf accumulator buffers of bn columns, rounded up to a power of two >= 32
   unsigned tmem_cols = 32;
   while (tmem_cols < (unsigned)(p.nbuf * p.bn)) tmem_cols <<= 1;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
+    spec_bp_ready = 0;
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
@@ -707,10 +716,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
       }
     }
-  } else if (warp < EPI_WARP0 + epi_active) {
+  } else if (((warp - EPI_WARP0) >> 2) % wpq < wpq_active) {
     // ================= epilogue: TMEM -> int32 accumulators + max magnitude =================
     const int quarter = warp & 3;               // TMEM lanes [32 * quarter, +32)
-    const int chunk_phase = (warp - EPI_WARP0) >> 2;    // this warp takes 32-column chunks phase, phase + EPI_PER_Q, ...
+    const int wq = (warp - EPI_WARP0) >> 2;     // index among the four warps of this quarter
+    const int egroup = wq / wpq;                // tiles use % egroups == egroup are this warp's
+    const int chunk_phase = wq % wpq;           // it takes 32-column chunks phase, phase + wpq, ...
     const int row_in_tile = quarter * 32 + lane;
     unsigned use = 0;
     unsigned mx = 0;
@@ -731,7 +742,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int ci0 = (blk % p.wg_nci) * 64, co0 = (blk / p.wg_nci) * 64;
         if (!mbar_wait(tfull0, use & 1u, &abort_flag, status)) { ok = false; break; }
         tc_fence_after();
-        for (int job = chunk_phase; job < 10; job += EPI_PER_Q) {
+        for (int job = chunk_phase; job < 10; job += wpq) {
           const int pi = job >> 1, c0 = (job & 1) * 32;
           const int tap = 2 * pi + which;
           int v[32];
@@ -749,7 +760,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       item_end = first_item;
     }
-    for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
+    use = (unsigned)egroup;
+    for (long long item = first_item + egroup * item_step; ok && item < item_end;
+         item += item_step * egroups, use += (unsigned)egroups) {
       int mu = 0, nt = 0, split = 0;
       if (!p.halo) decode_item(p, item, mu, nt, split);
       const int mt = mu * CTAS + (int)rank;
@@ -761,17 +774,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int ncols_valid;
       if (p.halo) {
         // 8 x 16 pixel tiles of one image, visited in order: coordinates are stepped, not divided
-        if (use == 0) {
-          h_wt = (int)(first_item % p.w_tiles);
-          h_ht = (int)((first_item / p.w_tiles) % p.h_tiles);
-          h_bt = (int)(first_item / ((long long)p.w_tiles * p.h_tiles));
+        if (use == (unsigned)egroup) {
+          h_wt = (int)(item % p.w_tiles);
+          h_ht = (int)((item / p.w_tiles) % p.h_tiles);
+          h_bt = (int)(item / ((long long)p.w_tiles * p.h_tiles));
         }
         const int w = h_wt * 8 + (row_in_tile & 7), h = h_ht * 16 + (row_in_tile >> 3);
         row_ok = w < p.PW && h < p.PH;
         out_row = ((long long)h_bt * p.PH + h) * p.PW + w;
         col0 = 0;
         ncols_valid = (int)p.gn;
-        if (++h_wt == p.w_tiles) { h_wt = 0; if (++h_ht == p.h_tiles) { h_ht = 0; ++h_bt; } }
+        for (int st = 0; st < egroups; ++st)
+          if (++h_wt == p.w_tiles) { h_wt = 0; if (++h_ht == p.h_tiles) { h_ht = 0; ++h_bt; } }
       } else if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) {
         int w0, h0, b0;
         pixel_box(p, mt, w0, h0, b0);
@@ -803,7 +817,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (p.epi_mode <= EPI_ATOMIC) {
         int32_t *dst = acc + out_row * p.gn + col0;
         const bool vec_ok = ((p.gn & 3) == 0) && ((col0 & 3) == 0);
-        for (int c = 32 * chunk_phase; c < p.bn; c += 32 * EPI_PER_Q) {
+        for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
           int v[32];
           tc_ld32(tm_row + (unsigned)c, v);
           if (row_ok && c < ncols_valid) {
@@ -835,10 +849,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
       } else {
+        if (p.epi_mode == EPI_SPECULATE && use == (unsigned)egroup && egroup != 0) {
+          // the group that drains this CTA's first tile publishes the shift through shared memory
+          long long t0 = clock64();
+          while (spec_bp_ready == 0) {
+            if (abort_flag) break;
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+              abort_flag = 1;
+              atomicOr(status, NITI_DEV_TIMEOUT);
+              break;
+            }
+          }
+          if (abort_flag) { ok = false; break; }
+          bp = spec_bp_ready - 1;
+        }
         if (p.epi_mode == EPI_SPECULATE && use == 0) {
           // first tile of this CTA: max only, then agree on the estimate with the whole grid
           unsigned m0 = 0;
-          for (int c = 32 * chunk_phase; c < p.bn; c += 32 * EPI_PER_Q) {
+          for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
             int v[32];
             tc_ld32(tm_row + (unsigned)c, v);
             if (row_ok) {
@@ -881,12 +909,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int b = niti_bitlen32((unsigned)scaled);
           bp = b > p.mbits ? b - p.mbits : 0;
           if (blockIdx.x == 0 && warp == EPI_WARP0 && lane == 0) hdr->spec_b = (unsigned)b;
+          if (lane == 0) spec_bp_ready = bp + 1;
         }
         int8_t *dst8 = out8 + out_row * p.gn + col0;
         const int8_t *msk = mask8 ? mask8 + out_row * p.gn + col0 : nullptr;
         const bool vec_ok = ((p.gn & 15) == 0) && ((col0 & 15) == 0);
         const RoundConst rk = make_round_const(bp, p.mbits, p.round_mode);
-        for (int c = 32 * chunk_phase; c < p.bn; c += 32 * EPI_PER_Q) {
+        for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
           int v[32];
           tc_ld32(tm_row + (unsigned)c, v);
           if (row_ok && c < ncols_valid) {
@@ -1326,6 +1355,11 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
     if (p.stages % d == 0) p.nprod = d;
   p.nbuf = 512 / p.bn;
   if (p.nbuf > MAX_TBUF) p.nbuf = MAX_TBUF;
+  // epilogue groups: as many as leave no warp without a chunk and one spare accumulator buffer
+  p.egroups = 1;
+  for (int gq = 2; gq <= 4; gq *= 2)
+    if (EPI_PER_Q / gq <= p.bn / 32 && p.nbuf >= gq + 1) p.egroups = gq;
+  p.nbuf = p.nbuf / p.egroups * p.egroups;     // a buffer always returns to the same group
   // convolution outputs are spatially structured (borders, images): contiguous item ranges make the
   // first tile of every CTA an even sample of the tensor for the speculative shift
   p.blocked = (g.kind == GK_CONV_FWD || g.kind == GK_CONV_DGRAD) ? 1 : 0;
