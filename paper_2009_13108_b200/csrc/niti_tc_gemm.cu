@@ -917,6 +917,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const RoundConst rk = make_round_const(bp, p.mbits, p.round_mode);
         for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
           int v[32];
+          // the ReLU mask bytes are fetched first so that their latency overlaps the TMEM load and
+          // the rounding arithmetic
+          int4 m0v = make_int4(0x01010101, 0x01010101, 0x01010101, 0x01010101), m1v = m0v;
+          if (msk && vec_ok && row_ok && c + 32 <= ncols_valid) {
+            m0v = *reinterpret_cast<const int4 *>(msk + c);
+            m1v = *reinterpret_cast<const int4 *>(msk + c + 16);
+          }
           tc_ld32(tm_row + (unsigned)c, v);
           if (row_ok && c < ncols_valid) {
             unsigned w8[8];
@@ -933,8 +940,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (vec_ok && c + 32 <= ncols_valid) {
               mx |= orv;
               if (msk) {
-                const int4 m0v = *reinterpret_cast<const int4 *>(msk + c);
-                const int4 m1v = *reinterpret_cast<const int4 *>(msk + c + 16);
                 w8[0] &= __vcmpgts4(m0v.x, 0); w8[1] &= __vcmpgts4(m0v.y, 0);
                 w8[2] &= __vcmpgts4(m0v.z, 0); w8[3] &= __vcmpgts4(m0v.w, 0);
                 w8[4] &= __vcmpgts4(m1v.x, 0); w8[5] &= __vcmpgts4(m1v.y, 0);
