@@ -212,6 +212,46 @@ def run_sweep(args):
     niti.check()
 
 
+def run_paper_table(args):
+    """The layer of the paper's convolution timing table (batch 64, 64 -> 128 channels, 3x3, stride 1,
+    pad 1, square inputs 224 ... 14): forward, dgrad and wgrad including bit-width, shift and rounding."""
+    import numpy as np
+    import torch
+    from paper_2009_13108_b200 import Niti
+    niti = Niti(0)
+    dev = niti.device
+    rng = np.random.Generator(np.random.PCG64(11))
+    paper_3090_ms = {224: (3.928, 4.731, 122.301), 112: (1.006, 1.269, 27.327), 56: (0.289, 0.453, 6.911),
+                     28: (0.089, 0.185, 1.074), 14: (0.038, 0.117, 0.272)}
+    for side in (224, 112, 56, 28, 14):
+        B, Ci, Co = 64, 64, 128
+        x = torch.from_numpy(rng.integers(-127, 128, size=(B, side, side, Ci), dtype=np.int8)).to(dev)
+        w = torch.from_numpy(rng.integers(-127, 128, size=(Co, 3, 3, Ci), dtype=np.int8)).to(dev)
+        e = torch.from_numpy(rng.integers(-127, 128, size=(B, side, side, Co), dtype=np.int8)).to(dev)
+        y, ep, g = torch.empty_like(e), torch.empty_like(x), torch.empty_like(w)
+        sx, sw = niti.scalar(-7), niti.scalar(-10)
+        ops = 2.0 * B * side * side * Ci * Co * 9
+        row = {"input": side, "batch": B, "cin": Ci, "cout": Co, "int8_ops": ops,
+               "paper_rtx3090_ms": dict(zip(("a", "e", "g"), paper_3090_ms[side]))}
+        for name, fn in (("a", lambda: niti.conv_fwd(x, sx, w, sw, y=y)),
+                         ("e", lambda: niti.conv_dgrad(e, w, (side, side), e_prev=ep)),
+                         ("g", lambda: niti.conv_wgrad(x, e, g=g))):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(True), torch.cuda.Event(True)
+            e0.record()
+            for _ in range(args.iters):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / args.iters
+            row[name + "_ms"] = ms
+            row[name + "_tops"] = ops / ms / 1e9
+        print(json.dumps(row), flush=True)
+    niti.check()
+
+
 def run_ours(args):
     import torch
     rank = int(os.environ.get("RANK", "0"))
@@ -343,10 +383,15 @@ def main():
                     help="MxNxK: time only the fused GEMM at this shape (for profiling a small case)")
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--sweep", action="store_true", help="run the fused-GEMM sweep (config 1), one JSON line per point")
+    ap.add_argument("--paper-table", action="store_true",
+                    help="time the conv layer of the paper's timing table (fwd / dgrad / wgrad, five input sizes)")
     ap.add_argument("--full-sweep", action="store_true", help="with --sweep: time the second operand set on every shape")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.paper_table:
+        run_paper_table(args)
         return
     if args.gemm_shape:
         from paper_2009_13108_b200 import Niti
