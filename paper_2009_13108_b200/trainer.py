@@ -67,6 +67,22 @@ class NitiTrainer:
         for w, w0 in zip(self.weights, self._initial):
             w.copy_(w0, non_blocking=True)
 
+    def capture(self, with_reset: bool = False):
+        """Captures one step (optionally preceded by reset_weights) into a CUDA graph; returns a
+        callable that replays it on the current stream.  Run at least one eager step first: the
+        library sizes its kernel attributes on first use, which must happen outside a capture."""
+        stream = torch.cuda.Stream(device=self.n.device)
+        stream.wait_stream(torch.cuda.current_stream(self.n.device))
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(graph, stream=stream):
+                if with_reset:
+                    self.reset_weights()
+                self.step()
+        torch.cuda.current_stream(self.n.device).wait_stream(stream)
+        self._graph = graph
+        return graph.replay
+
     def load_batch(self, x, labels):
         """Copies one batch (host or device tensors) into the resident input buffers."""
         self.x.copy_(torch.as_tensor(x).reshape(self.x.shape), non_blocking=True)
