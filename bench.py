@@ -252,6 +252,62 @@ def run_paper_table(args):
     niti.check()
 
 
+def run_elementwise(args):
+    """HBM-bound kernels at sizes well beyond the 126 MB L2: achieved GB/s = algorithmic bytes / time."""
+    import numpy as np
+    import torch
+    from paper_2009_13108_b200 import Niti
+    niti = Niti(0)
+    dev = niti.device
+    pk = _peaks()
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(5)
+
+    def rnd(shape, lo=-127, hi=128):
+        return torch.randint(lo, hi, shape, dtype=torch.int8, device=dev, generator=gen)
+
+    def timeit(fn, iters=args.iters):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(True), torch.cuda.Event(True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    n = 1 << 29                                   # 512 Mi elements
+    w, g = rnd((n,)), rnd((n,), -31, 32)
+    x = rnd((n,))
+    y = torch.empty_like(x)
+    B, H, W, C = 64, 224, 224, 64                  # the first pooled activation of the VGG-16 stack
+    px = rnd((B, H, W, C), 0, 128)
+    py = torch.empty((B, H // 2, W // 2, C), dtype=torch.int8, device=dev)
+    pe = rnd((B, H // 2, W // 2, C))
+    pex = torch.empty_like(px)
+    logits = rnd((65536, 1000))
+    labels = torch.randint(0, 1000, (65536,), dtype=torch.int32, device=dev, generator=gen)
+    le = torch.empty_like(logits)
+    s_a = niti.scalar(-4)
+    cases = [
+        ("niti_int_sgd_update", lambda: niti.int_sgd_update(w, g), 3.0 * n),
+        ("niti_relu_fwd", lambda: niti.relu_fwd(x, y), 2.0 * n),
+        ("niti_relu_bwd", lambda: niti.relu_bwd(x, g, y), 3.0 * n),
+        ("niti_maxpool2_fwd", lambda: niti.maxpool2_fwd(px, py), 1.25 * px.numel()),
+        ("niti_maxpool2_bwd", lambda: niti.maxpool2_bwd(px, pe, pex, relu=True), 2.25 * px.numel()),
+        ("niti_int_xent", lambda: niti.int_xent(logits, s_a, labels, e=le), 2.0 * logits.numel() + 4.0 * 65536),
+    ]
+    for name, fn, nbytes in cases:
+        ms = timeit(fn)
+        gbs = nbytes / ms / 1e6
+        print(json.dumps({"kernel": name, "algorithmic_bytes": nbytes, "ms": ms, "GB/s": gbs,
+                          "frac_of_measured_hbm": gbs / pk["hbm_gbs"], "hbm_peak_GB/s": pk["hbm_gbs"],
+                          "peak_source": pk["source"]}), flush=True)
+    niti.check()
+
+
 def run_ours(args):
     import torch
     rank = int(os.environ.get("RANK", "0"))
@@ -409,6 +465,7 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="run the fused-GEMM sweep (config 1), one JSON line per point")
     ap.add_argument("--paper-table", action="store_true",
                     help="time the conv layer of the paper's timing table (fwd / dgrad / wgrad, five input sizes)")
+    ap.add_argument("--elementwise", action="store_true", help="achieved GB/s of the HBM-bound kernels")
     ap.add_argument("--full-sweep", action="store_true", help="with --sweep: time the second operand set on every shape")
     args = ap.parse_args()
     if args.sweep:
@@ -416,6 +473,9 @@ def main():
         return
     if args.paper_table:
         run_paper_table(args)
+        return
+    if args.elementwise:
+        run_elementwise(args)
         return
     if args.gemm_shape:
         from paper_2009_13108_b200 import Niti

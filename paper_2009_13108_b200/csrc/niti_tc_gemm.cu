@@ -23,7 +23,7 @@ constexpr int EPI_PER_Q = EPI_WARPS / 4;
 // TMA copies are issued by single threads, and one thread sustains only about one copy per
 // 250 ns (measured: four issuing warps give four times the copy rate), so the k-blocks are dealt
 // round-robin to PROD_WARPS producer warps.
-constexpr int PROD_WARPS = 4;          // each stage of the ring belongs to one producer warp (stage % nprod)
+constexpr int PROD_WARPS = 3;          // each stage of the ring belongs to one producer warp (stage % nprod)
 constexpr int MMA_WARP = PROD_WARPS;
 constexpr int EPI_WARP0 = PROD_WARPS + 1;
 constexpr int NUM_THREADS = 32 * (PROD_WARPS + 1 + EPI_WARPS);
@@ -643,14 +643,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // starts one pixel up and left of the tile) and the tap's resident weight tile
         const unsigned a_hi = (unsigned)(p.a_desc >> 32), b_hi = (unsigned)(p.b_desc >> 32);
         const unsigned a_lo0 = (unsigned)p.a_desc, b_lo0 = (unsigned)p.b_desc + ((smem_base >> 4) & 0x3fff);
-        unsigned a_off[9], b_off[9];
-#pragma unroll
-        for (int tap = 0; tap < 9; ++tap) {
-          const int r = tap / 3, t = tap % 3;
-          const int rowoff = p.kind == GK_CONV_FWD ? r * 10 + t : (2 - r) * 10 + (2 - t);
-          a_off[tap] = (unsigned)(rowoff * p.kdepth) >> 4;
-          b_off[tap] = (unsigned)(tap * p.b_tile_bytes) >> 4;
-        }
+        // per tap: a_off = patch row * (row bytes / 16), b_off = tap * (weight tile bytes / 16); the row
+        // numbers are compile-time constants after unrolling, so these are two multiplies per tap
+        const unsigned row16 = (unsigned)p.kdepth >> 4, btile16 = (unsigned)p.b_tile_bytes >> 4;
+        const bool fwd_taps = p.kind == GK_CONV_FWD;
         const unsigned a_stage16 = (unsigned)p.a_bytes >> 4;
         unsigned a_stage_lo = a_lo0 + (((smem_base + p.b_res_bytes) >> 4) & 0x3fff);   // stage 0
         for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
@@ -662,11 +658,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const unsigned a_lo = a_stage_lo + (unsigned)stage * a_stage16;
 #pragma unroll
           for (int tap = 0; tap < 9; ++tap) {
+            const int r = tap / 3, t = tap % 3;
+            const unsigned rowoff = fwd_taps ? (unsigned)(r * 10 + t) : (unsigned)((2 - r) * 10 + (2 - t));
+            const unsigned a_tap = a_lo + rowoff * row16, b_tap = b_lo0 + (unsigned)tap * btile16;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
               if (k < p.ksteps)
-                tc_mma_i8_lh(tmem_d, a_lo + a_off[tap] + 2 * k, a_hi, b_lo0 + b_off[tap] + k * p.b_kstep16, b_hi,
-                             p.idesc, (tap > 0 || k > 0) ? 1u : 0u);
+                tc_mma_i8_lh(tmem_d, a_tap + 2 * k, a_hi, b_tap + k * p.b_kstep16, b_hi, p.idesc,
+                             (tap > 0 || k > 0) ? 1u : 0u);
             }
           }
           tc_commit(empty0 + 8 * stage);
@@ -1213,7 +1212,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
         p.a_bytes = 12288; p.b_bytes = 8192;
         p.a_boxes = p.b_boxes = 1;
         p.stages = MAX_STAGES;
-        p.nprod = PROD_WARPS;
+        p.nprod = 2;                                          // divides the eight stages
         p.nbuf = 5;                                           // five accumulators of 64 columns
         p.ksteps = 4;
         // MN-major, 64-byte swizzle: 8-row groups one patch row (10 pixels) apart for A, contiguous for B;
