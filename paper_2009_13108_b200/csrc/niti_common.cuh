@@ -36,7 +36,8 @@ struct WsHeader {
   unsigned long long maxabs64;      // same for the 64-bit loss accumulators
   unsigned int tile_counter;        // arrival counter of the grid-wide wait
   unsigned int spec_b;              // bit-width the speculative epilogue rounded with
-  unsigned int pad1[2];
+  unsigned int done_ctas;           // CTAs that have finished (single-wave launches publish b themselves)
+  unsigned int pad1[1];
 };
 
 #define NITI_CUDA_TRY(ctx, expr)                                                        \

@@ -85,6 +85,8 @@ struct TcParams {
   int epi_mode;                 // EPI_SPILL / EPI_ATOMIC / EPI_SPECULATE / EPI_KNOWN_B
   int mbits, round_mode, relu;
   unsigned spec_mul256;         // the sampled max is scaled by this / 256 before taking its bit length
+  int single_wave;              // every CTA has at most one tile: the sample is the whole tensor, the shift
+                                // is exact, and the last CTA to finish publishes b and the exponent
 };
 
 // Epilogue modes.  The shift of Algorithm 2 needs the bit-width of the WHOLE accumulator tensor:
@@ -985,6 +987,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     __syncthreads();
   }
+  if (p.single_wave && p.epi_mode == EPI_SPECULATE && threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(&hdr->done_ctas, 1u) == gridDim.x - 1) {
+      __threadfence();
+      const int b_true = niti_bitlen32(*(volatile unsigned *)&hdr->maxabs32);
+      const int bpf = b_true > p.mbits ? b_true - p.mbits : 0;
+      if (b_out) *b_out = b_true;
+      if (s_out) {
+        int sv = bpf + (s_a ? *s_a : 0) + (s_w ? *s_w : 0);
+        *s_out = sv;
+        if (sv < -128 || sv > 127) atomicOr(status, NITI_DEV_EXP_RANGE);
+      }
+    }
+  }
   if (CTAS == 2) cluster_sync_all();   // nobody leaves while the peer may still touch this CTA
   if (warp == MMA_WARP) {
     tc_fence_after();
@@ -1378,11 +1394,40 @@ int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long 
 
 size_t niti_tc_scratch_bytes(const GemmProblem &) { return 0; }
 
+// CTAs (CTAS = 1) or CTA pairs (CTAS = 2) that can be resident at the same time.  SMs pair up inside a
+// GPC, so the number of pairs can be below sm_count / 2; a persistent grid larger than that would run
+// a second, short wave.
+template <int CTAS>
+static int tc_units(niti_ctx *ctx) {
+  static int cached = 0;
+  if (cached) return cached;
+  cached = ctx->sm_count / CTAS;
+  if (CTAS == 2) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)(ctx->sm_count / 2 * 2), 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = 200 * 1024;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    (void)cudaFuncSetAttribute(tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 201 * 1024);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, tc_gemm_kernel<2>, &cfg) == cudaSuccess && n > 0 && n < cached) cached = n;
+    else (void)cudaGetLastError();
+  }
+  return cached;
+}
+
 template <int CTAS>
 static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CUtensorMap &ma, const CUtensorMap &mb,
                      int32_t *acc, WsHeader *hdr, const RoundSpec &r) {
   size_t smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + (size_t)p.b_res_bytes + 1024;
-  static size_t attr_smem = 0;
+  static size_t attr_smem = CTAS == 2 ? 201 * 1024 : 0;
   if (smem > attr_smem) {
     NITI_CUDA_TRY(ctx, cudaFuncSetAttribute(tc_gemm_kernel<CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     attr_smem = smem;
@@ -1400,20 +1445,7 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  // CTA pairs that can be resident at the same time (SMs pair up inside a GPC, so this can be
-  // fewer than sm_count / 2); a persistent grid larger than that would run a second, short wave
-  static int units_cached = 0;
-  if (!units_cached) {
-    units_cached = ctx->sm_count / CTAS;
-    if (CTAS == 2) {
-      int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, tc_gemm_kernel<CTAS>, &cfg) == cudaSuccess && n > 0 && n < units_cached)
-        units_cached = n;
-      else
-        (void)cudaGetLastError();
-    }
-  }
-  const int units = units_cached;
+  const int units = tc_units<CTAS>(ctx);
   long long grid = (p.items < units ? p.items : units) * CTAS;
   cfg.gridDim = dim3((unsigned)grid, 1, 1);
   NITI_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, tc_gemm_kernel<CTAS>, ma, mb, p, acc, hdr, ctx->d_status, r.out, r.mask,
@@ -1447,13 +1479,14 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
   {
     // expected ratio between the max of the whole tensor (N values) and the max of the first tile of
     // every CTA (n values) for roughly Gaussian sums: sqrt(ln N / ln n)
-    const int units = ctx->sm_count / p.ctas;
+    const int units = p.ctas == 2 ? tc_units<2>(ctx) : tc_units<1>(ctx);
     const double n_all = (double)g.gm * (double)g.gn;
     const double frac = p.items > units ? (double)units / (double)p.items : 1.0;
     const double n_s = n_all * frac;
     double f = (n_s > 16.0 && frac < 1.0) ? sqrt(log(n_all) / log(n_s)) : 1.0;
     p.spec_mul256 = (unsigned)(f * 256.0 + 0.5);
   }
+  p.single_wave = (p.items <= (p.ctas == 2 ? tc_units<2>(ctx) : tc_units<1>(ctx)) && p.spec_mul256 == 256) ? 1 : 0;
   p.mbits = r.mbits;
   p.round_mode = r.round_mode;
   p.relu = r.relu;
@@ -1466,7 +1499,9 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
   if (prof) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st);
   int rc = p.ctas == 2 ? launch_tc<2>(ctx, st, p, ma, mb, acc, hdr, r) : launch_tc<1>(ctx, st, p, ma, mb, acc, hdr, r);
   if (rc != NITI_OK) return rc;
-  if (p.epi_mode == EPI_SPECULATE) {
+  if (p.epi_mode == EPI_SPECULATE && p.single_wave) {
+    *fused = true;                     // exact shift, scalars published by the last CTA: no second launch
+  } else if (p.epi_mode == EPI_SPECULATE) {
     // publishes b and the exponent; recomputes with the true bit-width only if the guess was low
     p.epi_mode = EPI_KNOWN_B;
     rc = p.ctas == 2 ? launch_tc<2>(ctx, st, p, ma, mb, acc, hdr, r) : launch_tc<1>(ctx, st, p, ma, mb, acc, hdr, r);
