@@ -5,6 +5,7 @@
 int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr);
 int niti_launch_im2col32(niti_ctx *ctx, cudaStream_t st, const int8_t *x, int8_t *xcol, int B, int H, int W,
                          int Ci, int R, int S, int pad, int Ho, int Wo);
+int niti_launch_pad_pitch(niti_ctx *ctx, cudaStream_t st, const int8_t *src, int8_t *dst, int rows, int n, int pitch);
 int niti_launch_pad_rows32(niti_ctx *ctx, cudaStream_t st, const int8_t *w, int8_t *wcol, int rows, int k);
 int niti_launch_round_compact32(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, const WsHeader *hdr, int8_t *out,
                                 int rows, int k, int mbits, int round_mode, int32_t *b_out);
@@ -181,6 +182,7 @@ extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
       fill_fc(p2, GK_FC_WGRAD, (int)d[0], (int)d[1], (int)d[2]);
       size_t e1 = niti_tc_scratch_bytes(p), e2 = niti_tc_scratch_bytes(p2);
       extra = e1 > e2 ? e1 : e2;
+      if (d[1] % 16) extra += round_up((size_t)d[0] * (size_t)((d[1] + 15) / 16 * 16), 256);   // e with padded rows
       break;
     }
     case NITI_OP_CONV_FWD:
@@ -261,14 +263,29 @@ extern "C" int niti_linear_bwd(niti_ctx *ctx, void *stream, const int8_t *a, con
     return niti_fail(ctx, NITI_ERR_ARG, "niti_linear_bwd: bad argument (pointers must be 16-byte aligned)");
   int64_t dims[3] = {M, N, K};
   size_t need = niti_workspace_bytes(NITI_OP_LINEAR_BWD, dims, 3);
+  // TMA needs 16-byte row pitches: an error tensor with N % 16 != 0 (10 or 1000 classes) is copied
+  // once into rows padded to the next multiple of 16 for the tensor-core engine
+  const int8_t *e_tc = e;
+  long long e_ld = 0;
+  if ((N % 16) != 0 && N >= 32 && ctx->engine != 1) {
+    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
+      return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    const int pitch = (N + 15) / 16 * 16;
+    size_t a_out = (size_t)M * K, b_out = (size_t)N * K;
+    int8_t *epad = (int8_t *)((char *)ws + NITI_WS_HEADER + round_up((a_out > b_out ? a_out : b_out) * 4, 256));
+    int rcp = niti_launch_pad_pitch(ctx, (cudaStream_t)stream, e, epad, M, N, pitch);
+    if (rcp != NITI_OK) return rcp;
+    e_tc = epad;
+    e_ld = pitch;
+  }
   GemmProblem p;
   fill_fc(p, GK_FC_WGRAD, M, N, K);
-  p.p0 = e; p.p1 = a;
+  p.p0 = e_tc; p.p1 = a; p.ld0 = e_ld;
   int rc = run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, g, m_u, round_mode, 0, nullptr,
                           nullptr, nullptr, nullptr, b_g);
   if (rc != NITI_OK || !e_prev) return rc;
   fill_fc(p, GK_FC_DGRAD, M, N, K);
-  p.p0 = e; p.p1 = w;
+  p.p0 = e_tc; p.p1 = w; p.ld0 = e_ld;
   return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, e_prev, 7, round_mode, 0,
                         relu_mask_src, nullptr, nullptr, nullptr, b_e);
 }

@@ -100,6 +100,8 @@ struct GemmProblem {
   int B, H, W, Ho, Wo, Ci, Co, R, S, pad;
   // the matrix multiply actually run
   long long gm, gn, gk;
+  // row pitch in bytes of p0 when its rows are padded (fully connected kinds; 0 = dense)
+  long long ld0;
 };
 
 // Plain CUDA-core engine: writes int32 accumulators to acc[gm][gn] and max|acc| to hdr->maxabs32.

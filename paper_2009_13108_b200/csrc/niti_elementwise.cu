@@ -122,6 +122,23 @@ __global__ void pad_rows32_kernel(const int8_t *__restrict__ w, int8_t *__restri
   }
 }
 
+// rows of n bytes -> rows of pitch bytes (pitch >= n), zero padded
+__global__ void pad_pitch_kernel(const int8_t *__restrict__ src, int8_t *__restrict__ dst, int rows, int n, int pitch) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < (long long)rows * pitch) {
+    const int r = (int)(idx / pitch), c = (int)(idx % pitch);
+    dst[idx] = c < n ? src[(long long)r * n + c] : (int8_t)0;
+  }
+}
+
+int niti_launch_pad_pitch(niti_ctx *ctx, cudaStream_t st, const int8_t *src, int8_t *dst, int rows, int n, int pitch) {
+  long long total = (long long)rows * pitch;
+  pad_pitch_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(src, dst, rows, n, pitch);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
 // Rounds acc[rows][32] (int32) and keeps the first k columns: out[rows][k].
 __global__ void round_compact32_kernel(const int32_t *__restrict__ acc, const WsHeader *__restrict__ hdr,
                                        int8_t *__restrict__ out, int rows, int k, int mbits, int round_mode,

@@ -16,6 +16,7 @@ struct Addr {
   int M, N, K;                                  // fully connected dims
   int H, W, Ho, Wo, Ci, Co, R, S, pad;          // convolution dims
   long long gm, gn, gk;
+  long long pitch0;                             // row pitch of p0 for the fully connected backward kinds
 };
 
 // element A(m, k) of the implicit left operand, 0 outside the problem
@@ -23,8 +24,8 @@ __device__ __forceinline__ int8_t load_a(const Addr &q, long long m, long long k
   if (m >= q.gm || k >= q.gk) return 0;
   switch (q.kind) {
     case GK_FC_FWD: return q.p0[m * q.K + k];
-    case GK_FC_DGRAD: return q.p0[m * q.N + k];               // e[m][n], k == n
-    case GK_FC_WGRAD: return q.p0[k * q.N + m];               // e[mm][n], m == n, k == mm
+    case GK_FC_DGRAD: return q.p0[m * q.pitch0 + k];          // e[m][n], k == n
+    case GK_FC_WGRAD: return q.p0[k * q.pitch0 + m];          // e[mm][n], m == n, k == mm
     case GK_CONV_FWD: {
       int ci = (int)(k % q.Ci);
       int rs = (int)(k / q.Ci);
@@ -219,6 +220,7 @@ int niti_simt_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t
   q.M = p.M; q.N = p.N; q.K = p.K;
   q.H = p.H; q.W = p.W; q.Ho = p.Ho; q.Wo = p.Wo; q.Ci = p.Ci; q.Co = p.Co; q.R = p.R; q.S = p.S; q.pad = p.pad;
   q.gm = p.gm; q.gn = p.gn; q.gk = p.gk;
+  q.pitch0 = p.ld0 ? p.ld0 : p.N;
   long long gx = (p.gn + TN - 1) / TN, gy = (p.gm + TM - 1) / TM;
   if (gy > 65535) return niti_fail(ctx, NITI_ERR_SHAPE, "simt gemm: too many row tiles");
   // split the contraction when the output grid alone cannot fill the GPU

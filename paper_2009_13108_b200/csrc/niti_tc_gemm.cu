@@ -1121,7 +1121,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
       p.bn = g.gn >= 256 ? 256 : (int)((g.gn + b_sw - 1) / b_sw * b_sw);
       if (p.bn % 32) return false;
       a_sw = p.kdepth;
-      sa = {2, {(cuuint64_t)g.gk, (cuuint64_t)g.gm}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, BM}, a_sw, g.p0};
+      sa = {2, {(cuuint64_t)g.gk, (cuuint64_t)g.gm}, {(cuuint64_t)(g.ld0 ? g.ld0 : g.gk)}, {(cuuint32_t)p.kdepth, BM}, a_sw, g.p0};
       sb = {2, {(cuuint64_t)g.gn, (cuuint64_t)g.gk}, {(cuuint64_t)g.gn}, {(cuuint32_t)b_sw, (cuuint32_t)p.kdepth}, b_sw, g.p1};
       p.kb_total = (int)((g.gk + p.kdepth - 1) / p.kdepth);
       m_tiles = (g.gm + BM - 1) / BM;
@@ -1136,7 +1136,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
       p.kdepth = g.gk >= 128 ? 128 : (g.gk >= 64 ? 64 : 32);
       p.bn = g.gn >= 256 ? 256 : (int)((g.gn + b_sw - 1) / b_sw * b_sw);
       if (p.bn % 32) return false;
-      sa = {2, {(cuuint64_t)g.gm, (cuuint64_t)g.gk}, {(cuuint64_t)g.gm}, {(cuuint32_t)a_sw, (cuuint32_t)p.kdepth}, a_sw, g.p0};
+      sa = {2, {(cuuint64_t)g.gm, (cuuint64_t)g.gk}, {(cuuint64_t)(g.ld0 ? g.ld0 : g.gm)}, {(cuuint32_t)a_sw, (cuuint32_t)p.kdepth}, a_sw, g.p0};
       sb = {2, {(cuuint64_t)g.gn, (cuuint64_t)g.gk}, {(cuuint64_t)g.gn}, {(cuuint32_t)b_sw, (cuuint32_t)p.kdepth}, b_sw, g.p1};
       p.kb_total = (int)((g.gk + p.kdepth - 1) / p.kdepth);
       m_tiles = (g.gm + BM - 1) / BM;
