@@ -113,6 +113,12 @@ uint64_t niti_tc_pair_launch_count(niti_ctx *ctx);
  * run so far (synchronises `stream`; -1 on error). */
 int64_t niti_redo_count(niti_ctx *ctx, void *stream);
 
+/* Self-test of the failure detection: every wait inside the kernels is bounded; this enqueues a
+ * one-warp kernel that waits (about 50 ms) on a barrier nothing completes, gives up, raises
+ * NITI_DEV_TIMEOUT in the device status word and returns normally.  niti_check() then reports
+ * NITI_ERR_DEVICE once, and the context and the GPU remain usable. */
+int niti_selftest_timeout(niti_ctx *ctx, void *stream);
+
 /* Timing of the tensor-core matrix-multiply kernel.  While enabled, every launch of that
  * kernel is bracketed by a pair of CUDA events on its stream (up to 8192 launches are kept).
  * niti_profile_read() waits for the recorded events, returns their summed duration in

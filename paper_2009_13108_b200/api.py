@@ -20,7 +20,7 @@ OP_LINEAR_FWD, OP_LINEAR_BWD, OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_INT_
 EXPORTS = [
     "niti_create", "niti_destroy", "niti_last_error", "niti_check", "niti_workspace_bytes",
     "niti_set_engine", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
-    "niti_redo_count", "niti_profile_enable", "niti_profile_read_launches",
+    "niti_redo_count", "niti_selftest_timeout", "niti_profile_enable", "niti_profile_read_launches",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
     "niti_conv_dgrad", "niti_conv_wgrad", "niti_int_xent", "niti_int_xent_noalloc", "niti_int_sgd_update",
     "niti_relu_fwd",
@@ -60,6 +60,7 @@ def load_library():
     lib.niti_tc_pair_launch_count.restype = C.c_uint64
     lib.niti_profile_read_launches.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), i32]
     lib.niti_redo_count.argtypes = [vp, vp]
+    lib.niti_selftest_timeout.argtypes = [vp, vp]
     lib.niti_redo_count.restype = C.c_int64
     lib.niti_profile_enable.argtypes = [vp, i32]
     lib.niti_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64),
@@ -150,6 +151,9 @@ class Niti:
 
     def redo_count(self) -> int:
         return int(self.lib.niti_redo_count(self.h, self._stream()))
+
+    def selftest_timeout(self):
+        self._ck(self.lib.niti_selftest_timeout(self.h, self._stream()))
 
     def profile_enable(self, on: bool):
         self._ck(self.lib.niti_profile_enable(self.h, int(on)))

@@ -81,6 +81,12 @@ extern "C" int64_t niti_redo_count(niti_ctx *ctx, void *stream) {
   return (int64_t)h;
 }
 
+int niti_tc_timeout_probe(niti_ctx *ctx, cudaStream_t st);
+extern "C" int niti_selftest_timeout(niti_ctx *ctx, void *stream) {
+  if (!ctx) return NITI_ERR_ARG;
+  return niti_tc_timeout_probe(ctx, (cudaStream_t)stream);
+}
+
 extern "C" int niti_profile_enable(niti_ctx *ctx, int on) {
   if (!ctx) return NITI_ERR_ARG;
   if (on && !ctx->prof_ev) {

@@ -145,13 +145,13 @@ __device__ __forceinline__ bool mbar_try_sleep(unsigned bar, unsigned parity, un
 // Bounded wait.  Returns false (and raises the abort flag) if the barrier did not flip in time or
 // another thread already gave up.
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int *abort_flag,
-                                          uint32_t *status) {
+                                          uint32_t *status, long long limit_cycles = WAIT_LIMIT_CYCLES) {
   if (mbar_try(bar, parity)) return true;
   long long t0 = clock64();
   while (true) {
     if (mbar_try_sleep(bar, parity, 20000u)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+    if (clock64() - t0 > limit_cycles) {
       *abort_flag = 1;
       atomicOr(status, NITI_DEV_TIMEOUT);
       return false;
@@ -1011,6 +1011,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever completes, gives up
+// after ~50 ms, raises NITI_DEV_TIMEOUT and returns normally (the context stays usable).
+__global__ void timeout_probe_kernel(uint32_t *status) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ volatile int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) (void)mbar_wait(smem_u32(&bar), 0, &abort_flag, status, 100000000LL);
+  __syncthreads();
+}
+
 // ------------------------------------------------------------------------------------------
 // Host side: tensor maps, descriptors, eligibility
 // ------------------------------------------------------------------------------------------
@@ -1393,6 +1408,13 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
 int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr);
 
 size_t niti_tc_scratch_bytes(const GemmProblem &) { return 0; }
+
+int niti_tc_timeout_probe(niti_ctx *ctx, cudaStream_t st) {
+  timeout_probe_kernel<<<1, 32, 0, st>>>(ctx->d_status);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
 
 // CTAs (CTAS = 1) or CTA pairs (CTAS = 2) that can be resident at the same time.  SMs pair up inside a
 // GPC, so the number of pairs can be below sm_count / 2; a persistent grid larger than that would run

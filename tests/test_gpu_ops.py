@@ -262,3 +262,20 @@ def test_argument_errors(niti):
                                   niti.scalar().data_ptr(), a.data_ptr(), None, None, 4, 4, 32, 0, 0,
                                   niti._ws.data_ptr(), ctypes.c_size_t(16))
     assert rc == 3
+
+
+def test_bounded_wait_reports_a_timeout_and_the_context_survives(niti, oref):
+    """Failure detection without a fault: a wait that nothing satisfies runs out, the device status
+    word says so, and the next call works."""
+    from paper_2009_13108_b200 import NitiError
+    niti.selftest_timeout()
+    with pytest.raises(NitiError) as ei:
+        niti.check()
+    assert ei.value.code == 6 and "0x1" in str(ei.value)
+    assert niti.check() == 0
+    rng = np.random.default_rng(5)
+    a, w = _i8(rng, (128, 256)), _i8(rng, (64, 256))
+    want, s, b = oref.linear_fwd(a, -7, w, -10)
+    out, s_out, b_out = niti.linear_fwd(_T(niti, a), niti.scalar(-7), _T(niti, w), niti.scalar(-10))
+    _eq(out, want)
+    niti.check()

@@ -43,6 +43,26 @@ def _run_both(niti, net, steps):
     return tr
 
 
+def test_nearest_rounding_and_smaller_update_width(niti):
+    """The paper's accuracy runs round a and e to nearest and shrink m_u over training."""
+    from oracle import OracleNetState, oracle_train_step
+    from paper_2009_13108_b200 import NitiTrainer
+    for m_u, mode in [(3, 1), (4, 0)]:
+        net = config_net(2, batch=16)
+        net.m_u = m_u
+        x, labels, weights = make_net_inputs(net)
+        st = OracleNetState([w.copy() for w in weights])
+        tr = NitiTrainer(niti, net, weights, round_mode=mode)
+        tr.load_batch(x, labels)
+        for _ in range(2):
+            rec = oracle_train_step(net, x, labels, st, round_mode=mode)
+            tr.step()
+            niti.check()
+            assert int(tr.n_correct) == rec["n_correct"]
+            for wg, wo in zip(tr.weights, st.weights):
+                assert np.array_equal(wg.cpu().numpy(), wo)
+
+
 def test_config0_mlp_full_size(niti):
     _run_both(niti, config_net(0), steps=5)
 
