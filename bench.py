@@ -323,7 +323,8 @@ def run_ours(args):
 
     niti = Niti(local)
     net = config_net(args.config)
-    net.seed = net.seed + 1000 * rank            # every rank draws its own batch and replica
+    from paper_2009_13108_b200.dist_util import aggregate_throughput, max_over_ranks, rank_seed
+    net.seed = rank_seed(net.seed, rank)         # every rank draws its own batch and replica
     x, labels, weights = make_net_inputs(net)
     tr = NitiTrainer(niti, net, weights)
     xh = torch.from_numpy(x).pin_memory()
@@ -402,10 +403,7 @@ def run_ours(args):
     ms_e2e = t0.elapsed_time(t1)
     clocks = sampler.stop()
     niti.check()
-    if dist is not None:
-        t = torch.tensor([ms, ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], device="cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -418,7 +416,8 @@ def run_ours(args):
     int8_peak = 2.0 * pk["bf16_sustained"]
     achieved = k_ops / max(k_ms, 1e-9) / 1e9
     line = {
-        "metric": METRIC, "value": images / (ms / 1e3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": aggregate_throughput(net.batch * args.steps, ms, world), "unit": UNIT,
+        "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s8",
         "data": "synthetic",
