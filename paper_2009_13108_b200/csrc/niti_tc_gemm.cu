@@ -326,6 +326,53 @@ __device__ __forceinline__ void tc_mma_i8_pair(unsigned tmem_d, unsigned long lo
       : "memory");
 }
 
+__device__ __forceinline__ void tc_mma_i8_pair_lh(unsigned tmem_d, unsigned a_lo, unsigned a_hi, unsigned b_lo,
+                                                  unsigned b_hi, unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %5, p;\n\t}"
+      ::"r"(tmem_d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// The issuing thread is a single instruction stream: every scalar instruction between two MMAs is
+// on the critical path of the tensor pipe (measured: run-time trip counts, selects and multiplies
+// per MMA cost ~35 cycles each time, more than half of an N = 64 MMA).  The issue loops are therefore
+// compiled per k-step count, with every offset either a literal or a register filled before the
+// tile loop.
+//
+// One 3x3 tile from the resident patch: nine taps, KS k-steps each, into one accumulator.
+template <int KS>
+__device__ __forceinline__ void halo_issue_tile(unsigned tmem_d, unsigned a_lo, unsigned a_hi, const unsigned (&a_off)[9],
+                                                unsigned b_hi, const unsigned (&b_tap)[9], unsigned b_kstep16,
+                                                unsigned idesc) {
+#pragma unroll
+  for (int tap = 0; tap < 9; ++tap) {
+    const unsigned a_t = a_lo + a_off[tap];
+#pragma unroll
+    for (int k = 0; k < KS; ++k)
+      tc_mma_i8_lh(tmem_d, a_t + 2u * k, a_hi, b_tap[tap] + (unsigned)k * b_kstep16, b_hi, idesc,
+                   (tap > 0 || k > 0) ? 1u : 0u);
+  }
+}
+// One k-block of the generic loop: KS MMAs whose operands advance by the k-step strides.
+template <int CTAS, int KS>
+__device__ __forceinline__ void issue_kblock(unsigned tmem_d, unsigned a_lo, unsigned a_hi, unsigned b_lo, unsigned b_hi,
+                                             unsigned a_kstep16, unsigned b_kstep16, unsigned idesc, unsigned first_acc) {
+#pragma unroll
+  for (int k = 0; k < KS; ++k) {
+    if (CTAS == 2)
+      tc_mma_i8_pair_lh(tmem_d, a_lo + (unsigned)k * a_kstep16, a_hi, b_lo + (unsigned)k * b_kstep16, b_hi, idesc,
+                        k > 0 ? 1u : first_acc);
+    else
+      tc_mma_i8_lh(tmem_d, a_lo + (unsigned)k * a_kstep16, a_hi, b_lo + (unsigned)k * b_kstep16, b_hi, idesc,
+                   k > 0 ? 1u : first_acc);
+  }
+}
+
 template <int CTAS>
 __device__ __forceinline__ void load2(unsigned dst, const CUtensorMap *m, unsigned bar, int c0, int c1) {
   if (CTAS == 2) tma_load_2d_pair(dst, m, bar, c0, c1); else tma_load_2d(dst, m, bar, c0, c1);
@@ -645,12 +692,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // starts one pixel up and left of the tile) and the tap's resident weight tile
         const unsigned a_hi = (unsigned)(p.a_desc >> 32), b_hi = (unsigned)(p.b_desc >> 32);
         const unsigned a_lo0 = (unsigned)p.a_desc, b_lo0 = (unsigned)p.b_desc + ((smem_base >> 4) & 0x3fff);
-        // per tap: a_off = patch row * (row bytes / 16), b_off = tap * (weight tile bytes / 16); the row
-        // numbers are compile-time constants after unrolling, so these are two multiplies per tap
+        // per tap, filled once: a_off = patch row * (row bytes / 16), b_tap = descriptor of the tap's
+        // resident weight tile
         const unsigned row16 = (unsigned)p.kdepth >> 4, btile16 = (unsigned)p.b_tile_bytes >> 4;
         const bool fwd_taps = p.kind == GK_CONV_FWD;
         const unsigned a_stage16 = (unsigned)p.a_bytes >> 4;
-        unsigned a_stage_lo = a_lo0 + (((smem_base + p.b_res_bytes) >> 4) & 0x3fff);   // stage 0
+        const unsigned a_stage_lo = a_lo0 + (((smem_base + p.b_res_bytes) >> 4) & 0x3fff);   // stage 0
+        const unsigned b_kstep16 = p.b_kstep16, idesc = p.idesc;
+        const int ksteps = p.ksteps;
+        unsigned a_off[9], b_tap[9];
+#pragma unroll
+        for (int tap = 0; tap < 9; ++tap) {
+          const int r = tap / 3, t = tap % 3;
+          a_off[tap] = (fwd_taps ? (unsigned)(r * 10 + t) : (unsigned)((2 - r) * 10 + (2 - t))) * row16;
+          b_tap[tap] = b_lo0 + (unsigned)tap * btile16;
+        }
         for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
           const unsigned buf = use % (unsigned)p.nbuf;
           if (!mbar_wait(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
@@ -658,24 +714,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tc_fence_after();
           const unsigned tmem_d = tmem_base + buf * (unsigned)p.bn;
           const unsigned a_lo = a_stage_lo + (unsigned)stage * a_stage16;
-#pragma unroll
-          for (int tap = 0; tap < 9; ++tap) {
-            const int r = tap / 3, t = tap % 3;
-            const unsigned rowoff = fwd_taps ? (unsigned)(r * 10 + t) : (unsigned)((2 - r) * 10 + (2 - t));
-            const unsigned a_tap = a_lo + rowoff * row16, b_tap = b_lo0 + (unsigned)tap * btile16;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              if (k < p.ksteps)
-                tc_mma_i8_lh(tmem_d, a_tap + 2 * k, a_hi, b_tap + k * p.b_kstep16, b_hi, p.idesc,
-                             (tap > 0 || k > 0) ? 1u : 0u);
-            }
-          }
+          if (ksteps == 2) halo_issue_tile<2>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
+          else if (ksteps == 4) halo_issue_tile<4>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
+          else halo_issue_tile<1>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
           tc_commit(empty0 + 8 * stage);
           tc_commit(tfull0 + 8 * buf);
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
         }
         item_end = first_item;
       }
+      // generic loop: everything an MMA needs that does not change is read into registers here
+      const unsigned g_a_lo0 = (unsigned)p.a_desc, g_b_lo0 = (unsigned)p.b_desc;
+      const unsigned g_a_hi = (unsigned)(p.a_desc >> 32), g_b_hi = (unsigned)(p.b_desc >> 32);
+      const unsigned g_ak = p.a_kstep16, g_bk = p.b_kstep16, g_idesc = p.idesc, g_a_bytes = (unsigned)p.a_bytes;
+      const int g_ksteps = p.ksteps;
       for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
         const int split = (int)(item % p.splits);
         const int kb0 = split * p.kb_per_split;
@@ -690,24 +742,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (!mbar_wait(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
           tc_fence_after();
           const unsigned sa = smem_base + stage * stage_bytes;
-          const unsigned sb = sa + p.a_bytes;
-          if (CTAS == 2) {
-            unsigned long long da = p.a_desc | (unsigned long long)((sa >> 4) & 0x3fff);
-            unsigned long long db = p.b_desc | (unsigned long long)((sb >> 4) & 0x3fff);
-            for (int k = 0; k < p.ksteps; ++k) {
-              tc_mma_i8_pair(tmem_d, da, db, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-              da += p.a_kstep16;
-              db += p.b_kstep16;
-            }
-          } else {
-            unsigned a_lo = (unsigned)p.a_desc + ((sa >> 4) & 0x3fff), b_lo = (unsigned)p.b_desc + ((sb >> 4) & 0x3fff);
-            const unsigned a_hi = (unsigned)(p.a_desc >> 32), b_hi = (unsigned)(p.b_desc >> 32);
-            for (int k = 0; k < p.ksteps; ++k) {
-              tc_mma_i8_lh(tmem_d, a_lo, a_hi, b_lo, b_hi, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-              a_lo += p.a_kstep16;
-              b_lo += p.b_kstep16;
-            }
-          }
+          const unsigned a_lo = g_a_lo0 + ((sa >> 4) & 0x3fff), b_lo = g_b_lo0 + (((sa + g_a_bytes) >> 4) & 0x3fff);
+          const unsigned first_acc = kb > kb0 ? 1u : 0u;
+          if (g_ksteps == 4) issue_kblock<CTAS, 4>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+          else if (g_ksteps == 2) issue_kblock<CTAS, 2>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+          else if (g_ksteps == 1) issue_kblock<CTAS, 1>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+          else issue_kblock<CTAS, 3>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
           // frees the stage (in every CTA of the pair) once these MMAs have read it
           if (CTAS == 2) tc_commit_pair(empty0 + 8 * stage); else tc_commit(empty0 + 8 * stage);
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
