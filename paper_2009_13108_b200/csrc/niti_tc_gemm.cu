@@ -158,6 +158,33 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatil
     }
   }
 }
+// The same bounded wait for a whole converged warp: every lane polls, the votes make the outcome (and
+// with it the caller's control flow) warp-uniform, so the compiler can keep the caller's address
+// arithmetic in uniform registers.
+__device__ __forceinline__ bool mbar_wait_warp(unsigned bar, unsigned parity, volatile int *abort_flag,
+                                               uint32_t *status, long long limit_cycles = WAIT_LIMIT_CYCLES) {
+  if (__all_sync(0xffffffffu, mbar_try(bar, parity))) return true;
+  const long long t0 = clock64();
+  while (true) {
+    if (__all_sync(0xffffffffu, mbar_try_sleep(bar, parity, 20000u))) return true;
+    if (__any_sync(0xffffffffu, *abort_flag != 0)) return false;
+    if (__any_sync(0xffffffffu, clock64() - t0 > limit_cycles)) {
+      *abort_flag = 1;
+      atomicOr(status, NITI_DEV_TIMEOUT);
+      return false;
+    }
+  }
+}
+// One lane of a converged warp (the same one every time it is asked).
+__device__ __forceinline__ bool elect_one() {
+  unsigned pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -431,7 +458,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ volatile int abort_flag;
   __shared__ volatile int spec_bp_ready;      // 0: not yet; else the speculative binary point + 1
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const unsigned rank = CTAS == 2 ? cluster_ctarank() : 0u;
   const unsigned smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int stage_bytes = p.a_bytes + p.b_bytes;
@@ -641,7 +668,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else if (warp == MMA_WARP) {
     // ================= MMA issuer (leader CTA only) =================
-    if (lane == 0 && rank == 0) {
+    // The whole warp runs the loops in lock step and one elected lane issues: with warp-uniform
+    // control flow the descriptor arithmetic stays in the uniform datapath that feeds tcgen05.mma.
+    if (rank == 0) {
+      const bool leader = elect_one();
       int stage = 0;
       unsigned phase = 0;
       unsigned use = 0;                 // tiles processed by this CTA (pair)
@@ -664,29 +694,31 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int t0 = split * p.kb_per_split;
           int t1 = t0 + p.kb_per_split;
           if (t1 > p.kb_total) t1 = p.kb_total;
-          if (!mbar_wait(tempty0, (use & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
+          if (!mbar_wait_warp(tempty0, (use & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
           tc_fence_after();
           for (int t = t0; t < t1; ++t) {
-            if (!mbar_wait(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
+            if (!mbar_wait_warp(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
             tc_fence_after();
             const unsigned sa16 = ((smem_base + stage * stage_bytes) >> 4) & 0x3fff;
             const unsigned sb16 = ((smem_base + stage * stage_bytes + p.a_bytes) >> 4) & 0x3fff;
             const unsigned first = t > t0 ? 1u : 0u;
+            if (leader) {
 #pragma unroll
-            for (int pi = 0; pi < 5; ++pi) {
+              for (int pi = 0; pi < 5; ++pi) {
 #pragma unroll
-              for (int j = 0; j < 4; ++j)      // 32 pixels = four rows of eight per MMA
-                tc_mma_i8_lh(tmem_base + 64u * pi, sa16 + a_pair[pi] + 160u * j, a_hi, b_lo0 + sb16 + 128u * j, b_hi,
-                             p.idesc, j > 0 ? 1u : first);
+                for (int j = 0; j < 4; ++j)      // 32 pixels = four rows of eight per MMA
+                  tc_mma_i8_lh(tmem_base + 64u * pi, sa16 + a_pair[pi] + 160u * j, a_hi, b_lo0 + sb16 + 128u * j, b_hi,
+                               p.idesc, j > 0 ? 1u : first);
+              }
+              tc_commit(empty0 + 8 * stage);
             }
-            tc_commit(empty0 + 8 * stage);
             if (++stage == p.stages) { stage = 0; phase ^= 1; }
           }
-          if (ok) tc_commit(tfull0);
+          if (ok && leader) tc_commit(tfull0);
         }
         item_end = first_item;
       } else if (p.halo) {
-        ok = mbar_wait(bres_bar, 0, &abort_flag, status);
+        ok = mbar_wait_warp(bres_bar, 0, &abort_flag, status);
         // descriptor low words per tap, computed once: the patch row where the tap starts
         // (forward reads x[i + r - 1][j + t - 1], dgrad reads e[i - r + 1][j - t + 1]; the patch
         // starts one pixel up and left of the tile) and the tap's resident weight tile
@@ -709,16 +741,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
           const unsigned buf = use % (unsigned)p.nbuf;
-          if (!mbar_wait(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
-          if (!mbar_wait(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
+          if (!mbar_wait_warp(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
+          if (!mbar_wait_warp(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
           tc_fence_after();
           const unsigned tmem_d = tmem_base + buf * (unsigned)p.bn;
           const unsigned a_lo = a_stage_lo + (unsigned)stage * a_stage16;
-          if (ksteps == 2) halo_issue_tile<2>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
-          else if (ksteps == 4) halo_issue_tile<4>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
-          else halo_issue_tile<1>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
-          tc_commit(empty0 + 8 * stage);
-          tc_commit(tfull0 + 8 * buf);
+          if (leader) {
+            if (ksteps == 2) halo_issue_tile<2>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
+            else if (ksteps == 4) halo_issue_tile<4>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
+            else halo_issue_tile<1>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
+            tc_commit(empty0 + 8 * stage);
+            tc_commit(tfull0 + 8 * buf);
+          }
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
         }
         item_end = first_item;
@@ -735,24 +769,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (kb1 > p.kb_total) kb1 = p.kb_total;
         const unsigned buf = use % (unsigned)p.nbuf;
         // wait until the epilogue has drained this accumulator buffer (the first nbuf uses pass at once)
-        if (!mbar_wait(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
+        if (!mbar_wait_warp(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
         tc_fence_after();
         const unsigned tmem_d = tmem_base + buf * (unsigned)p.bn;
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
+          if (!mbar_wait_warp(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
           tc_fence_after();
           const unsigned sa = smem_base + stage * stage_bytes;
           const unsigned a_lo = g_a_lo0 + ((sa >> 4) & 0x3fff), b_lo = g_b_lo0 + (((sa + g_a_bytes) >> 4) & 0x3fff);
           const unsigned first_acc = kb > kb0 ? 1u : 0u;
-          if (g_ksteps == 4) issue_kblock<CTAS, 4>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
-          else if (g_ksteps == 2) issue_kblock<CTAS, 2>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
-          else if (g_ksteps == 1) issue_kblock<CTAS, 1>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
-          else issue_kblock<CTAS, 3>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
-          // frees the stage (in every CTA of the pair) once these MMAs have read it
-          if (CTAS == 2) tc_commit_pair(empty0 + 8 * stage); else tc_commit(empty0 + 8 * stage);
+          if (leader) {
+            if (g_ksteps == 4) issue_kblock<CTAS, 4>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+            else if (g_ksteps == 2) issue_kblock<CTAS, 2>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+            else if (g_ksteps == 1) issue_kblock<CTAS, 1>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+            else issue_kblock<CTAS, 3>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+            // frees the stage (in every CTA of the pair) once these MMAs have read it
+            if (CTAS == 2) tc_commit_pair(empty0 + 8 * stage); else tc_commit(empty0 + 8 * stage);
+          }
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
         }
-        if (ok) {                               // accumulator complete
+        if (ok && leader) {                     // accumulator complete
           if (CTAS == 2) tc_commit_pair(tfull0 + 8 * buf); else tc_commit(tfull0 + 8 * buf);
         }
       }
