@@ -527,7 +527,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (warp < PROD_WARPS) {
     // ================= TMA producers (every CTA loads its own rows of A and its share of B) ========
-    if (lane == 0) {
+    // Each producer warp runs its loop in lock step and one elected lane issues the copies (warp-uniform
+    // control flow keeps the coordinate arithmetic in the uniform datapath that feeds the TMA unit).
+    {
+      const bool leader = elect_one();
       int stage = 0;
       unsigned phase = 0;
       bool ok = true;
@@ -543,12 +546,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           int wt = t0 % p.w_tiles, ht = (t0 / p.w_tiles) % p.h_tiles, bt = t0 / (p.w_tiles * p.h_tiles);
           for (int t = t0; t < t1; ++t) {
             if (stage % p.nprod == warp) {
-              if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
+              if (!mbar_wait_warp(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
               const unsigned full = full0 + 8 * stage;
               const unsigned sa = smem_base + stage * stage_bytes;
-              mbar_expect_tx(full, (unsigned)(p.a_box_bytes + p.b_box_bytes));
-              tma_load_4d(sa, &map_a, full, ci0, wt * 8 - 1, ht * 16 - 1, bt);          // input patch
-              tma_load_4d(sa + p.a_bytes, &map_b, full, co0, wt * 8, ht * 16, bt);     // error tile
+              if (leader) {
+                mbar_expect_tx(full, (unsigned)(p.a_box_bytes + p.b_box_bytes));
+                tma_load_4d(sa, &map_a, full, ci0, wt * 8 - 1, ht * 16 - 1, bt);          // input patch
+                tma_load_4d(sa + p.a_bytes, &map_b, full, co0, wt * 8, ht * 16, bt);     // error tile
+              }
             }
             if (++stage == p.stages) { stage = 0; phase ^= 1; }
             if (++wt == p.w_tiles) { wt = 0; if (++ht == p.h_tiles) { ht = 0; ++bt; } }
@@ -558,8 +563,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       } else if (p.halo) {
         // resident weights: one tile per tap, [bn rows][kdepth] K-major (forward) or
         // [kdepth rows][bn] MN-major in b_boxes column chunks (dgrad)
-        if (warp == 0) mbar_expect_tx(bres_bar, (unsigned)(9 * p.b_boxes * p.b_box_bytes));
-        for (int tap = 0; warp == 0 && tap < 9; ++tap) {
+        if (warp == 0 && leader) mbar_expect_tx(bres_bar, (unsigned)(9 * p.b_boxes * p.b_box_bytes));
+        for (int tap = 0; warp == 0 && leader && tap < 9; ++tap) {
           const unsigned dst = smem_base + tap * p.b_tile_bytes;
           if (p.kind == GK_CONV_FWD) {
             tma_load_2d(dst, &map_b, bres_bar, tap * p.kdepth, 0);
@@ -573,10 +578,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int bt = (int)(first_item / ((long long)p.w_tiles * p.h_tiles));
         for (long long item = first_item; ok && item < item_end; ++item) {
           if (stage % p.nprod == warp) {
-            if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
+            if (!mbar_wait_warp(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
             const unsigned full = full0 + 8 * stage;
-            mbar_expect_tx(full, (unsigned)p.a_box_bytes);
-            tma_load_4d(smem_base + p.b_res_bytes + stage * p.a_bytes, &map_a, full, 0, wt * 8 - 1, ht * 16 - 1, bt);
+            if (leader) {
+              mbar_expect_tx(full, (unsigned)p.a_box_bytes);
+              tma_load_4d(smem_base + p.b_res_bytes + stage * p.a_bytes, &map_a, full, 0, wt * 8 - 1, ht * 16 - 1, bt);
+            }
           }
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
           if (++wt == p.w_tiles) { wt = 0; if (++ht == p.h_tiles) { ht = 0; ++bt; } }
@@ -614,10 +621,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const unsigned tx_bytes = (unsigned)(CTAS * (p.a_boxes * p.a_box_bytes + p.b_boxes * p.b_box_bytes));
         for (int kb = kb0; kb < kb1; ++kb) {
          if (stage % p.nprod == warp) {
-          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
+          if (!mbar_wait_warp(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
           const unsigned full = lead_full0 + 8 * stage;
           const unsigned sa = smem_base + stage * stage_bytes;
           const unsigned sb = sa + p.a_bytes;
+          if (leader) {
           if (rank == 0) mbar_expect_tx(full0 + 8 * stage, tx_bytes);
           switch (p.kind) {
             case GK_FC_FWD:       // A [M][K] K-major, B [N][K] K-major
@@ -655,6 +663,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             kh0 + wg_r - p.pad, kbb0);
               break;
             }
+          }
           }
          }
           if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) {
