@@ -241,57 +241,87 @@ __device__ __forceinline__ void tc_ld32(unsigned taddr, int (&v)[32]) {
 
 // Shift-and-round of four accumulators (Algorithm 2 + 3, or round-to-nearest) packed into four int8.
 //
-// Pseudo-stochastic rule on a magnitude a with bp discarded bits (h = bp / 2, odd = bp & 1):
-// y = a >> odd drops the lowest bit when bp is odd; its low 2h bits are top * 2^h + bot, and the
-// integer part is incremented iff top > bot.  Adding C - bot * 2^h with C = 2^(2h) - 2^h carries
-// into bit 2h exactly in that case:  q = (y + C - (y & (2^h - 1)) * 2^h) >> 2h.
-// Round-to-nearest is the same expression with odd = 0, mask = 0, C = 2^(bp-1) (0 if bp = 0) and
-// a final shift by bp.  `orv` collects the OR of the magnitudes (same bit length as their maximum).
+// Pseudo-stochastic rule on a magnitude a with bp discarded bits (h = bp / 2, o = bp & 1): the lowest
+// bit is dropped when bp is odd; the next 2h bits are top * 2^h + bot and the integer part is
+// incremented iff top > bot.  With mask2 = (2^h - 1) << o the term (~a & mask2) is (2^h - 1 - bot) << o,
+// and adding it times 2^h carries into bit bp exactly when top > bot:
+//     q = (a + (~a & mask2) * 2^h) >> bp           (the dropped lowest bit cannot carry).
+// Round-to-nearest is the same expression with mask2 = 0 and the constant 2^(bp-1) in place of the
+// product.  Saturation at 2^mbits - 1 happens only when the integer part is already 2^mbits - 1, so
+// clamping the magnitude to cap = (2^mbits - 1) << bp beforehand gives the same result.
+//
+// The integer pipe of an SM issues one warp instruction every two cycles, and the epilogue of every
+// output element runs on it: the instruction count per element here bounds the layers with few
+// input channels.  ReLU outputs therefore never form |x|: max(min(x, cap), 0) is one instruction and
+// rounds negative inputs to zero by itself; the true extremes are tracked with three-input min/max.
 struct RoundConst {
-  int odd;        // pre-shift
-  unsigned mask;  // 2^h - 1
-  unsigned negp;  // -(2^h) as an unsigned multiplier
-  unsigned c;     // additive constant
-  int shift;      // final shift
-  unsigned qmax;  // saturation 2^mbits - 1
+  unsigned mask2;   // (2^h - 1) << o, or 0
+  unsigned orc;     // 0, or 1 for round-to-nearest with bp > 0
+  unsigned mulp;    // 2^h, or 2^(bp-1)
+  int shift;        // bp
+  int cap;          // (2^mbits - 1) << bp
 };
 __device__ __forceinline__ RoundConst make_round_const(int bp, int mbits, int round_mode) {
   RoundConst k;
-  k.qmax = (1u << mbits) - 1u;
+  k.shift = bp;
+  k.cap = (int)(((1u << mbits) - 1u) << bp);
   if (round_mode == NITI_ROUND_PSR) {
     const int h = bp >> 1;
-    k.odd = bp & 1;
-    k.mask = (1u << h) - 1u;
-    k.negp = 0u - (1u << h);
-    k.c = (1u << (2 * h)) - (1u << h);
-    k.shift = 2 * h;
+    k.mask2 = ((1u << h) - 1u) << (bp & 1);
+    k.orc = 0;
+    k.mulp = 1u << h;
   } else {
-    k.odd = 0;
-    k.mask = 0;
-    k.negp = 0;
-    k.c = bp > 0 ? 1u << (bp - 1) : 0u;
-    k.shift = bp;
+    k.mask2 = 0;
+    k.orc = bp > 0 ? 1u : 0u;
+    k.mulp = bp > 0 ? 1u << (bp - 1) : 0u;
   }
   return k;
 }
-__device__ __forceinline__ unsigned round_mag1(unsigned a, const RoundConst &k) {
-  const unsigned y = a >> k.odd;
-  const unsigned q = ((y & k.mask) * k.negp + (y + k.c)) >> k.shift;
-  return min(q, k.qmax);
+// magnitude already clamped to cap
+__device__ __forceinline__ unsigned round_mag1(unsigned m, const RoundConst &k) {
+  return ((((~m) & k.mask2) | k.orc) * k.mulp + m) >> k.shift;
 }
+// Extremes of the raw accumulators seen by one thread.
+struct Extremes {
+  int hi, lo;       // running max (>= 0) and min (<= 0)
+  unsigned orv;     // OR of magnitudes (same bit length as their maximum)
+  __device__ __forceinline__ unsigned magnitude_bits() const {
+    return orv | (unsigned)hi | (0u - (unsigned)lo);
+  }
+};
 template <bool RELU>
-__device__ __forceinline__ unsigned round_pack4(int x0, int x1, int x2, int x3, const RoundConst &k, unsigned &orv) {
-  const unsigned a0 = (unsigned)abs(x0), a1 = (unsigned)abs(x1), a2 = (unsigned)abs(x2), a3 = (unsigned)abs(x3);
-  orv |= a0 | a1;
-  orv |= a2 | a3;
-  unsigned q0 = round_mag1(a0, k), q1 = round_mag1(a1, k), q2 = round_mag1(a2, k), q3 = round_mag1(a3, k);
-  const unsigned s0 = (unsigned)(x0 >> 31), s1 = (unsigned)(x1 >> 31), s2 = (unsigned)(x2 >> 31), s3 = (unsigned)(x3 >> 31);
+__device__ __forceinline__ unsigned round_pack4(int x0, int x1, int x2, int x3, const RoundConst &k, Extremes &e) {
+  unsigned q0, q1, q2, q3;
   if (RELU) {
-    q0 &= ~s0; q1 &= ~s1; q2 &= ~s2; q3 &= ~s3;
+    e.hi = __vimax3_s32(e.hi, x0, x1);
+    e.hi = __vimax3_s32(e.hi, x2, x3);
+    e.lo = __vimin3_s32(e.lo, x0, x1);
+    e.lo = __vimin3_s32(e.lo, x2, x3);
+    q0 = round_mag1((unsigned)__vimin_s32_relu(x0, k.cap), k);
+    q1 = round_mag1((unsigned)__vimin_s32_relu(x1, k.cap), k);
+    q2 = round_mag1((unsigned)__vimin_s32_relu(x2, k.cap), k);
+    q3 = round_mag1((unsigned)__vimin_s32_relu(x3, k.cap), k);
   } else {
-    q0 = (q0 ^ s0) - s0; q1 = (q1 ^ s1) - s1; q2 = (q2 ^ s2) - s2; q3 = (q3 ^ s3) - s3;
+    const unsigned a0 = (unsigned)abs(x0), a1 = (unsigned)abs(x1), a2 = (unsigned)abs(x2), a3 = (unsigned)abs(x3);
+    e.orv |= a0 | a1;
+    e.orv |= a2 | a3;
+    const unsigned cap = (unsigned)k.cap;
+    q0 = round_mag1(min(a0, cap), k); q1 = round_mag1(min(a1, cap), k);
+    q2 = round_mag1(min(a2, cap), k); q3 = round_mag1(min(a3, cap), k);
+    // sign as a multiply by +-1: the multiply runs beside the integer pipe
+    q0 *= (unsigned)((x0 >> 31) | 1); q1 *= (unsigned)((x1 >> 31) | 1);
+    q2 *= (unsigned)((x2 >> 31) | 1); q3 *= (unsigned)((x3 >> 31) | 1);
   }
   return __byte_perm(__byte_perm(q0, q1, 0x4040), __byte_perm(q2, q3, 0x4040), 0x5410);
+}
+
+// 0xff in every byte of b that is greater than zero as a signed byte (the ReLU gate of the backward pass).
+__device__ __forceinline__ unsigned bytes_gt0(unsigned b) {
+  unsigned t = (b & 0x7f7f7f7fu) + 0x7f7f7f7fu;   // bit 7 of a byte: its low seven bits are not all zero
+  t = t & ~b & 0x80808080u;                       // ... and its sign bit is clear
+  unsigned r;
+  asm("prmt.b32 %0, %1, %1, 0xba98;" : "=r"(r) : "r"(t));   // replicate bit 7 over each byte
+  return r;
 }
 
 // Coordinates of an output tile / k-block in the pixel grid of a convolution.
@@ -1013,23 +1043,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tc_ld32(tm_row + (unsigned)c, v);
           if (row_ok && c < ncols_valid) {
             unsigned w8[8];
-            unsigned orv = 0;
+            Extremes ex = {0, 0, 0u};
             if (p.relu) {
 #pragma unroll
               for (int j = 0; j < 8; ++j)
-                w8[j] = round_pack4<true>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, orv);
+                w8[j] = round_pack4<true>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, ex);
             } else {
 #pragma unroll
               for (int j = 0; j < 8; ++j)
-                w8[j] = round_pack4<false>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, orv);
+                w8[j] = round_pack4<false>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, ex);
             }
             if (vec_ok && c + 32 <= ncols_valid) {
-              mx |= orv;
+              mx |= ex.magnitude_bits();
               if (msk) {
-                w8[0] &= __vcmpgts4(m0v.x, 0); w8[1] &= __vcmpgts4(m0v.y, 0);
-                w8[2] &= __vcmpgts4(m0v.z, 0); w8[3] &= __vcmpgts4(m0v.w, 0);
-                w8[4] &= __vcmpgts4(m1v.x, 0); w8[5] &= __vcmpgts4(m1v.y, 0);
-                w8[6] &= __vcmpgts4(m1v.z, 0); w8[7] &= __vcmpgts4(m1v.w, 0);
+                w8[0] &= bytes_gt0(m0v.x); w8[1] &= bytes_gt0(m0v.y);
+                w8[2] &= bytes_gt0(m0v.z); w8[3] &= bytes_gt0(m0v.w);
+                w8[4] &= bytes_gt0(m1v.x); w8[5] &= bytes_gt0(m1v.y);
+                w8[6] &= bytes_gt0(m1v.z); w8[7] &= bytes_gt0(m1v.w);
               }
               *reinterpret_cast<int4 *>(dst8 + c) = make_int4(w8[0], w8[1], w8[2], w8[3]);
               *reinterpret_cast<int4 *>(dst8 + c + 16) = make_int4(w8[4], w8[5], w8[6], w8[7]);
