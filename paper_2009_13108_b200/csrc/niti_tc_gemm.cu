@@ -38,6 +38,8 @@ struct TcParams {
   int kb_per_split;
   int splits;
   long long items;              // tiles * splits
+  int mrep;                     // 128-row tiles per item (row-batched mode of short contractions), else 1
+  int bn_mma;                   // N of one MMA; bn = mrep * bn_mma accumulator columns per item
   long long gm, gn;             // output extent (rows, columns); row pitch of acc is gn
   int bn;                       // tile width (multiple of 32, <= 256)
   int kdepth;                   // contraction elements per k-block (32, 64 or 128)
@@ -441,17 +443,24 @@ __device__ __forceinline__ void load4(unsigned dst, const CUtensorMap *m, unsign
 
 // item -> (row unit, column tile, split).  Row units (one CTA's 128 rows, or a pair's 256) are
 // visited in groups of raster_g so that the CTAs running at the same time share operand tiles in L2.
-__device__ __forceinline__ void decode_item(const TcParams &p, long long item, int &mu, int &nt, int &split) {
-  const long long tile = item / p.splits;
-  split = (int)(item % p.splits);
+// (32-bit arithmetic throughout: one thread of the producer, issuer and epilogue warps runs this per
+// tile, and 64-bit divisions there cost more than a small tile's whole multiply.)
+__device__ __forceinline__ void decode_item(const TcParams &p, int item, int &mu, int &nt, int &split) {
+  int tile = item;
+  split = 0;
+  if (p.splits > 1) {
+    tile = item / p.splits;
+    split = item - tile * p.splits;
+  }
   if (p.raster_g <= 0) {
-    mu = (int)(tile / p.n_tiles_n);
-    nt = (int)(tile % p.n_tiles_n);
+    if (p.n_tiles_n == 1) { mu = tile; nt = 0; return; }
+    mu = tile / p.n_tiles_n;
+    nt = tile - mu * p.n_tiles_n;
     return;
   }
-  const long long per_group = (long long)p.raster_g * p.n_tiles_n;
-  const int g = (int)(tile / per_group);
-  const int rem = (int)(tile % per_group);
+  const int per_group = p.raster_g * p.n_tiles_n;
+  const int g = tile / per_group;
+  const int rem = tile - g * per_group;
   int in_group = p.m_units - g * p.raster_g;
   if (in_group > p.raster_g) in_group = p.raster_g;
   mu = g * p.raster_g + rem % in_group;
@@ -501,10 +510,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const unsigned lead_full0 = CTAS == 2 ? map_to_cta(full0, 0) : full0;
   const unsigned lead_tempty0 = CTAS == 2 ? map_to_cta(tempty0, 0) : tempty0;
   // items of this CTA (pair): first_item, first_item + item_step, ... below item_end
-  long long first_item = blockIdx.x / CTAS, item_step = gridDim.x / CTAS, item_end = p.items;
+  int first_item = blockIdx.x / CTAS, item_step = gridDim.x / CTAS, item_end = (int)p.items;
   if (p.blocked) {
-    const long long units = gridDim.x / CTAS, u = blockIdx.x / CTAS;
-    const long long per = p.items / units, extra = p.items % units;
+    const int units = gridDim.x / CTAS, u = blockIdx.x / CTAS;
+    const int per = (int)p.items / units, extra = (int)p.items % units;
     first_item = u * per + (u < extra ? u : extra);
     item_end = first_item + per + (u < extra ? 1 : 0);
     item_step = 1;
@@ -566,8 +575,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bool ok = true;
       const int bn_cta = p.bn / CTAS;             // B rows (output columns) staged by this CTA
       if (p.halo == 2) {
-        for (long long item = first_item; ok && item < item_end; item += item_step) {
-          const int split = (int)(item % p.splits);
+        for (int item = first_item; ok && item < item_end; item += item_step) {
+          const int split = p.splits > 1 ? item % p.splits : 0;
           const int blk = (int)(item / p.splits);
           const int ci0 = (blk % p.wg_nci) * 64, co0 = (blk / p.wg_nci) * 64;
           const int t0 = split * p.kb_per_split;
@@ -606,7 +615,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // consecutive items are consecutive tiles (blocked assignment): step the tile coordinates
         int wt = (int)(first_item % p.w_tiles), ht = (int)((first_item / p.w_tiles) % p.h_tiles);
         int bt = (int)(first_item / ((long long)p.w_tiles * p.h_tiles));
-        for (long long item = first_item; ok && item < item_end; ++item) {
+        for (int item = first_item; ok && item < item_end; ++item) {
           if (stage % p.nprod == warp) {
             if (!mbar_wait_warp(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
             const unsigned full = full0 + 8 * stage;
@@ -620,7 +629,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         item_end = first_item;                    // nothing left for the generic loop
       }
-      for (long long item = first_item; ok && item < item_end; item += item_step) {
+      for (int item = first_item; ok && item < item_end; item += item_step) {
         int mu, nt, split;
         decode_item(p, item, mu, nt, split);
         const int mt = mu * CTAS + (int)rank;     // this CTA's 128-row tile
@@ -659,7 +668,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (rank == 0) mbar_expect_tx(full0 + 8 * stage, tx_bytes);
           switch (p.kind) {
             case GK_FC_FWD:       // A [M][K] K-major, B [N][K] K-major
-              load2<CTAS>(sa, &map_a, full, kb * p.kdepth, mt * BM);
+              for (int j = 0; j < p.mrep; ++j)     // rows past the end of A are zero-filled by the copy
+                load2<CTAS>(sa + j * p.a_box_bytes, &map_a, full, kb * p.kdepth, (mt * p.mrep + j) * BM);
               load2<CTAS>(sb, &map_b, full, kb * p.kdepth, nb);
               break;
             case GK_FC_DGRAD:     // A = e [M][N] K-major; B(k', n) = w[n][k'] MN-major
@@ -728,8 +738,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int lbo_rows = rb > ra ? rb - ra : 1;
           a_pair[pi] = (unsigned)(ra * 4) | ((unsigned)(lbo_rows * 4) << 16);     // 64-byte rows, 16-byte units
         }
-        for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
-          const int split = (int)(item % p.splits);
+        for (int item = first_item; ok && item < item_end; item += item_step, ++use) {
+          const int split = p.splits > 1 ? item % p.splits : 0;
           const int t0 = split * p.kb_per_split;
           int t1 = t0 + p.kb_per_split;
           if (t1 > p.kb_total) t1 = p.kb_total;
@@ -778,7 +788,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           a_off[tap] = (fwd_taps ? (unsigned)(r * 10 + t) : (unsigned)((2 - r) * 10 + (2 - t))) * row16;
           b_tap[tap] = b_lo0 + (unsigned)tap * btile16;
         }
-        for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
+        for (int item = first_item; ok && item < item_end; item += item_step, ++use) {
           const unsigned buf = use % (unsigned)p.nbuf;
           if (!mbar_wait_warp(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
           if (!mbar_wait_warp(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
@@ -800,9 +810,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const unsigned g_a_lo0 = (unsigned)p.a_desc, g_b_lo0 = (unsigned)p.b_desc;
       const unsigned g_a_hi = (unsigned)(p.a_desc >> 32), g_b_hi = (unsigned)(p.b_desc >> 32);
       const unsigned g_ak = p.a_kstep16, g_bk = p.b_kstep16, g_idesc = p.idesc, g_a_bytes = (unsigned)p.a_bytes;
-      const int g_ksteps = p.ksteps;
-      for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
-        const int split = (int)(item % p.splits);
+      const int g_ksteps = p.ksteps, g_mrep = p.mrep;
+      const unsigned g_bn_mma = (unsigned)p.bn_mma, g_slice16 = (unsigned)p.a_box_bytes >> 4;
+      for (int item = first_item; ok && item < item_end; item += item_step, ++use) {
+        const int split = p.splits > 1 ? item % p.splits : 0;
         const int kb0 = split * p.kb_per_split;
         int kb1 = kb0 + p.kb_per_split;
         if (kb1 > p.kb_total) kb1 = p.kb_total;
@@ -818,7 +829,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const unsigned a_lo = g_a_lo0 + ((sa >> 4) & 0x3fff), b_lo = g_b_lo0 + (((sa + g_a_bytes) >> 4) & 0x3fff);
           const unsigned first_acc = kb > kb0 ? 1u : 0u;
           if (leader) {
-            if (g_ksteps == 4) issue_kblock<CTAS, 4>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+            if (g_mrep > 1) {
+              for (int j = 0; j < g_mrep; ++j) {
+                const unsigned td = tmem_d + (unsigned)j * g_bn_mma, aj = a_lo + (unsigned)j * g_slice16;
+                if (g_ksteps == 1) issue_kblock<CTAS, 1>(td, aj, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+                else if (g_ksteps == 2) issue_kblock<CTAS, 2>(td, aj, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+                else if (g_ksteps == 4) issue_kblock<CTAS, 4>(td, aj, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+                else issue_kblock<CTAS, 3>(td, aj, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
+              }
+            }
+            else if (g_ksteps == 4) issue_kblock<CTAS, 4>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
             else if (g_ksteps == 2) issue_kblock<CTAS, 2>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
             else if (g_ksteps == 1) issue_kblock<CTAS, 1>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
             else issue_kblock<CTAS, 3>(tmem_d, a_lo, g_a_hi, b_lo, g_b_hi, g_ak, g_bk, g_idesc, first_acc);
@@ -853,7 +873,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       // lane = (tap of the pair, input channel), column = output channel; partial sums of this
       // CTA's pixel range are added to g32[co][tap][ci]
       const int which = row_in_tile >> 6, ci = row_in_tile & 63;
-      for (long long item = first_item; ok && item < item_end; item += item_step, ++use) {
+      for (int item = first_item; ok && item < item_end; item += item_step, ++use) {
         const int blk = (int)(item / p.splits);
         const int ci0 = (blk % p.wg_nci) * 64, co0 = (blk / p.wg_nci) * 64;
         if (!mbar_wait(tfull0, use & 1u, &abort_flag, status)) { ok = false; break; }
@@ -877,7 +897,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       item_end = first_item;
     }
     use = (unsigned)egroup;
-    for (long long item = first_item + egroup * item_step; ok && item < item_end;
+    for (int item = first_item + egroup * item_step; ok && item < item_end;
          item += item_step * egroups, use += (unsigned)egroups) {
       int mu = 0, nt = 0, split = 0;
       if (!p.halo) decode_item(p, item, mu, nt, split);
@@ -921,7 +941,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int rem = p.Cn - ci0;
         ncols_valid = rem < p.bn ? rem : p.bn;
       } else {
-        out_row = (long long)mt * BM + row_in_tile;
+        // (row-batched mode: the row of the first of the item's mrep tiles; column chunk c of the
+        // accumulator then belongs to tile c / bn_mma)
+        out_row = (long long)mt * (BM * p.mrep) + row_in_tile;
         row_ok = out_row < p.gm;
         col0 = (long long)nt * p.bn;
         long long rem = p.gn - col0;
@@ -985,10 +1007,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
             int v[32];
             tc_ld32(tm_row + (unsigned)c, v);
-            if (row_ok) {
+            int cc = c;
+            bool rok = row_ok;
+            if (p.mrep > 1) {
+              const int jt = c / p.bn_mma;
+              cc = c - jt * p.bn_mma;
+              rok = out_row + (long long)jt * BM < p.gm;
+            }
+            if (rok) {
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                if (c + j < ncols_valid) {
+                if (cc + j < ncols_valid) {
                   unsigned a = v[j] < 0 ? 0u - (unsigned)v[j] : (unsigned)v[j];
                   m0 = a > m0 ? a : m0;
                 }
@@ -1027,21 +1056,31 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (blockIdx.x == 0 && warp == EPI_WARP0 && lane == 0) hdr->spec_b = (unsigned)b;
           if (lane == 0) spec_bp_ready = bp + 1;
         }
-        int8_t *dst8 = out8 + out_row * p.gn + col0;
-        const int8_t *msk = mask8 ? mask8 + out_row * p.gn + col0 : nullptr;
         const bool vec_ok = ((p.gn & 15) == 0) && ((col0 & 15) == 0);
         const RoundConst rk = make_round_const(bp, p.mbits, p.round_mode);
         for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
           int v[32];
+          // chunk geometry: in row-batched mode chunk c holds columns cc of the item's tile c / bn_mma
+          int cc = c;
+          long long orow = out_row;
+          bool rok = row_ok;
+          if (p.mrep > 1) {
+            const int jt = c / p.bn_mma;
+            cc = c - jt * p.bn_mma;
+            orow = out_row + (long long)jt * BM;
+            rok = orow < p.gm;
+          }
+          int8_t *dst8 = out8 + orow * p.gn + col0;
+          const int8_t *msk = mask8 ? mask8 + orow * p.gn + col0 : nullptr;
           // the ReLU mask bytes are fetched first so that their latency overlaps the TMEM load and
           // the rounding arithmetic
           int4 m0v = make_int4(0x01010101, 0x01010101, 0x01010101, 0x01010101), m1v = m0v;
-          if (msk && vec_ok && row_ok && c + 32 <= ncols_valid) {
-            m0v = *reinterpret_cast<const int4 *>(msk + c);
-            m1v = *reinterpret_cast<const int4 *>(msk + c + 16);
+          if (msk && vec_ok && rok && cc + 32 <= ncols_valid) {
+            m0v = *reinterpret_cast<const int4 *>(msk + cc);
+            m1v = *reinterpret_cast<const int4 *>(msk + cc + 16);
           }
           tc_ld32(tm_row + (unsigned)c, v);
-          if (row_ok && c < ncols_valid) {
+          if (rok && cc < ncols_valid) {
             unsigned w8[8];
             Extremes ex = {0, 0, 0u};
             if (p.relu) {
@@ -1053,7 +1092,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               for (int j = 0; j < 8; ++j)
                 w8[j] = round_pack4<false>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, ex);
             }
-            if (vec_ok && c + 32 <= ncols_valid) {
+            if (vec_ok && cc + 32 <= ncols_valid) {
               mx |= ex.magnitude_bits();
               if (msk) {
                 w8[0] &= bytes_gt0(m0v.x); w8[1] &= bytes_gt0(m0v.y);
@@ -1061,16 +1100,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 w8[4] &= bytes_gt0(m1v.x); w8[5] &= bytes_gt0(m1v.y);
                 w8[6] &= bytes_gt0(m1v.z); w8[7] &= bytes_gt0(m1v.w);
               }
-              *reinterpret_cast<int4 *>(dst8 + c) = make_int4(w8[0], w8[1], w8[2], w8[3]);
-              *reinterpret_cast<int4 *>(dst8 + c + 16) = make_int4(w8[4], w8[5], w8[6], w8[7]);
+              *reinterpret_cast<int4 *>(dst8 + cc) = make_int4(w8[0], w8[1], w8[2], w8[3]);
+              *reinterpret_cast<int4 *>(dst8 + cc + 16) = make_int4(w8[4], w8[5], w8[6], w8[7]);
             } else {
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                if (c + j < ncols_valid) {
+                if (cc + j < ncols_valid) {
                   mx |= (unsigned)abs(v[j]);
                   int8_t q = (int8_t)((w8[j >> 2] >> (8 * (j & 3))) & 0xff);
-                  if (msk && msk[c + j] <= 0) q = 0;
-                  dst8[c + j] = q;
+                  if (msk && msk[cc + j] <= 0) q = 0;
+                  dst8[cc + j] = q;
                 }
             }
           }
@@ -1434,6 +1473,18 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
     p.a_desc = desc_kmajor(a_sw);
     p.a_kstep16 = 2;
   }
+  // Row-batched mode: a multiply with one or two k-blocks and a narrow output (the gathered first
+  // layer: K = 32, N = 64) is all per-tile bookkeeping.  One item then covers mrep 128-row tiles: one
+  // stage holds their A boxes, one MMA per tile writes its own bn_mma columns of the accumulator,
+  // and the barriers, commits and tile decoding are paid once per item.
+  p.mrep = 1;
+  if (g.kind == GK_FC_FWD && ctas == 1 && ctx->engine != 4 && p.n_tiles_n == 1 && p.kb_total <= 2 && p.bn <= 128 &&
+      m_tiles >= 8LL * ctx->sm_count) {
+    p.mrep = p.bn <= 64 ? 4 : 2;
+    p.a_boxes = p.mrep;
+    p.a_bytes = p.mrep * p.a_box_bytes;
+    m_tiles = (m_tiles + p.mrep - 1) / p.mrep;
+  }
   const int bn_cta = p.bn / ctas;               // output columns staged by each CTA
   if (bn_cta % 16) return false;
   if (b_mn) {
@@ -1470,6 +1521,8 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
   // instruction descriptor: s32 accumulate, signed 8-bit operands, majorness, N, M
   p.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((unsigned)a_mn << 15) | ((unsigned)b_mn << 16) |
             ((unsigned)(p.bn >> 3) << 17) | ((unsigned)((BM * ctas) >> 4) << 24);
+  p.bn_mma = p.bn;
+  p.bn *= p.mrep;
   p.m_units = (int)((m_tiles + ctas - 1) / ctas);
   long long tiles = (long long)p.m_units * p.n_tiles_n;
   const int units = ctx->sm_count / ctas;       // CTAs (or CTA pairs) that run at the same time
@@ -1514,6 +1567,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
   // first tile of every CTA an even sample of the tensor for the speculative shift
   p.blocked = (g.kind == GK_CONV_FWD || g.kind == GK_CONV_DGRAD) ? 1 : 0;
   p.items = tiles * p.splits;
+  if (p.items >= (1LL << 30)) return false;      // the kernel counts items in 32 bits
   if (!encode(ctx, &ma, sa) || !encode(ctx, &mb, sb)) return false;
   return true;
 }
@@ -1605,6 +1659,8 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
   if ((g.kind == GK_CONV_FWD || g.kind == GK_CONV_DGRAD || g.kind == GK_CONV_WGRAD) && ctx->engine != 3 &&
       ctx->engine != 5)
     planned = plan(ctx, g, 1, true, p, ma, mb) && p.halo;
+  if (!planned && g.kind == GK_FC_FWD && ctx->engine != 3)      // row-batched mode of short contractions
+    planned = plan(ctx, g, 1, false, p, ma, mb) && p.mrep > 1;
   if (!planned && ctx->engine != 2 && g.gm >= 2 * BM) {
     planned = plan(ctx, g, 2, false, p, ma, mb);
     if (planned && ctx->engine != 3 && p.items < ctx->sm_count / 2) planned = false;

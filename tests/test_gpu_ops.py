@@ -55,6 +55,23 @@ def test_linear_fwd(niti, oref, M, N, K, engine):
     niti.check()
 
 
+# Many rows, a contraction of one or two k-blocks and a narrow output: the engine batches several
+# 128-row tiles per work item (the shape of the gathered RGB first layer).  M is not a multiple of
+# the batch (4 x 128 rows) nor of 128, so the last item has missing tiles and a ragged one.
+@pytest.mark.parametrize("M,N,K", [(152000 + 77, 64, 32), (152000 + 300, 48, 200), (152000 + 513, 128, 96),
+                                   (152000, 20, 32)])
+def test_linear_fwd_row_batched(niti, oref, M, N, K):
+    rng = np.random.default_rng(M + N + K)
+    a, w = _i8(rng, (M, K)), _i8(rng, (N, K))
+    for relu, mode in [(True, 0), (False, 1)]:
+        want, s, b = oref.linear_fwd(a, -7, w, -10, relu, mode)
+        out, s_out, b_out = niti.linear_fwd(_T(niti, a), niti.scalar(-7), _T(niti, w),
+                                            niti.scalar(-10), relu=relu, round_mode=mode)
+        _eq(out, want)
+        assert (int(s_out), int(b_out)) == (s, b)
+    niti.check()
+
+
 @pytest.mark.parametrize("engine", [0, 1, 2, 3, 4])
 @pytest.mark.parametrize("M,N,K", FC_SHAPES[:7] + [(640, 256, 512)])
 def test_linear_bwd(niti, oref, M, N, K, engine):
