@@ -262,11 +262,14 @@ struct RoundConst {
   unsigned mulp;    // 2^h, or 2^(bp-1)
   int shift;        // bp
   int cap;          // (2^mbits - 1) << bp
+  unsigned hi_mul;  // 2^(32 - bp) for bp > 0: the high half of v * hi_mul is v >> bp, a multiply
+                    // instead of a shift because the multiplier pipe has the spare issue slots
 };
 __device__ __forceinline__ RoundConst make_round_const(int bp, int mbits, int round_mode) {
   RoundConst k;
   k.shift = bp;
   k.cap = (int)(((1u << mbits) - 1u) << bp);
+  k.hi_mul = bp > 0 ? 1u << (32 - bp) : 0u;
   if (round_mode == NITI_ROUND_PSR) {
     const int h = bp >> 1;
     k.mask2 = ((1u << h) - 1u) << (bp & 1);
@@ -280,8 +283,10 @@ __device__ __forceinline__ RoundConst make_round_const(int bp, int mbits, int ro
   return k;
 }
 // magnitude already clamped to cap
+template <bool SHIFT>
 __device__ __forceinline__ unsigned round_mag1(unsigned m, const RoundConst &k) {
-  return ((((~m) & k.mask2) | k.orc) * k.mulp + m) >> k.shift;
+  const unsigned v = (((~m) & k.mask2) | k.orc) * k.mulp + m;
+  return SHIFT ? __umulhi(v, k.hi_mul) : v;
 }
 // Extremes of the raw accumulators seen by one thread.
 struct Extremes {
@@ -291,7 +296,7 @@ struct Extremes {
     return orv | (unsigned)hi | (0u - (unsigned)lo);
   }
 };
-template <bool RELU>
+template <bool RELU, bool SHIFT>
 __device__ __forceinline__ unsigned round_pack4(int x0, int x1, int x2, int x3, const RoundConst &k, Extremes &e) {
   unsigned q0, q1, q2, q3;
   if (RELU) {
@@ -299,22 +304,44 @@ __device__ __forceinline__ unsigned round_pack4(int x0, int x1, int x2, int x3, 
     e.hi = __vimax3_s32(e.hi, x2, x3);
     e.lo = __vimin3_s32(e.lo, x0, x1);
     e.lo = __vimin3_s32(e.lo, x2, x3);
-    q0 = round_mag1((unsigned)__vimin_s32_relu(x0, k.cap), k);
-    q1 = round_mag1((unsigned)__vimin_s32_relu(x1, k.cap), k);
-    q2 = round_mag1((unsigned)__vimin_s32_relu(x2, k.cap), k);
-    q3 = round_mag1((unsigned)__vimin_s32_relu(x3, k.cap), k);
-  } else {
-    const unsigned a0 = (unsigned)abs(x0), a1 = (unsigned)abs(x1), a2 = (unsigned)abs(x2), a3 = (unsigned)abs(x3);
-    e.orv |= a0 | a1;
-    e.orv |= a2 | a3;
-    const unsigned cap = (unsigned)k.cap;
-    q0 = round_mag1(min(a0, cap), k); q1 = round_mag1(min(a1, cap), k);
-    q2 = round_mag1(min(a2, cap), k); q3 = round_mag1(min(a3, cap), k);
-    // sign as a multiply by +-1: the multiply runs beside the integer pipe
-    q0 *= (unsigned)((x0 >> 31) | 1); q1 *= (unsigned)((x1 >> 31) | 1);
-    q2 *= (unsigned)((x2 >> 31) | 1); q3 *= (unsigned)((x3 >> 31) | 1);
+    q0 = round_mag1<SHIFT>((unsigned)__vimin_s32_relu(x0, k.cap), k);
+    q1 = round_mag1<SHIFT>((unsigned)__vimin_s32_relu(x1, k.cap), k);
+    q2 = round_mag1<SHIFT>((unsigned)__vimin_s32_relu(x2, k.cap), k);
+    q3 = round_mag1<SHIFT>((unsigned)__vimin_s32_relu(x3, k.cap), k);
+    // values below 2^7: bytes assembled with multiply-adds
+    return (q1 * 0x100u + q0) + (q3 * 0x1000000u + q2 * 0x10000u);
   }
+  const unsigned a0 = (unsigned)abs(x0), a1 = (unsigned)abs(x1), a2 = (unsigned)abs(x2), a3 = (unsigned)abs(x3);
+  e.orv |= a0 | a1;
+  e.orv |= a2 | a3;
+  const unsigned cap = (unsigned)k.cap;
+  q0 = round_mag1<SHIFT>(min(a0, cap), k); q1 = round_mag1<SHIFT>(min(a1, cap), k);
+  q2 = round_mag1<SHIFT>(min(a2, cap), k); q3 = round_mag1<SHIFT>(min(a3, cap), k);
+  // sign as a multiply by +-1: the multiply runs beside the integer pipe
+  q0 *= (unsigned)((x0 >> 31) | 1); q1 *= (unsigned)((x1 >> 31) | 1);
+  q2 *= (unsigned)((x2 >> 31) | 1); q3 *= (unsigned)((x3 >> 31) | 1);
   return __byte_perm(__byte_perm(q0, q1, 0x4040), __byte_perm(q2, q3, 0x4040), 0x5410);
+}
+// all four variants behind one call: relu and "bp > 0" are the same for every element of a pass
+__device__ __forceinline__ void round_chunk32(const int (&v)[32], unsigned (&w8)[8], const RoundConst &k, bool relu,
+                                              Extremes &e) {
+  if (relu) {
+    if (k.shift > 0) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) w8[j] = round_pack4<true, true>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], k, e);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) w8[j] = round_pack4<true, false>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], k, e);
+    }
+  } else {
+    if (k.shift > 0) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) w8[j] = round_pack4<false, true>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], k, e);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) w8[j] = round_pack4<false, false>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], k, e);
+    }
+  }
 }
 
 // 0xff in every byte of b that is greater than zero as a signed byte (the ReLU gate of the backward pass).
@@ -1083,15 +1110,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (rok && cc < ncols_valid) {
             unsigned w8[8];
             Extremes ex = {0, 0, 0u};
-            if (p.relu) {
-#pragma unroll
-              for (int j = 0; j < 8; ++j)
-                w8[j] = round_pack4<true>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, ex);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 8; ++j)
-                w8[j] = round_pack4<false>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, ex);
-            }
+            round_chunk32(v, w8, rk, p.relu != 0, ex);
             if (vec_ok && cc + 32 <= ncols_valid) {
               mx |= ex.magnitude_bits();
               if (msk) {
