@@ -157,10 +157,12 @@ def test_speculative_shift_is_corrected(niti, oref, engine):
     want, s, b = oref.linear_fwd(a, -7, w, -10, True)
     niti.set_engine(engine)
     try:
+        redo0 = niti.redo_count()
         out, s_out, b_out = niti.linear_fwd(_T(niti, a), niti.scalar(-7), _T(niti, w),
                                             niti.scalar(-10), relu=True)
         _eq(out, want)
         assert (int(s_out), int(b_out)) == (s, b)
+        assert niti.redo_count() > redo0, "the second pass did not run: the case no longer tests it"
         # and the mirrored case through the masked dgrad epilogue
         e = rng.integers(-2, 3, size=(M, N), dtype=np.int8)
         e[-3:] = 127
@@ -172,6 +174,33 @@ def test_speculative_shift_is_corrected(niti, oref, engine):
         assert (int(b_e), int(b_g)) == (be, bg)
     finally:
         niti.set_engine(0)
+    niti.check()
+
+
+def test_speculative_shift_is_corrected_in_conv_and_row_batched_modes(niti, oref):
+    """Same for the resident-weights convolution (small channel counts) and for the row-batched
+    multiply of short contractions: only the end of the tensor is large."""
+    rng = np.random.default_rng(78)
+    B, H, W, C = 40, 32, 32, 64
+    x = rng.integers(-3, 4, size=(B, H, W, C), dtype=np.int8)
+    x[-1, -4:, -8:] = rng.integers(100, 128, size=(4, 8, C), dtype=np.int8)   # inside the last 8x16 tile only
+    w = rng.integers(64, 128, size=(C, 3, 3, C), dtype=np.int8)
+    want, s, b = oref.conv_fwd(x, -7, w, -9, 1, True)
+    redo0 = niti.redo_count()
+    y, s_y, b_y = niti.conv_fwd(_T(niti, x), niti.scalar(-7), _T(niti, w), niti.scalar(-9), relu=True)
+    _eq(y, want)
+    assert (int(s_y), int(b_y)) == (s, b)
+    assert niti.redo_count() > redo0
+    M, N, K = 152000 + 130, 64, 32
+    a = rng.integers(-3, 4, size=(M, K), dtype=np.int8)
+    a[-5:] = rng.integers(100, 128, size=(5, K), dtype=np.int8)
+    wf = rng.integers(64, 128, size=(N, K), dtype=np.int8)
+    want, s, b = oref.linear_fwd(a, -7, wf, -10, False)
+    redo0 = niti.redo_count()
+    out, s_out, b_out = niti.linear_fwd(_T(niti, a), niti.scalar(-7), _T(niti, wf), niti.scalar(-10))
+    _eq(out, want)
+    assert (int(s_out), int(b_out)) == (s, b)
+    assert niti.redo_count() > redo0
     niti.check()
 
 
