@@ -308,6 +308,47 @@ def run_elementwise(args):
     niti.check()
 
 
+def run_per_launch(args):
+    """One eager training step of the chosen config with a CUDA event pair around every tensor-core
+    multiply (the library's own profiling hooks): one text line per multiply, in launch order."""
+    import torch
+    from paper_2009_13108_b200 import Niti, NitiTrainer
+    from synth import config_net, make_net_inputs
+    niti = Niti(0)
+    net = config_net(args.config)
+    x, labels, weights = make_net_inputs(net)
+    tr = NitiTrainer(niti, net, weights)
+    tr.load_batch(x, labels)
+    tr.snapshot_weights()
+    for _ in range(2):
+        tr.reset_weights()
+        tr.step()
+    torch.cuda.synchronize()
+    redo0 = niti.redo_count()
+    niti.profile_enable(True)
+    e0, e1 = torch.cuda.Event(True), torch.cuda.Event(True)
+    tr.reset_weights()
+    e0.record()
+    tr.step()
+    e1.record()
+    torch.cuda.synchronize()
+    launches = niti.profile_read_launches()
+    wl = [(i, l) for i, l in enumerate(net.layers) if l["op"] != "pool"]
+    names = ["fwd   L%d %s" % (i, l["op"]) for i, l in wl]
+    for i, l in reversed(wl):
+        names.append("wgrad L%d %s" % (i, l["op"]))
+        if i != wl[0][0]:
+            names.append("dgrad L%d %s" % (i, l["op"]))
+    print("eager step %.3f ms, second passes in the step: %d" % (e0.elapsed_time(e1), niti.redo_count() - redo0))
+    total = 0.0
+    for k, (ms, ops) in enumerate(launches):
+        total += ms
+        name = names[k] if len(names) == len(launches) else ""
+        print("%3d %-18s %8.1f us %7.0f TOP/s %8.1f Gop" % (k, name, ms * 1e3, ops / ms / 1e9, ops / 1e9))
+    print("tensor-core multiplies: %.3f ms in %d launches" % (total, len(launches)))
+    niti.check()
+
+
 def run_ours(args):
     import torch
     rank = int(os.environ.get("RANK", "0"))
@@ -465,6 +506,8 @@ def main():
     ap.add_argument("--paper-table", action="store_true",
                     help="time the conv layer of the paper's timing table (fwd / dgrad / wgrad, five input sizes)")
     ap.add_argument("--elementwise", action="store_true", help="achieved GB/s of the HBM-bound kernels")
+    ap.add_argument("--per-launch", action="store_true",
+                    help="one eager step with a CUDA event pair around every tensor-core multiply")
     ap.add_argument("--full-sweep", action="store_true", help="with --sweep: time the second operand set on every shape")
     args = ap.parse_args()
     if args.sweep:
@@ -475,6 +518,9 @@ def main():
         return
     if args.elementwise:
         run_elementwise(args)
+        return
+    if args.per_launch:
+        run_per_launch(args)
         return
     if args.gemm_shape:
         from paper_2009_13108_b200 import Niti

@@ -199,10 +199,10 @@ int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const int32_t *s
  * that forbids allocator calls after start-up, a host process that has already handed all device
  * memory to its own pool, or a plug-in that is given tensors and a stream but no allocator.  Such
  * a caller cannot create a context (niti_create allocates the status word) nor a workspace, so
- * this call takes neither: its scratch (256 bytes of reduction scalars + 8 bytes per logit) lives
- * in a fixed array inside the library image, NITI_XENT_NOALLOC_MAX_ELEMS logits at most
- * (B * N <= 65536, i.e. 512 KiB + 256 B that every GPU loading the library holds until exit).
- * Larger B * N returns NITI_ERR_TOO_LARGE and enqueues nothing.
+ * this call takes neither: its scratch (256 bytes of reduction scalars + 16 bytes per sample)
+ * lives in a fixed array inside the library image of 512 KiB + 256 B, which every GPU loading the
+ * library holds until exit.  Limits: B * N <= NITI_XENT_NOALLOC_MAX_ELEMS (65536 logits) and
+ * B <= 32768; anything larger returns NITI_ERR_TOO_LARGE and enqueues nothing.
  *
  * a, labels, e, s_a, b_e, n_correct: device pointers as in niti_int_xent (b_e, n_correct may be
  * NULL); `stream` is the caller's cudaStream_t.  The call allocates nothing and frees nothing.  The

@@ -211,7 +211,7 @@ extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
     }
     case NITI_OP_INT_XENT:
       if (nd != 2 || d[0] <= 0 || d[1] <= 0) return 0;
-      return NITI_WS_HEADER + round_up((size_t)(d[0] * d[1]) * 8, 256);
+      return NITI_WS_HEADER + round_up((size_t)d[0] * 16, 256);   // two 64-bit scalars per sample
     default:
       return 0;
   }

@@ -243,116 +243,149 @@ int niti_launch_round_compact32(niti_ctx *ctx, cudaStream_t st, const int32_t *a
 }
 
 // ---------------------------------------------------------------------------------------------
-// Integer cross-entropy gradient, Section 3.5.  Pass 1: one block per sample computes the integer
-// T_i (Eq. 2 or Eq. 3-4), their sum, e32 = T_i - [i == label] * sum (64-bit), the tensor-wide
-// max magnitude, and the arg-max hit count.  Pass 2: shared binary point, rounding to int8.
+// Integer cross-entropy gradient, Section 3.5.  Pass 1: one warp per sample computes the integer
+// T_i (Eq. 2 or Eq. 3-4), their sum, the largest magnitude of e32 = T_i - [i == label] * sum
+// (64-bit) and the arg-max hit.  Pass 2: shared binary point, e32 recomputed and rounded to int8.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ long long block_reduce_ll(long long v, int op /*0 sum,1 max,2 min*/,
-                                                     long long *sh) {
+// One warp per sample.  Pass 1 keeps two 64-bit scalars per sample (the offset p of Eq. 4 and the
+// sum of the T_i) instead of the T_i themselves; pass 2 recomputes T_i from the logit, which is a few
+// integer operations, so that the only per-element traffic is the logit read twice and the int8
+// result written once.
+__device__ __forceinline__ long long warp_reduce_ll(long long v, int op /*0 sum,1 max,2 min*/) {
   for (int o = 16; o > 0; o >>= 1) {
     long long u = __shfl_xor_sync(0xffffffffu, v, o);
     v = op == 0 ? v + u : (op == 1 ? (u > v ? u : v) : (u < v ? u : v));
   }
-  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
-  __syncthreads();
-  if (lane == 0) sh[warp] = v;
-  __syncthreads();
-  long long r = sh[0];
-  for (int i = 1; i < nw; ++i) {
-    long long u = sh[i];
-    r = op == 0 ? r + u : (op == 1 ? (u > r ? u : r) : (u < r ? u : r));
-  }
-  return r;
+  return v;
 }
+// x-hat of Eq. 3: (47274 * a) >> (15 - s), a left shift when s > 15
+__device__ __forceinline__ long long xent_xhat(int a, long long sh_amt) {
+  const long long P = 47274LL * (long long)a;
+  return sh_amt >= 0 ? (P >> sh_amt) : P * (1LL << (-sh_amt));
+}
+// T_i of Eq. 2 (s <= -7) or Eq. 4
+__device__ __forceinline__ long long xent_T(int a, int s, long long sh_amt, long long p) {
+  if (s <= -7) {
+    const long long ai = a;
+    return (1LL << (1 - 2 * s)) + ai * (1LL << (1 - s)) + ai * ai;
+  }
+  const long long xt = xent_xhat(a, sh_amt) - p;
+  return 1LL << (xt > 0 ? xt : 0);
+}
+constexpr int XENT_WARPS = 8;
 
-__global__ void __launch_bounds__(256)
-xent_acc_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
-                const int32_t *__restrict__ labels, long long *__restrict__ e64, WsHeader *hdr,
-                int32_t *__restrict__ n_correct, int N, uint32_t *__restrict__ status) {
-  __shared__ long long sh[8];
-  const int r = blockIdx.x;
+__global__ void __launch_bounds__(32 * XENT_WARPS)
+xent_row_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
+                const int32_t *__restrict__ labels, long long *__restrict__ rowinfo, WsHeader *hdr,
+                int32_t *__restrict__ n_correct, int B, int N, uint32_t *__restrict__ status) {
+  __shared__ unsigned long long sh_max[XENT_WARPS];
+  __shared__ int sh_hit[XENT_WARPS];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = blockIdx.x * XENT_WARPS + warp;
   const int s = *s_a_ptr;
-  const int label = labels[r];
-  const int8_t *row = a + (long long)r * N;
-  long long *erow = e64 + (long long)r * N;
-  if (s < -22 || s > 24 || label < 0 || label >= N) {
-    if (threadIdx.x == 0) atomicOr(status, (s < -22 || s > 24) ? NITI_DEV_XENT_RANGE : NITI_DEV_BAD_LABEL);
-    for (int i = threadIdx.x; i < N; i += blockDim.x) erow[i] = 0;
-    return;
-  }
-  const long long LLMIN = -0x7fffffffffffffffLL - 1, LLMAX = 0x7fffffffffffffffLL;
-  long long mx = LLMIN;
-  long long sh_amt = 15 - (long long)s;
-  if (s > -7) {
-    for (int i = threadIdx.x; i < N; i += blockDim.x) {
-      long long P = 47274LL * (long long)row[i];
-      long long xh = sh_amt >= 0 ? (P >> sh_amt) : P * (1LL << (-sh_amt));
-      mx = xh > mx ? xh : mx;
-    }
-    mx = block_reduce_ll(mx, 1, sh);
-  }
-  long long p = LLMAX;
-  if (s > -7) {
-    for (int i = threadIdx.x; i < N; i += blockDim.x) {
-      long long P = 47274LL * (long long)row[i];
-      long long xh = sh_amt >= 0 ? (P >> sh_amt) : P * (1LL << (-sh_amt));
-      if (xh > mx - 10 && xh < p) p = xh;
-    }
-    p = block_reduce_ll(p, 2, sh);
-  }
-  // T_i and their sum; also the first arg-max of the row for the hit count
-  long long csum = 0;
-  int best_v = -1000, best_i = 0x7fffffff;
-  for (int i = threadIdx.x; i < N; i += blockDim.x) {
-    long long ai = row[i];
-    long long T;
-    if (s <= -7) {
-      T = (1LL << (1 - 2 * s)) + ai * (1LL << (1 - s)) + ai * ai;
+  unsigned long long row_max = 0;
+  int hit = 0;
+  if (r < B) {
+    const int label = labels[r];
+    const int8_t *row = a + (long long)r * N;
+    if (s < -22 || s > 24 || label < 0 || label >= N) {
+      if (lane == 0) {
+        atomicOr(status, (s < -22 || s > 24) ? NITI_DEV_XENT_RANGE : NITI_DEV_BAD_LABEL);
+        rowinfo[2 * (long long)r] = 0;
+        rowinfo[2 * (long long)r + 1] = 0;
+      }
     } else {
-      long long P = 47274LL * ai;
-      long long xh = sh_amt >= 0 ? (P >> sh_amt) : P * (1LL << (-sh_amt));
-      long long xt = xh - p;
-      T = 1LL << (xt > 0 ? xt : 0);
+      const long long LLMIN = -0x7fffffffffffffffLL - 1, LLMAX = 0x7fffffffffffffffLL;
+      const long long sh_amt = 15 - (long long)s;
+      long long p = 0;
+      if (s > -7) {
+        long long mx = LLMIN;
+        for (int i = lane; i < N; i += 32) {
+          const long long xh = xent_xhat(row[i], sh_amt);
+          mx = xh > mx ? xh : mx;
+        }
+        mx = warp_reduce_ll(mx, 1);
+        p = LLMAX;
+        for (int i = lane; i < N; i += 32) {
+          const long long xh = xent_xhat(row[i], sh_amt);
+          if (xh > mx - 10 && xh < p) p = xh;
+        }
+        p = warp_reduce_ll(p, 2);
+      }
+      // sum of T_i, the largest T_i off the label, and the first arg-max of the row for the hit count
+      long long csum = 0, t_other = 0;
+      int best_v = -1000, best_i = 0x7fffffff;
+      for (int i = lane; i < N; i += 32) {
+        const int ai = row[i];
+        const long long T = xent_T(ai, s, sh_amt, p);
+        csum += T;
+        if (i != label && T > t_other) t_other = T;
+        if (ai > best_v) { best_v = ai; best_i = i; }
+      }
+      csum = warp_reduce_ll(csum, 0);
+      t_other = warp_reduce_ll(t_other, 1);
+      long long key = ((long long)(best_v + 1000) << 32) | (unsigned)(0x7fffffff - best_i);
+      key = warp_reduce_ll(key, 1);
+      // e32 = T_i off the label (positive) and T_label - sum (not positive) on it
+      const long long t_label = xent_T(row[label], s, sh_amt, p);
+      const long long on_label = csum - t_label;
+      row_max = (unsigned long long)(t_other > on_label ? t_other : on_label);
+      hit = (0x7fffffff - (int)(key & 0xffffffffLL)) == label ? 1 : 0;
+      if (lane == 0) {
+        rowinfo[2 * (long long)r] = p;
+        rowinfo[2 * (long long)r + 1] = csum;
+      }
     }
-    erow[i] = T;
-    csum += T;
-    if ((int)ai > best_v) { best_v = (int)ai; best_i = i; }
   }
-  csum = block_reduce_ll(csum, 0, sh);
-  // first arg-max: maximise (value, -index)
-  long long key = ((long long)(best_v + 1000) << 32) | (unsigned)(0x7fffffff - best_i);
-  key = block_reduce_ll(key, 1, sh);
+  if (lane == 0) { sh_max[warp] = row_max; sh_hit[warp] = hit; }
   __syncthreads();
-  unsigned long long lmax = 0;
-  for (int i = threadIdx.x; i < N; i += blockDim.x) {
-    long long v = erow[i] - (i == label ? csum : 0);
-    erow[i] = v;
-    unsigned long long m = v < 0 ? 0ull - (unsigned long long)v : (unsigned long long)v;
-    lmax = m > lmax ? m : lmax;
-  }
-  long long bm = block_reduce_ll((long long)lmax, 1, sh);
   if (threadIdx.x == 0) {
-    atomicMax(&hdr->maxabs64, (unsigned long long)bm);
-    if (n_correct) {
-      int arg = 0x7fffffff - (int)(key & 0xffffffffLL);
-      if (arg == label) atomicAdd(n_correct, 1);
-    }
+    unsigned long long m = 0;
+    int h = 0;
+    for (int w = 0; w < XENT_WARPS; ++w) { m = sh_max[w] > m ? sh_max[w] : m; h += sh_hit[w]; }
+    if (m > *(volatile unsigned long long *)&hdr->maxabs64) atomicMax(&hdr->maxabs64, m);
+    if (n_correct && h) atomicAdd(n_correct, h);
   }
 }
 
-__global__ void __launch_bounds__(256)
-round_i64_kernel(const long long *__restrict__ e64, const WsHeader *__restrict__ hdr,
-                 int8_t *__restrict__ out, long long n, int round_mode, int32_t *__restrict__ b_out) {
-  unsigned long long mxv = hdr->maxabs64;
+__global__ void __launch_bounds__(32 * XENT_WARPS)
+xent_round_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
+                  const int32_t *__restrict__ labels, const long long *__restrict__ rowinfo,
+                  const WsHeader *__restrict__ hdr, int8_t *__restrict__ out, int B, int N, int round_mode,
+                  int32_t *__restrict__ b_out) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = blockIdx.x * XENT_WARPS + warp;
+  const unsigned long long mxv = hdr->maxabs64;
   const int b = 64 - __clzll((long long)mxv);
   const int bp = b > 7 ? b - 7 : 0;
   if (blockIdx.x == 0 && threadIdx.x == 0 && b_out) *b_out = b;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n;
-       i += (long long)gridDim.x * blockDim.x) {
-    long long v = e64[i];
-    unsigned long long m = v < 0 ? 0ull - (unsigned long long)v : (unsigned long long)v;
-    long long q = (long long)niti_round_mag<unsigned long long>(m, bp, 127ull, round_mode);
-    out[i] = (int8_t)(v < 0 ? -q : q);
+  if (r >= B) return;
+  const int s = *s_a_ptr;
+  const int label = labels[r];
+  const int8_t *row = a + (long long)r * N;
+  int8_t *orow = out + (long long)r * N;
+  const bool bad = s < -22 || s > 24 || label < 0 || label >= N;
+  const long long sh_amt = 15 - (long long)s;
+  const long long p = rowinfo[2 * (long long)r], csum = rowinfo[2 * (long long)r + 1];
+  auto one = [&](int i, int ai) -> int {
+    if (bad) return 0;
+    const long long v = xent_T(ai, s, sh_amt, p) - (i == label ? csum : 0);
+    const unsigned long long m = v < 0 ? 0ull - (unsigned long long)v : (unsigned long long)v;
+    const long long q = (long long)niti_round_mag<unsigned long long>(m, bp, 127ull, round_mode);
+    return (int)(v < 0 ? -q : q);
+  };
+  if ((N & 3) == 0 && (((uintptr_t)a | (uintptr_t)out) & 3) == 0) {
+    // four logits per lane per step: 128 contiguous bytes per warp instruction
+    for (int i = 4 * lane; i < N; i += 128) {
+      const unsigned w = *reinterpret_cast<const unsigned *>(row + i);
+      unsigned o = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        o |= ((unsigned)one(i + k, (int)(int8_t)(w >> (8 * k))) & 0xffu) << (8 * k);
+      *reinterpret_cast<unsigned *>(orow + i) = o;
+    }
+  } else {
+    for (int i = lane; i < N; i += 32) orow[i] = (int8_t)one(i, row[i]);
   }
 }
 
@@ -367,27 +400,25 @@ extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const
     return niti_fail(ctx, NITI_ERR_WORKSPACE, "niti_int_xent: workspace missing, misaligned or too small");
   cudaStream_t st = (cudaStream_t)stream;
   WsHeader *hdr = (WsHeader *)ws;
-  long long *e64 = (long long *)((char *)ws + NITI_WS_HEADER);
+  long long *rowinfo = (long long *)((char *)ws + NITI_WS_HEADER);
   NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, sizeof(WsHeader), st));
   ctx->launches++;
   if (n_correct) {
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st));
     ctx->launches++;
   }
-  xent_acc_kernel<<<B, 256, 0, st>>>(a, s_a, labels, e64, hdr, n_correct, N, ctx->d_status);
+  const unsigned blocks = (unsigned)((B + XENT_WARPS - 1) / XENT_WARPS);
+  xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, ctx->d_status);
   ctx->launches++;
-  long long n = (long long)B * N;
-  long long blocks = (n + 255) / 256;
-  if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
-  round_i64_kernel<<<(unsigned)blocks, 256, 0, st>>>(e64, hdr, e, n, round_mode, b_e);
+  xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
   ctx->launches++;
   NITI_CUDA_TRY(ctx, cudaGetLastError());
   return NITI_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
-// niti_int_xent_noalloc: the same two kernels with their scratch (reduction header + 64-bit loss
-// accumulators) in a fixed device array that is part of the library image, for callers that must
+// niti_int_xent_noalloc: the same two kernels with their scratch (reduction header + two 64-bit
+// scalars per sample) in a fixed device array that is part of the library image, for callers that must
 // not allocate device memory.  Every GPU that loads the library carries the array until exit.
 // ---------------------------------------------------------------------------------------------
 #define NITI_NOALLOC_BYTES (NITI_WS_HEADER + 8 * NITI_XENT_NOALLOC_MAX_ELEMS)
@@ -401,7 +432,8 @@ extern "C" int niti_int_xent_noalloc(void *stream, const int8_t *a, const int32_
                                      int8_t *e, int32_t *b_e, int32_t *n_correct, int B, int N, int round_mode) {
   if (!a || !s_a || !labels || !e || B <= 0 || N <= 0 || N > 65536 || (round_mode != 0 && round_mode != 1))
     return NITI_ERR_ARG;
-  if ((long long)B * N > NITI_XENT_NOALLOC_MAX_ELEMS) return NITI_ERR_TOO_LARGE;
+  if ((long long)B * N > NITI_XENT_NOALLOC_MAX_ELEMS || B > NITI_XENT_NOALLOC_MAX_ELEMS / 2)
+    return NITI_ERR_TOO_LARGE;                   // 16 bytes of scratch per sample must fit the array
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NITI_ERR_CUDA;
   void *base = nullptr;
@@ -416,17 +448,15 @@ extern "C" int niti_int_xent_noalloc(void *stream, const int8_t *a, const int32_
   }
   cudaStream_t st = (cudaStream_t)stream;
   WsHeader *hdr = (WsHeader *)base;
-  long long *e64 = (long long *)((char *)base + NITI_WS_HEADER);
+  long long *rowinfo = (long long *)((char *)base + NITI_WS_HEADER);
   // the array keeps what the previous call left: the reduction scalars must start at zero.  The last
   // word of the header takes the (unreported) status bits of this variant.
   uint32_t *status = (uint32_t *)((char *)base + NITI_WS_HEADER - sizeof(uint32_t));
   if (cudaMemsetAsync(base, 0, NITI_WS_HEADER, st) != cudaSuccess) return NITI_ERR_CUDA;
   if (n_correct && cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st) != cudaSuccess) return NITI_ERR_CUDA;
-  xent_acc_kernel<<<B, 256, 0, st>>>(a, s_a, labels, e64, hdr, n_correct, N, status);
-  const long long n = (long long)B * N;
-  long long blocks = (n + 255) / 256;
-  if (blocks > 1024) blocks = 1024;
-  round_i64_kernel<<<(unsigned)blocks, 256, 0, st>>>(e64, hdr, e, n, round_mode, b_e);
+  const unsigned blocks = (unsigned)((B + XENT_WARPS - 1) / XENT_WARPS);
+  xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
+  xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
   if (cudaGetLastError() != cudaSuccess) return NITI_ERR_CUDA;
   return NITI_OK;
 }
