@@ -503,8 +503,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                const TcParams p, int32_t *__restrict__ acc, WsHeader *hdr, uint32_t *status,
                int8_t *__restrict__ out8, const int8_t *__restrict__ mask8, const int32_t *s_a,
                const int32_t *s_w, int32_t *s_out, int32_t *b_out) {
+  if (p.epi_mode == EPI_SPECULATE && !p.single_wave) {
+    // the follow-up launch may be scheduled now (it is launched as a programmatic dependent): its CTAs
+    // take the SMs as this grid's CTAs retire and wait there for the whole grid to finish
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
   if (p.epi_mode == EPI_KNOWN_B) {
     // follow-up of a speculative pass: publish the scalars, then leave unless the guess was wrong
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // the first pass has completed and is visible
     const int b_true = niti_bitlen32(hdr->maxabs32), b_est = (int)hdr->spec_b;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       const int bp = b_true > p.mbits ? b_true - p.mbits : 0;
@@ -1648,13 +1654,19 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
   cfg.blockDim = dim3(NUM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CTAS;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (p.epi_mode == EPI_KNOWN_B) {
+    // programmatic dependent launch: the launch latency of the follow-up overlaps the first pass
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
+  }
   const int units = tc_units<CTAS>(ctx);
   long long grid = (p.items < units ? p.items : units) * CTAS;
   cfg.gridDim = dim3((unsigned)grid, 1, 1);
