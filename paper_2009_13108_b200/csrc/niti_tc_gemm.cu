@@ -1401,7 +1401,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
       // (64 x 64)-channel blocks re-read the activations once per block of the other operand, so this
       // mode is kept for layers with few blocks; wide layers use the per-tap tiles below
       if (want_halo && ctas == 1 && g.R == 3 && g.S == 3 && g.pad == 1 && g.Ci % 64 == 0 && g.Co % 64 == 0 &&
-          g.W >= 10 && g.H >= 18 && (long long)g.Ci * g.Co <= 65536) {
+          g.W >= 10 && g.H >= 18 && (long long)g.Ci * g.Co <= 32768) {
         p.halo = 2;
         p.kdepth = 128;
         p.bn = 64;
@@ -1694,7 +1694,9 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
     planned = plan(ctx, g, 1, false, p, ma, mb) && p.mrep > 1;
   if (!planned && ctx->engine != 2 && g.gm >= 2 * BM) {
     planned = plan(ctx, g, 2, false, p, ma, mb);
-    if (planned && ctx->engine != 3 && p.items < ctx->sm_count / 2) planned = false;
+    // (pairs halve the operand traffic per MMA; they are kept unless they would leave more than a
+    // third of the GPU idle)
+    if (planned && ctx->engine != 3 && p.items * 3 < (long long)(ctx->sm_count / 2) * 2) planned = false;
   }
   if (!planned) {
     if (ctx->engine == 3) return NITI_ERR_SHAPE;
