@@ -367,6 +367,13 @@ def run_ours(args):
     from paper_2009_13108_b200.dist_util import aggregate_throughput, max_over_ranks, rank_seed
     net.seed = rank_seed(net.seed, rank)         # every rank draws its own batch and replica
     x, labels, weights = make_net_inputs(net)
+    import hashlib
+    wh = hashlib.sha256()
+    for w in weights:
+        wh.update(memoryview(w).cast("B"))
+    input_digests = {"x": hashlib.sha256(memoryview(x).cast("B")).hexdigest()[:16],
+                     "labels": hashlib.sha256(memoryview(labels).cast("B")).hexdigest()[:16],
+                     "weights": wh.hexdigest()[:16]}      # guards against drift of the seeded generator
     tr = NitiTrainer(niti, net, weights)
     xh = torch.from_numpy(x).pin_memory()
     lh = torch.from_numpy(labels).pin_memory()
@@ -467,7 +474,8 @@ def run_ours(args):
                    "l2": "working set (activations + int32 scratch) exceeds the 126 MB L2",
                    "state": "weights restored to the seeded initial values before every step",
                    "launch": "cuda-graph replay" if args.graph else "eager",
-                   "parallelism": "replicas" if world > 1 else "single"},
+                   "parallelism": "replicas" if world > 1 else "single",
+                   "inputs_sha256_16": input_digests},
         "step_tops": ops_step / (ms / args.steps) / 1e9,
         "clocks": clocks,
         "e2e": {"value": images / (ms_e2e / 1e3), "unit": UNIT, "h2d_bytes_per_step": int(xh.numel() + lh.numel() * 4),

@@ -389,6 +389,195 @@ xent_round_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_
   }
 }
 
+// ---- fast path (N % 4 == 0, 4-byte aligned rows): packed bytes and per-row tables ---------------
+// T_i depends on the logit value alone once the row's offset p is known, and x-hat is monotone in
+// the logit, so a row needs: the maxima of the logits before and after the label (packed byte max;
+// they also decide the arg-max hit), for Eq. 2 the sums of a and a^2 (dp4a), for Eq. 3-4 the smallest
+// logit whose x-hat exceeds max - 10 (a binary search over the 256 logit values gives the threshold,
+// a packed min the logit) and the sum of T over a 256-entry table.  Pass 2 builds a 256-entry table
+// of rounded results per row and looks every logit up; only the label element is computed apart.
+__device__ __forceinline__ int hmax_s8x4(unsigned w) {
+  const int b0 = (int)(int8_t)w, b1 = (int)(int8_t)(w >> 8), b2 = (int)(int8_t)(w >> 16), b3 = (int)(int8_t)(w >> 24);
+  return max(max(b0, b1), max(b2, b3));
+}
+__device__ __forceinline__ int hmin_s8x4(unsigned w) {
+  const int b0 = (int)(int8_t)w, b1 = (int)(int8_t)(w >> 8), b2 = (int)(int8_t)(w >> 16), b3 = (int)(int8_t)(w >> 24);
+  return min(min(b0, b1), min(b2, b3));
+}
+__device__ __forceinline__ int warp_max_i(int v) {
+  for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ int warp_min_i(int v) {
+  for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ int warp_sum_i(int v) {
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__global__ void __launch_bounds__(32 * XENT_WARPS)
+xent_row_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
+                     const int32_t *__restrict__ labels, long long *__restrict__ rowinfo, WsHeader *hdr,
+                     int32_t *__restrict__ n_correct, int B, int N, uint32_t *__restrict__ status) {
+  __shared__ unsigned long long sh_max[XENT_WARPS];
+  __shared__ int sh_hit[XENT_WARPS];
+  __shared__ unsigned short sh_T[XENT_WARPS][256];     // T(a) of Eq. 4 for a = -128 .. 127 (at most 2^9)
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = blockIdx.x * XENT_WARPS + warp;
+  const int s = *s_a_ptr;
+  unsigned long long row_max = 0;
+  int hit = 0;
+  if (r < B) {
+    const int label = labels[r];
+    if (s < -22 || s > 24 || label < 0 || label >= N) {
+      if (lane == 0) {
+        atomicOr(status, (s < -22 || s > 24) ? NITI_DEV_XENT_RANGE : NITI_DEV_BAD_LABEL);
+        rowinfo[2 * (long long)r] = 0;
+        rowinfo[2 * (long long)r + 1] = 0;
+      }
+    } else {
+      const unsigned *row = reinterpret_cast<const unsigned *>(a + (long long)r * N);
+      const int words = N >> 2, lw = label >> 2, lb = label & 3;
+      const long long sh_amt = 15 - (long long)s;
+      const int a_label = (int)a[(long long)r * N + label];
+      // sweep 1: packed maxima before / after the label, sums of a and a^2
+      unsigned mb = 0x80808080u, ma = 0x80808080u;
+      int sum_a = 0, sum_q = 0;
+      for (int wi = lane; wi < words; wi += 32) {
+        const unsigned w = row[wi];
+        sum_a = __dp4a((int)w, 0x01010101, sum_a);
+        sum_q = __dp4a((int)w, (int)w, sum_q);
+        if (wi < lw) mb = __vmaxs4(mb, w);
+        else if (wi > lw) ma = __vmaxs4(ma, w);
+        else {
+          const unsigned low = lb == 0 ? 0u : (0xffffffffu >> (32 - 8 * lb));          // bytes before the label
+          const unsigned high = lb == 3 ? 0u : (0xffffffffu << (8 * (lb + 1)));        // bytes after it
+          mb = __vmaxs4(mb, (w & low) | (0x80808080u & ~low));
+          ma = __vmaxs4(ma, (w & high) | (0x80808080u & ~high));
+        }
+      }
+      const int max_before = warp_max_i(hmax_s8x4(mb)), max_after = warp_max_i(hmax_s8x4(ma));
+      const int max_other = max(max_before, max_after);       // -128 when the row has one element
+      const int row_top = max(max_other, a_label);
+      hit = (a_label > max_before && a_label >= max_after) ? 1 : 0;   // the first arg-max is the label
+      long long p = 0, csum, t_other, t_label;
+      if (s <= -7) {
+        sum_a = warp_sum_i(sum_a);
+        sum_q = warp_sum_i(sum_q);
+        csum = (long long)N * (1LL << (1 - 2 * s)) + (long long)sum_a * (1LL << (1 - s)) + (long long)sum_q;
+        t_other = N > 1 ? xent_T(max_other, s, sh_amt, 0) : 0;     // T is increasing in the logit
+        t_label = xent_T(a_label, s, sh_amt, 0);
+      } else {
+        const long long mx = xent_xhat(row_top, sh_amt);
+        // smallest logit value whose x-hat exceeds mx - 10 (x-hat is non-decreasing in the logit)
+        int lo = -128, hi = row_top;
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;          // floor for negative sums as well
+          if (xent_xhat(mid, sh_amt) > mx - 10) hi = mid; else lo = mid + 1;
+        }
+        const unsigned thr4 = (unsigned)(lo & 0xff) * 0x01010101u;
+        // sweep 2: the smallest logit of the row that is at least that value
+        unsigned mn = 0x7f7f7f7fu;
+        for (int wi = lane; wi < words; wi += 32) {
+          const unsigned w = row[wi];
+          const unsigned m = __vcmpges4(w, thr4);
+          mn = __vmins4(mn, (w & m) | (0x7f7f7f7fu & ~m));
+        }
+        const int a_star = warp_min_i(hmin_s8x4(mn));
+        p = xent_xhat(a_star, sh_amt);
+        // table of T over the logit values, then sweep 3: the sum
+        for (int v = lane; v < 256; v += 32) sh_T[warp][v] = (unsigned short)xent_T(v - 128, s, sh_amt, p);
+        __syncwarp();
+        int acc = 0;
+        for (int wi = lane; wi < words; wi += 32) {
+          const unsigned w = row[wi] ^ 0x80808080u;            // logit + 128 per byte
+          acc += (int)sh_T[warp][w & 0xff] + (int)sh_T[warp][(w >> 8) & 0xff] + (int)sh_T[warp][(w >> 16) & 0xff] +
+                 (int)sh_T[warp][w >> 24];
+        }
+        csum = (long long)warp_sum_i(acc);
+        t_other = N > 1 ? (long long)sh_T[warp][max_other + 128] : 0;
+        t_label = (long long)sh_T[warp][a_label + 128];
+      }
+      const long long on_label = csum - t_label;
+      row_max = (unsigned long long)(t_other > on_label ? t_other : on_label);
+      if (lane == 0) {
+        rowinfo[2 * (long long)r] = p;
+        rowinfo[2 * (long long)r + 1] = csum;
+      }
+    }
+  }
+  if (lane == 0) { sh_max[warp] = row_max; sh_hit[warp] = hit; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long m = 0;
+    int h = 0;
+    for (int w = 0; w < XENT_WARPS; ++w) { m = sh_max[w] > m ? sh_max[w] : m; h += sh_hit[w]; }
+    if (m > *(volatile unsigned long long *)&hdr->maxabs64) atomicMax(&hdr->maxabs64, m);
+    if (n_correct && h) atomicAdd(n_correct, h);
+  }
+}
+
+__global__ void __launch_bounds__(32 * XENT_WARPS)
+xent_round_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
+                       const int32_t *__restrict__ labels, const long long *__restrict__ rowinfo,
+                       const WsHeader *__restrict__ hdr, int8_t *__restrict__ out, int B, int N, int round_mode,
+                       int32_t *__restrict__ b_out) {
+  __shared__ unsigned char sh_q[XENT_WARPS][256];        // rounded T(a) for a = -128 .. 127
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = blockIdx.x * XENT_WARPS + warp;
+  const unsigned long long mxv = hdr->maxabs64;
+  const int b = 64 - __clzll((long long)mxv);
+  const int bp = b > 7 ? b - 7 : 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0 && b_out) *b_out = b;
+  if (r >= B) return;
+  const int s = *s_a_ptr;
+  const int label = labels[r];
+  const unsigned *row = reinterpret_cast<const unsigned *>(a + (long long)r * N);
+  unsigned *orow = reinterpret_cast<unsigned *>(out + (long long)r * N);
+  const int words = N >> 2;
+  if (s < -22 || s > 24 || label < 0 || label >= N) {
+    for (int wi = lane; wi < words; wi += 32) orow[wi] = 0u;
+    return;
+  }
+  const long long sh_amt = 15 - (long long)s;
+  const long long p = rowinfo[2 * (long long)r], csum = rowinfo[2 * (long long)r + 1];
+  // off the label e32 = T(a) > 0: one rounded value per logit value
+  for (int v = lane; v < 256; v += 32) {
+    const unsigned long long T = (unsigned long long)xent_T(v - 128, s, sh_amt, p);
+    sh_q[warp][v] = (unsigned char)niti_round_mag<unsigned long long>(T, bp, 127ull, round_mode);
+  }
+  // on the label e32 = T - sum <= 0
+  const int a_label = (int)a[(long long)r * N + label];
+  const unsigned long long m_label = (unsigned long long)(csum - xent_T(a_label, s, sh_amt, p));
+  const unsigned q_label = (unsigned)(0 - (int)niti_round_mag<unsigned long long>(m_label, bp, 127ull, round_mode)) & 0xffu;
+  __syncwarp();
+  const int lw = label >> 2, lb = label & 3;
+  for (int wi = lane; wi < words; wi += 32) {
+    const unsigned w = row[wi] ^ 0x80808080u;
+    unsigned o = (unsigned)sh_q[warp][w & 0xff] | ((unsigned)sh_q[warp][(w >> 8) & 0xff] << 8) |
+                 ((unsigned)sh_q[warp][(w >> 16) & 0xff] << 16) | ((unsigned)sh_q[warp][w >> 24] << 24);
+    if (wi == lw) o = (o & ~(0xffu << (8 * lb))) | (q_label << (8 * lb));
+    orow[wi] = o;
+  }
+}
+
+// both passes; the packed path needs whole words per row
+static void launch_xent(cudaStream_t st, const int8_t *a, const int32_t *s_a, const int32_t *labels,
+                        long long *rowinfo, WsHeader *hdr, int8_t *e, int32_t *b_e, int32_t *n_correct, int B, int N,
+                        int round_mode, uint32_t *status) {
+  const unsigned blocks = (unsigned)((B + XENT_WARPS - 1) / XENT_WARPS);
+  const bool packed = (N & 3) == 0 && N >= 64 && (((uintptr_t)a | (uintptr_t)e) & 3) == 0;
+  if (packed) {
+    xent_row_fast_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
+    xent_round_fast_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
+  } else {
+    xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
+    xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
+  }
+}
+
 extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const int32_t *s_a,
                              const int32_t *labels, int8_t *e, int32_t *b_e, int32_t *n_correct,
                              int B, int N, int round_mode, void *ws, size_t ws_bytes) {
@@ -407,11 +596,8 @@ extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st));
     ctx->launches++;
   }
-  const unsigned blocks = (unsigned)((B + XENT_WARPS - 1) / XENT_WARPS);
-  xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, ctx->d_status);
-  ctx->launches++;
-  xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
-  ctx->launches++;
+  launch_xent(st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, ctx->d_status);
+  ctx->launches += 2;
   NITI_CUDA_TRY(ctx, cudaGetLastError());
   return NITI_OK;
 }
@@ -454,9 +640,7 @@ extern "C" int niti_int_xent_noalloc(void *stream, const int8_t *a, const int32_
   uint32_t *status = (uint32_t *)((char *)base + NITI_WS_HEADER - sizeof(uint32_t));
   if (cudaMemsetAsync(base, 0, NITI_WS_HEADER, st) != cudaSuccess) return NITI_ERR_CUDA;
   if (n_correct && cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st) != cudaSuccess) return NITI_ERR_CUDA;
-  const unsigned blocks = (unsigned)((B + XENT_WARPS - 1) / XENT_WARPS);
-  xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
-  xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
+  launch_xent(st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, status);
   if (cudaGetLastError() != cudaSuccess) return NITI_ERR_CUDA;
   return NITI_OK;
 }

@@ -243,7 +243,7 @@ def test_saturation_and_zero_tensor(niti, oref):
 
 
 @pytest.mark.parametrize("s_a", [-22, -9, -7, -6, -4, 0, 24])
-@pytest.mark.parametrize("B,N", [(64, 10), (64, 1000), (7, 33), (256, 10)])
+@pytest.mark.parametrize("B,N", [(64, 10), (64, 1000), (7, 33), (256, 10), (9, 64), (3, 4096)])
 def test_int_xent(niti, oref, s_a, B, N):
     rng = np.random.default_rng(1000 + s_a + B + N)
     a = _i8(rng, (B, N))
@@ -252,6 +252,35 @@ def test_int_xent(niti, oref, s_a, B, N):
         want, b, nc = oref.int_xent(a, s_a, labels, mode)
         e, b_e, n_correct = niti.int_xent(_T(niti, a), niti.scalar(s_a), _T(niti, labels),
                                           round_mode=mode)
+        _eq(e, want)
+        assert (int(b_e), int(n_correct)) == (b, nc)
+    niti.check()
+
+
+@pytest.mark.parametrize("s_a", [-22, -8, -7, -6, -5, -3, 0, 9, 16, 24])
+def test_int_xent_packed_rows(niti, oref, s_a):
+    """Rows of whole 32-bit words take the packed-byte path: ties of the maximum before and after
+    the label, labels in every byte position of a word, constant rows, narrow and wide logit ranges."""
+    rng = np.random.default_rng(5000 + s_a)
+    B, N = 48, 64 * 5
+    a = _i8(rng, (B, N))
+    labels = rng.integers(0, N, size=B).astype(np.int32)
+    a[0] = 0                                              # constant row
+    a[1] = rng.integers(-2, 3, size=N)                    # narrow range
+    a[2] = -127; a[2, 17] = 127; labels[2] = 17           # one dominant logit, on the label
+    a[3] = -127; a[3, 18] = 127; labels[3] = 200          # ... off the label
+    for k in range(4):                                    # label in every byte position, tie before it
+        r = 4 + k
+        labels[r] = 100 + k
+        a[r, 100 + k] = 90; a[r, 3] = 90; a[r] = np.minimum(a[r], 90)
+    for k in range(4):                                    # tie after the label only: the label is the first arg-max
+        r = 8 + k
+        labels[r] = 40 + k
+        a[r] = np.minimum(a[r], 77); a[r, 40 + k] = 77; a[r, 300] = 77; a[r, :40 + k] = np.minimum(a[r, :40 + k], 76)
+    labels[12], labels[13] = 0, N - 1                     # first and last element
+    for mode in (0, 1):
+        want, b, nc = oref.int_xent(a, s_a, labels, mode)
+        e, b_e, n_correct = niti.int_xent(_T(niti, a), niti.scalar(s_a), _T(niti, labels), round_mode=mode)
         _eq(e, want)
         assert (int(b_e), int(n_correct)) == (b, nc)
     niti.check()
