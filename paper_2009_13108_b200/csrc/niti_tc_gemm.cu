@@ -38,6 +38,8 @@ struct TcParams {
   int kb_per_split;
   int splits;
   long long items;              // tiles * splits
+  int stg_off;                  // > 0: byte offset (from the aligned base) of the epilogue warps' transpose
+                                // buffers for coalesced atomic adds, 32 x 33 words per warp
   int mrep;                     // 128-row tiles per item (row-batched mode of short contractions), else 1
   int bn_mma;                   // N of one MMA; bn = mrep * bn_mma accumulator columns per item
   long long gm, gn;             // output extent (rows, columns); row pitch of acc is gn
@@ -985,7 +987,33 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (!mbar_wait(tfull0 + 8 * buf, (use / (unsigned)p.nbuf) & 1u, &abort_flag, status)) { ok = false; break; }
       tc_fence_after();
       const unsigned tm_row = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * (unsigned)p.bn;
-      if (p.epi_mode <= EPI_ATOMIC) {
+      if (p.epi_mode == EPI_ATOMIC && p.stg_off > 0) {
+        // Partial sums of a split contraction.  A lane holds one row of the chunk, so an atomic add
+        // issued straight from the registers touches 32 different lines; the chunk is transposed
+        // through shared memory instead and every add instruction covers 32 consecutive columns of
+        // one row (one 128-byte line).  Output rows are consecutive here (no pixel-box mapping).
+        int *stg = reinterpret_cast<int *>(smem_raw + (smem_base - smem_u32(smem_raw)) + p.stg_off) +
+                   (warp - EPI_WARP0) * (32 * 33);
+        const long long row0 = out_row - lane;                 // output row of lane 0 of this warp
+        for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
+          int v[32];
+          tc_ld32(tm_row + (unsigned)c, v);
+          if (c < ncols_valid) {                               // (uniform across the warp)
+#pragma unroll
+            for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = v[j];
+            __syncwarp();
+            const bool col_ok = c + lane < ncols_valid;
+            int32_t *dcol = acc + row0 * p.gn + col0 + c + lane;
+            long long rows_left = p.gm - row0;
+            if (rows_left > 32) rows_left = 32;
+            for (int rr = 0; rr < (int)rows_left; ++rr) {
+              const int val = stg[rr * 33 + lane];
+              if (col_ok && val != 0) atomicAdd(dcol + (long long)rr * p.gn, val);
+            }
+            __syncwarp();
+          }
+        }
+      } else if (p.epi_mode <= EPI_ATOMIC) {
         int32_t *dst = acc + out_row * p.gn + col0;
         const bool vec_ok = ((p.gn & 3) == 0) && ((col0 & 3) == 0);
         for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
@@ -1572,6 +1600,18 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
   }
   p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
   p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+  // split contractions add their partial sums atomically: room for the epilogue warps' transpose
+  // buffers (consecutive output rows only: every multiply but the pixel-box convolutions)
+  p.stg_off = 0;
+  if (p.splits > 1 && !p.halo && g.kind != GK_CONV_FWD && g.kind != GK_CONV_DGRAD) {
+    const int stg_bytes = EPI_WARPS * 32 * 33 * 4;
+    int st = (200 * 1024 - stg_bytes) / stage_bytes;
+    if (st > MAX_STAGES) st = MAX_STAGES;
+    if (st >= 2) {
+      p.stages = st;
+      p.stg_off = st * stage_bytes;
+    }
+  }
   if (p.halo) {
     p.splits = 1;
     p.kb_per_split = p.kb_total;
@@ -1643,6 +1683,7 @@ template <int CTAS>
 static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CUtensorMap &ma, const CUtensorMap &mb,
                      int32_t *acc, WsHeader *hdr, const RoundSpec &r) {
   size_t smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + (size_t)p.b_res_bytes + 1024;
+  if (p.stg_off > 0) smem = (size_t)p.stg_off + (size_t)EPI_WARPS * 32 * 33 * 4 + 1024;
   static size_t attr_smem = CTAS == 2 ? 201 * 1024 : 0;
   if (smem > attr_smem) {
     NITI_CUDA_TRY(ctx, cudaFuncSetAttribute(tc_gemm_kernel<CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
