@@ -38,6 +38,8 @@ struct TcParams {
   int kb_per_split;
   int splits;
   long long items;              // tiles * splits
+  int one_commit;               // resident-weights mode with as many patch stages as accumulator buffers:
+                                // stage and buffer advance together, one barrier per tile serves both
   int stg_off;                  // > 0: byte offset (from the aligned base) of the epilogue warps' transpose
                                 // buffers for coalesced atomic adds, 32 x 33 words per warp
   int mrep;                     // 128-row tiles per item (row-batched mode of short contractions), else 1
@@ -650,9 +652,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // consecutive items are consecutive tiles (blocked assignment): step the tile coordinates
         int wt = (int)(first_item % p.w_tiles), ht = (int)((first_item / p.w_tiles) % p.h_tiles);
         int bt = (int)(first_item / ((long long)p.w_tiles * p.h_tiles));
+        const unsigned free0 = p.one_commit ? tfull0 : empty0;   // "tile done" also frees the patch stage
         for (int item = first_item; ok && item < item_end; ++item) {
           if (stage % p.nprod == warp) {
-            if (!mbar_wait_warp(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
+            if (!mbar_wait_warp(free0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
             const unsigned full = full0 + 8 * stage;
             if (leader) {
               mbar_expect_tx(full, (unsigned)p.a_box_bytes);
@@ -823,9 +826,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           a_off[tap] = (fwd_taps ? (unsigned)(r * 10 + t) : (unsigned)((2 - r) * 10 + (2 - t))) * row16;
           b_tap[tap] = b_lo0 + (unsigned)tap * btile16;
         }
+        const bool one_commit = p.one_commit != 0;
         for (int item = first_item; ok && item < item_end; item += item_step, ++use) {
-          const unsigned buf = use % (unsigned)p.nbuf;
-          if (!mbar_wait_warp(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
+          // (with one_commit the accumulator buffer is the stage and their parities coincide)
+          const unsigned buf = one_commit ? (unsigned)stage : use % (unsigned)p.nbuf;
+          const unsigned par = one_commit ? phase : (use / (unsigned)p.nbuf) & 1u;
+          if (!mbar_wait_warp(tempty0 + 8 * buf, par ^ 1u, &abort_flag, status)) { ok = false; break; }
           if (!mbar_wait_warp(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
           tc_fence_after();
           const unsigned tmem_d = tmem_base + buf * (unsigned)p.bn;
@@ -834,7 +840,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (ksteps == 2) halo_issue_tile<2>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
             else if (ksteps == 4) halo_issue_tile<4>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
             else halo_issue_tile<1>(tmem_d, a_lo, a_hi, a_off, b_hi, b_tap, b_kstep16, idesc);
-            tc_commit(empty0 + 8 * stage);
+            if (!one_commit) tc_commit(empty0 + 8 * stage);
             tc_commit(tfull0 + 8 * buf);
           }
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
@@ -1628,6 +1634,14 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
   for (int gq = 2; gq <= 4; gq *= 2)
     if (EPI_PER_Q / gq <= p.bn / 32 && p.nbuf >= gq + 1) p.egroups = gq;
   p.nbuf = p.nbuf / p.egroups * p.egroups;     // a buffer always returns to the same group
+  p.one_commit = 0;
+  if (p.halo == 1 && p.stages >= p.nbuf) {
+    p.one_commit = 1;
+    p.stages = p.nbuf;
+    p.nprod = 1;
+    for (int d = 2; d <= PROD_WARPS; ++d)
+      if (p.stages % d == 0) p.nprod = d;
+  }
   // convolution outputs are spatially structured (borders, images): contiguous item ranges make the
   // first tile of every CTA an even sample of the tensor for the speculative shift
   p.blocked = (g.kind == GK_CONV_FWD || g.kind == GK_CONV_DGRAD) ? 1 : 0;
