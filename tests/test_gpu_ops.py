@@ -207,6 +207,25 @@ def test_speculative_shift_is_corrected_in_conv_and_row_batched_modes(niti, oref
     niti.check()
 
 
+@pytest.mark.parametrize("Ci,Co", [(64, 64), (64, 128)])
+def test_conv_resident_weights_many_tiles(niti, oref, Ci, Co):
+    """Several tiles per CTA in the resident-weights mode (693 8x16 pixel tiles, an odd count, ragged
+    in W and H): stage and accumulator rings wrap, contiguous tile ranges differ in length."""
+    rng = np.random.default_rng(Ci + Co)
+    B, H, W = 7, 141, 85
+    x, w, e = _i8(rng, (B, H, W, Ci)), _i8(rng, (Co, 3, 3, Ci)), _i8(rng, (B, H, W, Co))
+    wy, s, b = oref.conv_fwd(x, -7, w, -9, 1, True)
+    y, s_y, b_y = niti.conv_fwd(_T(niti, x), niti.scalar(-7), _T(niti, w), niti.scalar(-9), relu=True)
+    _eq(y, wy)
+    assert (int(s_y), int(b_y)) == (s, b)
+    xm = np.maximum(x, 0)
+    wd, bd = oref.conv_dgrad(e, w, (H, W), 1, xm)
+    ep, b_e = niti.conv_dgrad(_T(niti, e), _T(niti, w), (H, W), relu_mask_src=_T(niti, xm))
+    _eq(ep, wd)
+    assert int(b_e) == bd
+    niti.check()
+
+
 def test_general_taps_and_padding_use_the_fallback(niti, oref):
     rng = np.random.default_rng(2)
     x, w = _i8(rng, (2, 9, 9, 4)), _i8(rng, (6, 5, 5, 4))
