@@ -1151,6 +1151,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (lane == 0) spec_bp_ready = bp + 1;
         }
         const bool vec_ok = ((p.gn & 15) == 0) && ((col0 & 15) == 0);
+        const bool vec32_ok = ((p.gn & 31) == 0) && ((col0 & 31) == 0) && (((uintptr_t)out8 & 31) == 0);
         const RoundConst rk = make_round_const(bp, p.mbits, p.round_mode);
         for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
           int v[32];
@@ -1186,8 +1187,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 w8[4] &= bytes_gt0(m1v.x); w8[5] &= bytes_gt0(m1v.y);
                 w8[6] &= bytes_gt0(m1v.z); w8[7] &= bytes_gt0(m1v.w);
               }
-              *reinterpret_cast<int4 *>(dst8 + cc) = make_int4(w8[0], w8[1], w8[2], w8[3]);
-              *reinterpret_cast<int4 *>(dst8 + cc + 16) = make_int4(w8[4], w8[5], w8[6], w8[7]);
+              if (vec32_ok) {
+                // one 32-byte sector per lane in a single request (half as many store requests)
+                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                             ::"l"(dst8 + cc), "r"(w8[0]), "r"(w8[1]), "r"(w8[2]), "r"(w8[3]), "r"(w8[4]), "r"(w8[5]),
+                               "r"(w8[6]), "r"(w8[7])
+                             : "memory");
+              } else {
+                *reinterpret_cast<int4 *>(dst8 + cc) = make_int4(w8[0], w8[1], w8[2], w8[3]);
+                *reinterpret_cast<int4 *>(dst8 + cc + 16) = make_int4(w8[4], w8[5], w8[6], w8[7]);
+              }
             } else {
 #pragma unroll
               for (int j = 0; j < 32; ++j)
