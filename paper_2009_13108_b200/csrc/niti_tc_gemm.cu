@@ -1171,8 +1171,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           // the rounding arithmetic
           int4 m0v = make_int4(0x01010101, 0x01010101, 0x01010101, 0x01010101), m1v = m0v;
           if (msk && vec_ok && rok && cc + 32 <= ncols_valid) {
-            m0v = *reinterpret_cast<const int4 *>(msk + cc);
-            m1v = *reinterpret_cast<const int4 *>(msk + cc + 16);
+            if (vec32_ok && (((uintptr_t)mask8 & 31) == 0)) {
+              asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                           : "=r"(m0v.x), "=r"(m0v.y), "=r"(m0v.z), "=r"(m0v.w), "=r"(m1v.x), "=r"(m1v.y), "=r"(m1v.z),
+                             "=r"(m1v.w)
+                           : "l"(msk + cc));
+            } else {
+              m0v = *reinterpret_cast<const int4 *>(msk + cc);
+              m1v = *reinterpret_cast<const int4 *>(msk + cc + 16);
+            }
           }
           tc_ld32(tm_row + (unsigned)c, v);
           if (rok && cc < ncols_valid) {
