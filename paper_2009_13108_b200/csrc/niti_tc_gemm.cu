@@ -533,6 +533,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ unsigned tmem_base_slot;
   __shared__ volatile int abort_flag;
   __shared__ volatile int spec_bp_ready;      // 0: not yet; else the speculative binary point + 1
+  __shared__ unsigned first_max, first_arrived;   // this CTA's first tile: max magnitude, warps that reported
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const unsigned rank = CTAS == 2 ? cluster_ctarank() : 0u;
@@ -572,6 +573,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (threadIdx.x == 0) {
     abort_flag = 0;
     spec_bp_ready = 0;
+    first_max = 0;
+    first_arrived = 0;
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
@@ -1121,34 +1124,52 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             unsigned u = __shfl_xor_sync(0xffffffffu, m0, o);
             m0 = u > m0 ? u : m0;
           }
+          // The warps of this CTA combine their maxima in shared memory; the last one to report speaks
+          // for the CTA in the grid-wide agreement (one atomic and one poller per CTA: with every warp
+          // of every CTA polling the same word the wait itself took microseconds) and publishes the
+          // shift to the others through shared memory.
           if (lane == 0) {
-            if (m0) atomicMax(&hdr->est_max, m0);
-            __threadfence();
-            atomicAdd(&hdr->tile_counter, 1u);
-            const unsigned expected = gridDim.x * (unsigned)epi_active;
-            long long t0 = clock64();
-            while (*(volatile unsigned *)&hdr->tile_counter < expected) {
+            if (m0) atomicMax(&first_max, m0);
+            __threadfence_block();
+            if (atomicAdd(&first_arrived, 1u) + 1u == (unsigned)epi_active) {
+              const unsigned cm = *(volatile unsigned *)&first_max;
+              if (cm) atomicMax(&hdr->est_max, cm);
+              __threadfence();
+              atomicAdd(&hdr->tile_counter, 1u);
+              const unsigned expected = gridDim.x;
+              long long t0 = clock64();
+              while (*(volatile unsigned *)&hdr->tile_counter < expected) {
+                if (abort_flag) break;
+                if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                  abort_flag = 1;
+                  atomicOr(status, NITI_DEV_TIMEOUT);
+                  break;
+                }
+                __nanosleep(40);
+              }
+              __threadfence();
+              const unsigned gmax = *(volatile unsigned *)&hdr->est_max;
+              // the first tiles are a sample: scale their max by the growth expected from the sample to
+              // the whole tensor before taking the bit length (a wrong guess only costs the redo pass)
+              unsigned long long scaled = ((unsigned long long)gmax * p.spec_mul256) >> 8;
+              if (scaled > 0x7fffffffull) scaled = 0x7fffffffull;
+              const int b = niti_bitlen32((unsigned)scaled);
+              if (blockIdx.x == 0) hdr->spec_b = (unsigned)b;
+              spec_bp_ready = (b > p.mbits ? b - p.mbits : 0) + 1;
+            }
+            long long t1 = clock64();
+            while (spec_bp_ready == 0) {
               if (abort_flag) break;
-              if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+              if (clock64() - t1 > WAIT_LIMIT_CYCLES) {
                 abort_flag = 1;
                 atomicOr(status, NITI_DEV_TIMEOUT);
                 break;
               }
             }
-            __threadfence();
           }
           __syncwarp();
           if (abort_flag) { ok = false; break; }
-          if (lane == 0) spec_max = *(volatile unsigned *)&hdr->est_max;
-          spec_max = __shfl_sync(0xffffffffu, spec_max, 0);
-          // the first tiles are a sample: scale their max by the growth expected from the sample to
-          // the whole tensor before taking the bit length (a wrong guess only costs the redo pass)
-          unsigned long long scaled = ((unsigned long long)spec_max * p.spec_mul256) >> 8;
-          if (scaled > 0x7fffffffull) scaled = 0x7fffffffull;
-          const int b = niti_bitlen32((unsigned)scaled);
-          bp = b > p.mbits ? b - p.mbits : 0;
-          if (blockIdx.x == 0 && warp == EPI_WARP0 && lane == 0) hdr->spec_b = (unsigned)b;
-          if (lane == 0) spec_bp_ready = bp + 1;
+          bp = spec_bp_ready - 1;
         }
         const bool vec_ok = ((p.gn & 15) == 0) && ((col0 & 15) == 0);
         const bool vec32_ok = ((p.gn & 31) == 0) && ((col0 & 31) == 0) && (((uintptr_t)out8 & 31) == 0);
