@@ -534,6 +534,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ volatile int abort_flag;
   __shared__ volatile int spec_bp_ready;      // 0: not yet; else the speculative binary point + 1
   __shared__ unsigned first_max, first_arrived;   // this CTA's first tile: max magnitude, warps that reported
+  __shared__ unsigned cta_max;                    // max magnitude of everything this CTA rounded
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const unsigned rank = CTAS == 2 ? cluster_ctarank() : 0u;
@@ -575,6 +576,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     spec_bp_ready = 0;
     first_max = 0;
     first_arrived = 0;
+    cta_max = 0;
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
@@ -1250,13 +1252,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         unsigned u = __shfl_xor_sync(0xffffffffu, mx, o);
         mx = u > mx ? u : mx;
       }
-      if (lane == 0 && mx) atomicMax(&hdr->maxabs32, mx);
+      if (lane == 0 && mx) atomicMax(&cta_max, mx);     // (one global atomic per CTA, below)
     }
   }
 
   // ================= common exit =================
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0 && cta_max) atomicMax(&hdr->maxabs32, cta_max);
   if (abort_flag) {
     // give copies and MMAs still in flight time to land before shared and tensor memory go away
     long long t0 = clock64();
