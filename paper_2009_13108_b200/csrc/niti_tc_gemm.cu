@@ -38,6 +38,8 @@ struct TcParams {
   int kb_per_split;
   int splits;
   long long items;              // tiles * splits
+  int quorum;                   // CTAs whose first tile must have reported before the speculative bit-width
+                                // is fixed (all of them when the sample is the whole tensor)
   int one_commit;               // resident-weights mode with as many patch stages as accumulator buffers:
                                 // stage and buffer advance together, one barrier per tile serves both
   int stg_off;                  // > 0: byte offset (from the aligned base) of the epilogue warps' transpose
@@ -515,7 +517,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (p.epi_mode == EPI_KNOWN_B) {
     // follow-up of a speculative pass: publish the scalars, then leave unless the guess was wrong
     asm volatile("griddepcontrol.wait;" ::: "memory");     // the first pass has completed and is visible
-    const int b_true = niti_bitlen32(hdr->maxabs32), b_est = (int)hdr->spec_b;
+    const int b_true = niti_bitlen32(hdr->maxabs32), b_est = (int)hdr->spec_b - 1;   // (stored + 1)
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       const int bp = b_true > p.mbits ? b_true - p.mbits : 0;
       if (b_out) *b_out = b_true;
@@ -571,21 +573,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   unsigned tmem_cols = 32;
   while (tmem_cols < (unsigned)(p.nbuf * p.bn)) tmem_cols <<= 1;
 
+  // Set-up is paid by every launch (measured: 1.8 us from entry to the first copy when one thread did
+  // all of it): the tensor maps are prefetched at once, every barrier is initialised by its own
+  // thread, and tensor memory is allocated by another warp meanwhile.
+  if (threadIdx.x == 32) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+  }
   if (threadIdx.x == 0) {
     abort_flag = 0;
     spec_bp_ready = 0;
     first_max = 0;
     first_arrived = 0;
     cta_max = 0;
-    for (int s = 0; s < p.stages; ++s) {
-      mbar_init(full0 + 8 * s, 1);
-      mbar_init(empty0 + 8 * s, 1);
-    }
-    mbar_init(bres_bar, 1);
-    for (int b = 0; b < p.nbuf; ++b) {
-      mbar_init(tfull0 + 8 * b, 1);
-      mbar_init(tempty0 + 8 * b, epi_active * CTAS);    // one arrival per working epilogue warp of every CTA
-    }
+  }
+  if (threadIdx.x < 2 * MAX_STAGES + 2 * MAX_TBUF + 1) {
+    const int bi = (int)threadIdx.x;
+    const bool is_tempty = bi >= 2 * MAX_STAGES + MAX_TBUF && bi < 2 * MAX_STAGES + 2 * MAX_TBUF;
+    // one arrival per barrier, except "accumulator drained": one per working epilogue warp of every CTA
+    mbar_init(smem_u32(&bars[bi]), is_tempty ? epi_active * CTAS : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -644,8 +650,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       } else if (p.halo) {
         // resident weights: one tile per tap, [bn rows][kdepth] K-major (forward) or
         // [kdepth rows][bn] MN-major in b_boxes column chunks (dgrad)
-        if (warp == 0 && leader) mbar_expect_tx(bres_bar, (unsigned)(9 * p.b_boxes * p.b_box_bytes));
-        for (int tap = 0; warp == 0 && leader && tap < 9; ++tap) {
+        // (issued by the last producer warp: the first one owns stage 0 and starts with tile 0's patch)
+        if (warp == PROD_WARPS - 1 && leader) mbar_expect_tx(bres_bar, (unsigned)(9 * p.b_boxes * p.b_box_bytes));
+        for (int tap = 0; warp == PROD_WARPS - 1 && leader && tap < 9; ++tap) {
           const unsigned dst = smem_base + tap * p.b_tile_bytes;
           if (p.kind == GK_CONV_FWD) {
             tma_load_2d(dst, &map_b, bres_bar, tap * p.kdepth, 0);
@@ -1138,9 +1145,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               if (cm) atomicMax(&hdr->est_max, cm);
               __threadfence();
               atomicAdd(&hdr->tile_counter, 1u);
-              const unsigned expected = gridDim.x;
+              // The bit-width is fixed as soon as a quorum of CTAs has reported, by whichever CTA sees
+              // that first (compare-and-swap on the published word); CTAs that start late find it
+              // published and never wait.  Waiting for every CTA meant waiting out the launch ramp of
+              // the whole grid (~10 k cycles) in every launch.
+              const unsigned quorum = (unsigned)p.quorum;
+              unsigned pub = 0;
               long long t0 = clock64();
-              while (*(volatile unsigned *)&hdr->tile_counter < expected) {
+              while ((pub = *(volatile unsigned *)&hdr->spec_b) == 0) {
+                if (*(volatile unsigned *)&hdr->tile_counter >= quorum) {
+                  __threadfence();
+                  const unsigned gmax = *(volatile unsigned *)&hdr->est_max;
+                  // the first tiles are a sample: scale their max by the growth expected from the sample
+                  // to the whole tensor before taking the bit length (a wrong guess only costs the redo)
+                  unsigned long long scaled = ((unsigned long long)gmax * p.spec_mul256) >> 8;
+                  if (scaled > 0x7fffffffull) scaled = 0x7fffffffull;
+                  atomicCAS(&hdr->spec_b, 0u, (unsigned)niti_bitlen32((unsigned)scaled) + 1u);
+                  continue;
+                }
                 if (abort_flag) break;
                 if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
                   abort_flag = 1;
@@ -1149,14 +1171,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 __nanosleep(40);
               }
-              __threadfence();
-              const unsigned gmax = *(volatile unsigned *)&hdr->est_max;
-              // the first tiles are a sample: scale their max by the growth expected from the sample to
-              // the whole tensor before taking the bit length (a wrong guess only costs the redo pass)
-              unsigned long long scaled = ((unsigned long long)gmax * p.spec_mul256) >> 8;
-              if (scaled > 0x7fffffffull) scaled = 0x7fffffffull;
-              const int b = niti_bitlen32((unsigned)scaled);
-              if (blockIdx.x == 0) hdr->spec_b = (unsigned)b;
+              const int b = (int)pub - 1;
               spec_bp_ready = (b > p.mbits ? b - p.mbits : 0) + 1;
             }
             long long t1 = clock64();
@@ -1830,11 +1845,18 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
     const int units = p.ctas == 2 ? tc_units<2>(ctx) : tc_units<1>(ctx);
     const double n_all = (double)g.gm * (double)g.gn;
     const double frac = p.items > units ? (double)units / (double)p.items : 1.0;
-    const double n_s = n_all * frac;
+    // (when the tensor has more tiles than the grid, the bit-width is fixed once half of the CTAs have
+    // reported; typically a few more have by then)
+    const double n_s = n_all * frac * (frac < 1.0 ? 0.6 : 1.0);
     double f = (n_s > 16.0 && frac < 1.0) ? sqrt(log(n_all) / log(n_s)) : 1.0;
     p.spec_mul256 = (unsigned)(f * 256.0 + 0.5);
   }
   p.single_wave = (p.items <= (p.ctas == 2 ? tc_units<2>(ctx) : tc_units<1>(ctx)) && p.spec_mul256 == 256) ? 1 : 0;
+  {
+    const long long units = p.ctas == 2 ? tc_units<2>(ctx) : tc_units<1>(ctx);
+    const long long grid = (p.items < units ? p.items : units) * p.ctas;
+    p.quorum = (int)(p.single_wave ? grid : (grid + 1) / 2);
+  }
   p.mbits = r.mbits;
   p.round_mode = r.round_mode;
   p.relu = r.relu;
