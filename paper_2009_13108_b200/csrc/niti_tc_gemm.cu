@@ -621,6 +621,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int stage = 0;
       unsigned phase = 0;
       bool ok = true;
+      // (an integer division costs a lone warp ~200 cycles: nothing below divides per k-block or per
+      // tile; the warp that owns the current stage is counted, stage % nprod)
+      int owner = 0;
+      const int nprod = p.nprod;
       const int bn_cta = p.bn / CTAS;             // B rows (output columns) staged by this CTA
       if (p.halo == 2) {
         for (int item = first_item; ok && item < item_end; item += item_step) {
@@ -632,7 +636,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (t1 > p.kb_total) t1 = p.kb_total;
           int wt = t0 % p.w_tiles, ht = (t0 / p.w_tiles) % p.h_tiles, bt = t0 / (p.w_tiles * p.h_tiles);
           for (int t = t0; t < t1; ++t) {
-            if (stage % p.nprod == warp) {
+            if (owner == warp) {
               if (!mbar_wait_warp(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
               const unsigned full = full0 + 8 * stage;
               const unsigned sa = smem_base + stage * stage_bytes;
@@ -642,7 +646,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tma_load_4d(sa + p.a_bytes, &map_b, full, co0, wt * 8, ht * 16, bt);     // error tile
               }
             }
-            if (++stage == p.stages) { stage = 0; phase ^= 1; }
+            if (++owner == nprod) owner = 0;
+          if (++stage == p.stages) { stage = 0; phase ^= 1; }
             if (++wt == p.w_tiles) { wt = 0; if (++ht == p.h_tiles) { ht = 0; ++bt; } }
           }
         }
@@ -666,7 +671,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int bt = (int)(first_item / ((long long)p.w_tiles * p.h_tiles));
         const unsigned free0 = p.one_commit ? tfull0 : empty0;   // "tile done" also frees the patch stage
         for (int item = first_item; ok && item < item_end; ++item) {
-          if (stage % p.nprod == warp) {
+          if (owner == warp) {
             if (!mbar_wait_warp(free0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
             const unsigned full = full0 + 8 * stage;
             if (leader) {
@@ -674,6 +679,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               tma_load_4d(smem_base + p.b_res_bytes + stage * p.a_bytes, &map_a, full, 0, wt * 8 - 1, ht * 16 - 1, bt);
             }
           }
+          if (++owner == nprod) owner = 0;
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
           if (++wt == p.w_tiles) { wt = 0; if (++ht == p.h_tiles) { ht = 0; ++bt; } }
         }
@@ -736,7 +742,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (p.kind == GK_CONV_WGRAD) { wg_r = tap_n / p.S; wg_s = tap_n % p.S; }
         const unsigned tx_bytes = (unsigned)(CTAS * (p.a_boxes * p.a_box_bytes + p.b_boxes * p.b_box_bytes));
         for (int kb = kb0; kb < kb1; ++kb) {
-         if (stage % p.nprod == warp) {
+         if (owner == warp) {
           if (!mbar_wait_warp(empty0 + 8 * stage, phase ^ 1, &abort_flag, status)) { ok = false; break; }
           const unsigned full = lead_full0 + 8 * stage;
           const unsigned sa = smem_base + stage * stage_bytes;
@@ -788,6 +794,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           } else if (p.kind == GK_CONV_WGRAD) {
             if (++kwt == p.w_tiles) { kwt = 0; if (++kht == p.h_tiles) { kht = 0; ++kbt; } }
           }
+          if (++owner == nprod) owner = 0;
           if (++stage == p.stages) { stage = 0; phase ^= 1; }
         }
       }
@@ -866,10 +873,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           b_tap[tap] = b_lo0 + (unsigned)tap * btile16;
         }
         const bool one_commit = p.one_commit != 0;
+        unsigned hbuf = 0, hpar = 0;          // use % nbuf, (use / nbuf) & 1, counted
         for (int item = first_item; ok && item < item_end; item += item_step, ++use) {
           // (with one_commit the accumulator buffer is the stage and their parities coincide)
-          const unsigned buf = one_commit ? (unsigned)stage : use % (unsigned)p.nbuf;
-          const unsigned par = one_commit ? phase : (use / (unsigned)p.nbuf) & 1u;
+          const unsigned buf = one_commit ? (unsigned)stage : hbuf;
+          const unsigned par = one_commit ? phase : hpar;
+          if (++hbuf == (unsigned)p.nbuf) { hbuf = 0; hpar ^= 1u; }
           if (!mbar_wait_warp(tempty0 + 8 * buf, par ^ 1u, &abort_flag, status)) { ok = false; break; }
           if (!mbar_wait_warp(full0 + 8 * stage, phase, &abort_flag, status)) { ok = false; break; }
           tc_fence_after();
@@ -892,14 +901,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const unsigned g_ak = p.a_kstep16, g_bk = p.b_kstep16, g_idesc = p.idesc, g_a_bytes = (unsigned)p.a_bytes;
       const int g_ksteps = p.ksteps, g_mrep = p.mrep;
       const unsigned g_bn_mma = (unsigned)p.bn_mma, g_slice16 = (unsigned)p.a_box_bytes >> 4;
+      unsigned gbuf = 0, gpar = 0;            // use % nbuf, (use / nbuf) & 1, counted
       for (int item = first_item; ok && item < item_end; item += item_step, ++use) {
         const int split = p.splits > 1 ? item % p.splits : 0;
         const int kb0 = split * p.kb_per_split;
         int kb1 = kb0 + p.kb_per_split;
         if (kb1 > p.kb_total) kb1 = p.kb_total;
-        const unsigned buf = use % (unsigned)p.nbuf;
+        const unsigned buf = gbuf;
         // wait until the epilogue has drained this accumulator buffer (the first nbuf uses pass at once)
-        if (!mbar_wait_warp(tempty0 + 8 * buf, ((use / (unsigned)p.nbuf) & 1u) ^ 1u, &abort_flag, status)) { ok = false; break; }
+        if (!mbar_wait_warp(tempty0 + 8 * buf, gpar ^ 1u, &abort_flag, status)) { ok = false; break; }
+        if (++gbuf == (unsigned)p.nbuf) { gbuf = 0; gpar ^= 1u; }
         tc_fence_after();
         const unsigned tmem_d = tmem_base + buf * (unsigned)p.bn;
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -977,12 +988,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       item_end = first_item;
     }
     use = (unsigned)egroup;
+    unsigned ebuf = (unsigned)egroup, epar = 0;       // use % nbuf, (use / nbuf) & 1 (nbuf is a multiple of egroups)
+    // this thread's pixel inside a pixel box (generic convolutions): the box sides are powers of two
+    const int wt_d = p.Wt > 0 ? p.Wt : 1, ht_d = p.Ht > 0 ? p.Ht : 1;     // (unset for plain matrix multiplies)
+    const int r_ww = row_in_tile % wt_d, r_t = row_in_tile / wt_d;
+    const int r_hh = r_t % ht_d, r_bb = r_t / ht_d;
     for (int item = first_item + egroup * item_step; ok && item < item_end;
          item += item_step * egroups, use += (unsigned)egroups) {
       int mu = 0, nt = 0, split = 0;
       if (!p.halo) decode_item(p, item, mu, nt, split);
       const int mt = mu * CTAS + (int)rank;
-      const unsigned buf = use % (unsigned)p.nbuf;
+      const unsigned buf = ebuf;
+      const unsigned tpar = epar;
+      ebuf += (unsigned)egroups;
+      if (ebuf >= (unsigned)p.nbuf) { ebuf -= (unsigned)p.nbuf; epar ^= 1u; }
       // output row / column base of this thread
       long long out_row;
       bool row_ok;
@@ -1005,8 +1024,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       } else if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) {
         int w0, h0, b0;
         pixel_box(p, mt, w0, h0, b0);
-        int ww = row_in_tile % p.Wt, t = row_in_tile / p.Wt;
-        int hh = t % p.Ht, bb = t / p.Ht;
+        const int ww = r_ww, hh = r_hh, bb = r_bb;
         int w = w0 + ww, h = h0 + hh, b = b0 + bb;
         row_ok = w < p.PW && h < p.PH && b < p.PB;
         out_row = ((long long)b * p.PH + h) * p.PW + w;
@@ -1029,7 +1047,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         long long rem = p.gn - col0;
         ncols_valid = rem < p.bn ? (int)rem : p.bn;
       }
-      if (!mbar_wait(tfull0 + 8 * buf, (use / (unsigned)p.nbuf) & 1u, &abort_flag, status)) { ok = false; break; }
+      if (!mbar_wait(tfull0 + 8 * buf, tpar, &abort_flag, status)) { ok = false; break; }
       tc_fence_after();
       const unsigned tm_row = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * (unsigned)p.bn;
       if (p.epi_mode == EPI_ATOMIC && p.stg_off > 0) {
