@@ -32,13 +32,15 @@ struct niti_ctx {
 // Scalars at the start of a workspace.
 struct WsHeader {
   unsigned int maxabs32;            // a value with the bit length of max |acc| (a max, or an OR of magnitudes)
-  unsigned int est_max;             // max |acc| over the first tile of every CTA (speculative shift)
-  unsigned long long maxabs64;      // same for the 64-bit loss accumulators
-  unsigned int tile_counter;        // arrival counter of the grid-wide wait
-  unsigned int spec_b;              // bit-width the speculative epilogue rounded with
   unsigned int done_ctas;           // CTAs that have finished (single-wave launches publish b themselves)
+  unsigned long long maxabs64;      // same for the 64-bit loss accumulators
+  // the three words of the speculative agreement share one 16-byte line so that one load polls them all
+  unsigned int est_max;             // max |acc| over the first tile of the CTAs that have reported
+  unsigned int tile_counter;        // CTAs that have reported
+  unsigned int spec_b;              // 0, or 1 + the bit-width the speculative epilogue rounds with
   unsigned int pad1[1];
 };
+static_assert(sizeof(WsHeader) == 32, "workspace header layout");
 
 #define NITI_CUDA_TRY(ctx, expr)                                                        \
   do {                                                                                  \

@@ -1170,16 +1170,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               const unsigned quorum = (unsigned)p.quorum;
               unsigned pub = 0;
               long long t0 = clock64();
-              while ((pub = *(volatile unsigned *)&hdr->spec_b) == 0) {
-                if (*(volatile unsigned *)&hdr->tile_counter >= quorum) {
-                  __threadfence();
-                  const unsigned gmax = *(volatile unsigned *)&hdr->est_max;
+              while (true) {
+                // one 16-byte load: {est_max, tile_counter, spec_b, -}
+                unsigned v_max, v_cnt, v_pub, v_pad;
+                asm volatile("ld.volatile.global.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(v_max), "=r"(v_cnt), "=r"(v_pub), "=r"(v_pad)
+                             : "l"(&hdr->est_max)
+                             : "memory");
+                if (v_pub) { pub = v_pub; break; }
+                if (v_cnt >= quorum) {
                   // the first tiles are a sample: scale their max by the growth expected from the sample
                   // to the whole tensor before taking the bit length (a wrong guess only costs the redo)
-                  unsigned long long scaled = ((unsigned long long)gmax * p.spec_mul256) >> 8;
+                  unsigned long long scaled = ((unsigned long long)v_max * p.spec_mul256) >> 8;
                   if (scaled > 0x7fffffffull) scaled = 0x7fffffffull;
-                  atomicCAS(&hdr->spec_b, 0u, (unsigned)niti_bitlen32((unsigned)scaled) + 1u);
-                  continue;
+                  const unsigned mine = (unsigned)niti_bitlen32((unsigned)scaled) + 1u;
+                  const unsigned old = atomicCAS(&hdr->spec_b, 0u, mine);
+                  pub = old ? old : mine;
+                  break;
                 }
                 if (abort_flag) break;
                 if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
@@ -1187,7 +1194,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   atomicOr(status, NITI_DEV_TIMEOUT);
                   break;
                 }
-                __nanosleep(40);
               }
               const int b = (int)pub - 1;
               spec_bp_ready = (b > p.mbits ? b - p.mbits : 0) + 1;
