@@ -38,6 +38,9 @@ struct TcParams {
   int kb_per_split;
   int splits;
   long long items;              // tiles * splits
+  // set-up arithmetic done on the host (integer divisions at kernel entry delay every launch)
+  int blk_per, blk_extra;       // blocked assignment: items per CTA (pair) and how many take one more
+  int k_wpq, k_wpq_active, k_epi_active, k_tmem_cols;
   int quorum;                   // CTAs whose first tile must have reported before the speculative bit-width
                                 // is fixed (all of them when the sample is the whole tensor)
   int one_commit;               // resident-weights mode with as many patch stages as accumulator buffers:
@@ -553,8 +556,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // items of this CTA (pair): first_item, first_item + item_step, ... below item_end
   int first_item = blockIdx.x / CTAS, item_step = gridDim.x / CTAS, item_end = (int)p.items;
   if (p.blocked) {
-    const int units = gridDim.x / CTAS, u = blockIdx.x / CTAS;
-    const int per = (int)p.items / units, extra = (int)p.items % units;
+    const int u = blockIdx.x / CTAS;
+    const int per = p.blk_per, extra = p.blk_extra;
     first_item = u * per + (u < extra ? u : extra);
     item_end = first_item + per + (u < extra ? 1 : 0);
     item_step = 1;
@@ -565,13 +568,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // time (narrow tiles have too few 32-column chunks to keep every warp busy on one tile).  Inside a
   // group each TMEM lane quarter has wpq warps that interleave the tile's chunks.
   const int egroups = p.halo == 2 ? 1 : p.egroups;
-  const int wpq = EPI_PER_Q / egroups;                       // warps per quarter per tile
-  const int chunks_all = p.bn / 32;
-  const int wpq_active = p.halo == 2 ? EPI_PER_Q : (chunks_all < wpq ? chunks_all : wpq);
-  const int epi_active = 4 * wpq_active;                     // warps that drain one tile
+  const int wpq = p.k_wpq;                                   // warps per quarter per tile
+  const int wpq_active = p.k_wpq_active;
+  const int epi_active = p.k_epi_active;                     // warps that drain one tile
   // TMEM columns: nbuf accumulator buffers of bn columns, rounded up to a power of two >= 32
-  unsigned tmem_cols = 32;
-  while (tmem_cols < (unsigned)(p.nbuf * p.bn)) tmem_cols <<= 1;
+  const unsigned tmem_cols = (unsigned)p.k_tmem_cols;
 
   // Set-up is paid by every launch (measured: 1.8 us from entry to the first copy when one thread did
   // all of it): the tensor maps are prefetched at once, every barrier is initialised by its own
@@ -1831,7 +1832,21 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
   const int units = tc_units<CTAS>(ctx);
   long long grid = (p.items < units ? p.items : units) * CTAS;
   cfg.gridDim = dim3((unsigned)grid, 1, 1);
-  NITI_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, tc_gemm_kernel<CTAS>, ma, mb, p, acc, hdr, ctx->d_status, r.out, r.mask,
+  TcParams q = p;
+  {
+    const int gunits = (int)(grid / CTAS);
+    q.blk_per = (int)(p.items / gunits);
+    q.blk_extra = (int)(p.items % gunits);
+    const int eg = p.halo == 2 ? 1 : p.egroups;
+    q.k_wpq = EPI_PER_Q / eg;
+    const int chunks_all = p.bn / 32;
+    q.k_wpq_active = p.halo == 2 ? EPI_PER_Q : (chunks_all < q.k_wpq ? chunks_all : q.k_wpq);
+    q.k_epi_active = 4 * q.k_wpq_active;
+    int cols = 32;
+    while (cols < p.nbuf * p.bn) cols <<= 1;
+    q.k_tmem_cols = cols;
+  }
+  NITI_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, tc_gemm_kernel<CTAS>, ma, mb, q, acc, hdr, ctx->d_status, r.out, r.mask,
                                         r.s_a, r.s_w, r.s_out, r.b_out));
   ctx->launches++;
   ctx->tc_launches++;
