@@ -41,6 +41,8 @@ struct TcParams {
   // set-up arithmetic done on the host (integer divisions at kernel entry delay every launch)
   int blk_per, blk_extra;       // blocked assignment: items per CTA (pair) and how many take one more
   int k_wpq, k_wpq_active, k_epi_active, k_tmem_cols;
+  unsigned magic_w, magic_h;    // floor(2^32 / tiles) + 1 for w_tiles, h_tiles: n / d = umulhi(n, magic) while
+                                // n * d < 2^32 (0: divide)
   int quorum;                   // CTAs whose first tile must have reported before the speculative bit-width
                                 // is fixed (all of them when the sample is the whole tensor)
   int one_commit;               // resident-weights mode with as many patch stages as accumulator buffers:
@@ -362,12 +364,21 @@ __device__ __forceinline__ unsigned bytes_gt0(unsigned b) {
   return r;
 }
 
+// n / d with the host's reciprocal (exact while n * d < 2^32, which the host checked), else a division
+__device__ __forceinline__ int div_tiles(int n, int d, unsigned magic) {
+  return magic ? (int)__umulhi((unsigned)n, magic) : n / d;
+}
+// tile index -> (column tile, row tile, image) with two reciprocal multiplies
+__device__ __forceinline__ void tile_coords(const TcParams &p, int idx, int &wt, int &ht, int &bt) {
+  const int t = div_tiles(idx, p.w_tiles, p.magic_w);
+  wt = idx - t * p.w_tiles;
+  bt = div_tiles(t, p.h_tiles, p.magic_h);
+  ht = t - bt * p.h_tiles;
+}
 // Coordinates of an output tile / k-block in the pixel grid of a convolution.
 __device__ __forceinline__ void pixel_box(const TcParams &p, int idx, int &w0, int &h0, int &b0) {
-  int wt = idx % p.w_tiles;
-  int t = idx / p.w_tiles;
-  int ht = t % p.h_tiles;
-  int bt = t / p.h_tiles;
+  int wt, ht, bt;
+  tile_coords(p, idx, wt, ht, bt);
   w0 = wt * p.Wt; h0 = ht * p.Ht; b0 = bt * p.Bt;
 }
 
@@ -668,8 +679,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
         // consecutive items are consecutive tiles (blocked assignment): step the tile coordinates
-        int wt = (int)(first_item % p.w_tiles), ht = (int)((first_item / p.w_tiles) % p.h_tiles);
-        int bt = (int)(first_item / ((long long)p.w_tiles * p.h_tiles));
+        int wt, ht, bt;
+        tile_coords(p, first_item, wt, ht, bt);
         const unsigned free0 = p.one_commit ? tfull0 : empty0;   // "tile done" also frees the patch stage
         for (int item = first_item; ok && item < item_end; ++item) {
           if (owner == warp) {
@@ -699,10 +710,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (item == first_item) {
             decode_item(p, item, c_mu, c_nt, split);
             const int mt0 = c_mu * CTAS + (int)rank;
-            c_wt = mt0 % p.w_tiles;
-            const int t = mt0 / p.w_tiles;
-            c_ht = t % p.h_tiles;
-            c_bt = t / p.h_tiles;
+            tile_coords(p, mt0, c_wt, c_ht, c_bt);
           } else if (++c_nt == p.n_tiles_n) {
             c_nt = 0;
             ++c_mu;
@@ -1011,9 +1019,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (p.halo) {
         // 8 x 16 pixel tiles of one image, visited in order: coordinates are stepped, not divided
         if (use == (unsigned)egroup) {
-          h_wt = (int)(item % p.w_tiles);
-          h_ht = (int)((item / p.w_tiles) % p.h_tiles);
-          h_bt = (int)(item / ((long long)p.w_tiles * p.h_tiles));
+          tile_coords(p, item, h_wt, h_ht, h_bt);
         }
         const int w = h_wt * 8 + (row_in_tile & 7), h = h_ht * 16 + (row_in_tile >> 3);
         row_ok = w < p.PW && h < p.PH;
@@ -1845,6 +1851,11 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
     int cols = 32;
     while (cols < p.nbuf * p.bn) cols <<= 1;
     q.k_tmem_cols = cols;
+    // reciprocals for tile index -> coordinates; dividends stay below the tile count
+    const unsigned long long n_max = (unsigned long long)(p.w_tiles > 0 ? p.w_tiles : 1) * (p.h_tiles > 0 ? p.h_tiles : 1) *
+                                     (p.b_tiles > 0 ? p.b_tiles : 1) + 2;
+    q.magic_w = (p.w_tiles > 1 && n_max * p.w_tiles < (1ull << 32)) ? (unsigned)((1ull << 32) / p.w_tiles + 1) : 0u;
+    q.magic_h = (p.h_tiles > 1 && n_max * p.h_tiles < (1ull << 32)) ? (unsigned)((1ull << 32) / p.h_tiles + 1) : 0u;
   }
   NITI_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, tc_gemm_kernel<CTAS>, ma, mb, q, acc, hdr, ctx->d_status, r.out, r.mask,
                                         r.s_a, r.s_w, r.s_out, r.b_out));
