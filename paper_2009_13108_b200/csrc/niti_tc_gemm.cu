@@ -1097,6 +1097,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     use = (unsigned)egroup;
     unsigned ebuf = (unsigned)egroup, epar = 0;       // use % nbuf, (use / nbuf) & 1 (nbuf is a multiple of egroups)
+    // what the fused rounding needs and no tile changes: the rounding constants (replaced once, when the
+    // speculative binary point is agreed) and the alignment of the output and mask rows
+    RoundConst rk = make_round_const(bp, p.mbits, p.round_mode);
+    const bool io_aligned = ((p.gn & 31) == 0) && (((uintptr_t)out8 & 31) == 0) &&
+                            (mask8 == nullptr || ((uintptr_t)mask8 & 31) == 0);
     // this thread's pixel inside a pixel box (generic convolutions): the box sides are powers of two
     const int wt_d = p.Wt > 0 ? p.Wt : 1, ht_d = p.Ht > 0 ? p.Ht : 1;     // (unset for plain matrix multiplies)
     const int r_ww = row_in_tile % wt_d, r_t = row_in_tile / wt_d;
@@ -1230,6 +1235,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
           if (abort_flag) { ok = false; break; }
           bp = spec_bp_ready - 1;
+          rk = make_round_const(bp, p.mbits, p.round_mode);
         }
         if (p.epi_mode == EPI_SPECULATE && use == 0) {
           // first tile of this CTA: max only, then agree on the estimate with the whole grid
@@ -1317,16 +1323,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           __syncwarp();
           if (abort_flag) { ok = false; break; }
           bp = spec_bp_ready - 1;
+          rk = make_round_const(bp, p.mbits, p.round_mode);
         }
         const bool vec_ok = ((p.gn & 15) == 0) && ((col0 & 15) == 0);
         const bool vec32_ok = ((p.gn & 31) == 0) && ((col0 & 31) == 0) && (((uintptr_t)out8 & 31) == 0);
-        const RoundConst rk = make_round_const(bp, p.mbits, p.round_mode);
         // Whole 32-column chunks with 32-byte aligned rows (every layer of the networks): the chunk
         // loop below does nothing per chunk but load, round and store; pointers are stepped.  (The
         // epilogue warps share their schedulers' integer pipe, which is the bound of layers with few
         // input channels: every instruction here is paid for 16 times per tile.)
-        const bool whole_chunks = vec32_ok && ncols_valid >= (p.mrep > 1 ? p.bn_mma : p.bn) &&
-                                  (mask8 == nullptr || ((uintptr_t)mask8 & 31) == 0);
+        const bool whole_chunks = io_aligned && ((col0 & 31) == 0) && ncols_valid >= (p.mrep > 1 ? p.bn_mma : p.bn);
         if (whole_chunks) {
           const bool relu = p.relu != 0;
           const int cstep = 32 * wpq, bn = p.bn, bn_mma = p.mrep > 1 ? p.bn_mma : p.bn;
