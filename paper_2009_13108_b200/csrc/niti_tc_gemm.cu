@@ -1331,10 +1331,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // loop below does nothing per chunk but load, round and store; pointers are stepped.  (The
         // epilogue warps share their schedulers' integer pipe, which is the bound of layers with few
         // input channels: every instruction here is paid for 16 times per tile.)
-        const bool whole_chunks = io_aligned && ((col0 & 31) == 0) && ncols_valid >= (p.mrep > 1 ? p.bn_mma : p.bn);
+        const bool whole_chunks = io_aligned && ((col0 & 31) == 0) &&
+                                  (p.mrep > 1 ? ncols_valid >= p.bn_mma : (ncols_valid & 31) == 0);
         if (whole_chunks) {
           const bool relu = p.relu != 0;
-          const int cstep = 32 * wpq, bn = p.bn, bn_mma = p.mrep > 1 ? p.bn_mma : p.bn;
+          // (the last column tile of a row may be narrower than the tile: its chunks beyond the
+          // matrix are not read at all)
+          const int cstep = 32 * wpq, bn = p.mrep > 1 ? p.bn : (ncols_valid < p.bn ? ncols_valid : p.bn);
+          const int bn_mma = p.mrep > 1 ? p.bn_mma : p.bn;
           const long long row_off = out_row * p.gn + col0;
           const long long sub_stride = (long long)BM * p.gn;      // next 128-row tile of a row-batched item
           int8_t *drow = out8 + row_off;
@@ -1655,6 +1659,15 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
             {(cuuint32_t)p.kdepth, (cuuint32_t)p.Wt, (cuuint32_t)p.Ht, (cuuint32_t)p.Bt}, a_sw, g.p0};
       if (fwd) {
         p.bn = Cn >= 256 ? 256 : round_up32(Cn);
+        if (ctas == 2 && Cn > 256) {
+          // Whole waves: with 256-wide tiles the 14 x 14 layers are 98 tile pairs on 74 pairs of SMs, two
+          // waves of which the second is a third full; 192-wide tiles make 147 items, two full waves
+          // of items that each take three quarters of the time.
+          const long long mu = ((long long)p.w_tiles * p.h_tiles * p.b_tiles + 1) / 2, units = ctx->sm_count / 2;
+          const long long w256 = (mu * ((Cn + 255) / 256) + units - 1) / units;
+          const long long w192 = (mu * ((Cn + 191) / 192) + units - 1) / units;
+          if (w192 * 192 * 10 < w256 * 256 * 9) p.bn = 192;
+        }
         b_sw = p.kdepth;
         sb = {2, {(cuuint64_t)g.gk, (cuuint64_t)Cn}, {(cuuint64_t)g.gk}, {(cuuint32_t)p.kdepth, (cuuint32_t)(p.bn / ctas)}, b_sw, g.p1};
       } else {
