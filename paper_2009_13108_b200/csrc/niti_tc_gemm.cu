@@ -14,6 +14,7 @@
 // that frees the tensor memory.
 #include "niti_common.cuh"
 #include <math.h>
+#include <type_traits>
 
 namespace {
 
@@ -1102,6 +1103,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     RoundConst rk = make_round_const(bp, p.mbits, p.round_mode);
     const bool io_aligned = ((p.gn & 31) == 0) && (((uintptr_t)out8 & 31) == 0) &&
                             (mask8 == nullptr || ((uintptr_t)mask8 & 31) == 0);
+    // the lean loop takes over after a warp's first item (which may be the CTA's speculative first
+    // tile) when every chunk of every tile is whole and aligned
+    const bool lean_ok = (p.epi_mode == EPI_KNOWN_B || p.epi_mode == EPI_SPECULATE) && io_aligned && p.splits == 1 &&
+                         (p.bn & 31) == 0 && p.halo != 2 && p.kind != GK_CONV_WGRAD &&
+                         (p.mrep == 1 || (p.gn == p.bn_mma && mask8 == nullptr));
+    int lean_item = -1;
+    Extremes ex_all = {0, 0, 0u};
     // this thread's pixel inside a pixel box (generic convolutions): the box sides are powers of two
     const int wt_d = p.Wt > 0 ? p.Wt : 1, ht_d = p.Ht > 0 ? p.Ht : 1;     // (unset for plain matrix multiplies)
     const int r_ww = row_in_tile % wt_d, r_t = row_in_tile / wt_d;
@@ -1443,6 +1451,106 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (CTAS == 2 && rank != 0) mbar_arrive_cluster(lead_tempty0 + 8 * buf);
         else mbar_arrive(tempty0 + 8 * buf);
       }
+      if (lean_ok && rk.aligned) {                 // the rest of this warp's items: lean loop below
+        lean_item = item + item_step * egroups;
+        use += (unsigned)egroups;
+        break;
+      }
+    }
+    // ---- lean loop: fused rounding of whole, aligned chunks (every layer of the networks) ----
+    // The epilogue warps share their schedulers' integer pipe with everything else, and with few
+    // input channels that pipe is the bound of the whole kernel: per tile and per chunk this loop
+    // executes only what changes (measured on the first layer: the general loop above spends a third
+    // of its integer instructions on tests whose outcome is the same for every tile).
+    if (ok && lean_item >= 0) {
+      auto lean = [&](auto relu_c, auto mask_c, auto batched_c) {
+        constexpr bool RELU = decltype(relu_c)::value, MASK = decltype(mask_c)::value, BATCHED = decltype(batched_c)::value;
+        const int kind = p.halo ? 0 : ((p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) ? 1 : 2);
+        const int istep = item_step * egroups, nbuf = p.nbuf, bn = p.bn, n_tiles_n = p.n_tiles_n;
+        const int cstep = 32 * wpq, c_first = 32 * chunk_phase;
+        const long long gn = p.gn, gm = p.gm;
+        const int bn_mma = BATCHED ? p.bn_mma : p.bn;
+        const long long sub_stride = (long long)BM * gn;
+        const bool counted = p.blocked && p.raster_g <= 0;     // consecutive items: (mu, nt) are stepped
+        int mu = 0, nt = 0, split = 0;
+        if (kind != 0) decode_item(p, lean_item, mu, nt, split);
+        for (int item = lean_item; item < item_end; item += istep) {
+          const unsigned buf = ebuf, tpar = epar;
+          ebuf += (unsigned)egroups;
+          if (ebuf >= (unsigned)nbuf) { ebuf -= (unsigned)nbuf; epar ^= 1u; }
+          long long out_row;
+          bool row_ok;
+          if (kind == 0) {
+            const int w = h_wt * 8 + (row_in_tile & 7), h = h_ht * 16 + (row_in_tile >> 3);
+            row_ok = w < p.PW && h < p.PH;
+            out_row = ((long long)h_bt * p.PH + h) * p.PW + w;
+            h_wt += egroups;
+            while (h_wt >= p.w_tiles) { h_wt -= p.w_tiles; if (++h_ht == p.h_tiles) { h_ht = 0; ++h_bt; } }
+          } else if (kind == 1) {
+            int w0, h0, b0;
+            pixel_box(p, mu * CTAS + (int)rank, w0, h0, b0);
+            const int w = w0 + r_ww, h = h0 + r_hh, b = b0 + r_bb;
+            row_ok = w < p.PW && h < p.PH && b < p.PB;
+            out_row = ((long long)b * p.PH + h) * p.PW + w;
+          } else {
+            out_row = (long long)(mu * CTAS + (int)rank) * (BM * p.mrep) + row_in_tile;
+            row_ok = out_row < gm;
+          }
+          const int col0 = nt * bn;
+          int cend = BATCHED ? bn : (int)(gn - col0);          // (whole chunks: gn is a multiple of 32)
+          if (cend > bn) cend = bn;
+          if (kind != 0) {                                      // next item of this warp
+            if (counted) { nt += egroups; while (nt >= n_tiles_n) { nt -= n_tiles_n; ++mu; } }
+            else if (item + istep < item_end) decode_item(p, item + istep, mu, nt, split);
+          }
+          if (!mbar_wait(tfull0 + 8 * buf, tpar, &abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const unsigned tm_row = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * (unsigned)bn;
+          const long long row_off = out_row * gn + col0;
+          int8_t *drow = out8 + row_off;
+          const int8_t *mrow = MASK ? mask8 + row_off : nullptr;
+          long long orow = out_row;
+          int cc = c_first;
+          if (BATCHED) while (cc >= bn_mma) { cc -= bn_mma; orow += BM; drow += sub_stride; if (MASK) mrow += sub_stride; }
+          for (int c = c_first; c < cend; c += cstep) {
+            int v[32];
+            const bool rok = BATCHED ? (row_ok && orow < gm) : row_ok;
+            unsigned m[8];
+            if (MASK && rok)
+              asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                           : "=r"(m[0]), "=r"(m[1]), "=r"(m[2]), "=r"(m[3]), "=r"(m[4]), "=r"(m[5]), "=r"(m[6]), "=r"(m[7])
+                           : "l"(mrow + cc));
+            tc_ld32(tm_row + (unsigned)c, v);
+            if (rok) {
+              unsigned w8[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                w8[j] = round_pack4_aligned<RELU>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, ex_all);
+                if (MASK) w8[j] &= bytes_gt0(m[j]);
+              }
+              asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                           ::"l"(drow + cc), "r"(w8[0]), "r"(w8[1]), "r"(w8[2]), "r"(w8[3]), "r"(w8[4]), "r"(w8[5]),
+                             "r"(w8[6]), "r"(w8[7])
+                           : "memory");
+            }
+            cc += cstep;
+            if (BATCHED) while (cc >= bn_mma) { cc -= bn_mma; orow += BM; drow += sub_stride; if (MASK) mrow += sub_stride; }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            if (CTAS == 2 && rank != 0) mbar_arrive_cluster(lead_tempty0 + 8 * buf);
+            else mbar_arrive(tempty0 + 8 * buf);
+          }
+        }
+      };
+      using T = std::true_type;
+      using F = std::false_type;
+      const bool relu = p.relu != 0, masked = mask8 != nullptr, batched = p.mrep > 1;
+      if (batched) { if (relu) lean(T{}, F{}, T{}); else lean(F{}, F{}, T{}); }      // (row-batched: forward only)
+      else if (relu) { if (masked) lean(T{}, T{}, F{}); else lean(T{}, F{}, F{}); }
+      else { if (masked) lean(F{}, T{}, F{}); else lean(F{}, F{}, F{}); }
+      mx |= ex_all.magnitude_bits();
     }
     if (p.epi_mode == EPI_SPILL || p.epi_mode == EPI_SPECULATE) {
       for (int o = 16; o > 0; o >>= 1) {
