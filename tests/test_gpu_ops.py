@@ -102,6 +102,9 @@ CONV_SHAPES = [(2, 8, 8, 3, 16), (2, 16, 16, 64, 64), (4, 8, 8, 128, 256), (8, 4
                (2, 32, 32, 32, 64), (3, 28, 28, 1, 32), (2, 28, 28, 32, 64), (32, 2, 2, 512, 512),
                (1, 56, 56, 64, 128), (2, 12, 20, 96, 160), (2, 24, 40, 128, 128), (1, 64, 48, 64, 64),
                (2, 18, 10, 128, 64), (3, 30, 22, 32, 96),
+               # more than 256 output channels: with CTA pairs (engine 3) the tile is 192 columns wide
+               # and the last column tile narrower
+               (4, 8, 8, 64, 320),
                # RGB first layers: staged gather (W % 4 == 0; one with more pixel groups than threads)
                # and the generic gather (W % 4 != 0)
                (3, 20, 36, 3, 32), (1, 6, 520, 3, 16), (2, 9, 10, 3, 16)]
