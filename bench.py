@@ -374,7 +374,7 @@ def run_ours(args):
     input_digests = {"x": hashlib.sha256(memoryview(x).cast("B")).hexdigest()[:16],
                      "labels": hashlib.sha256(memoryview(labels).cast("B")).hexdigest()[:16],
                      "weights": wh.hexdigest()[:16]}      # guards against drift of the seeded generator
-    tr = NitiTrainer(niti, net, weights)
+    tr = NitiTrainer(niti, net, weights, fused_update=args.fused_update)
     xh = torch.from_numpy(x).pin_memory()
     lh = torch.from_numpy(labels).pin_memory()
     tr.load_batch(xh, lh)
@@ -474,6 +474,7 @@ def run_ours(args):
                    "l2": "working set (activations + int32 scratch) exceeds the 126 MB L2",
                    "state": "weights restored to the seeded initial values before every step",
                    "launch": "cuda-graph replay" if args.graph else "eager",
+                   "weight_update": "fused with the weight gradient" if args.fused_update else "separate call",
                    "parallelism": "replicas" if world > 1 else "single",
                    "inputs_sha256_16": input_digests},
         "step_tops": ops_step / (ms / args.steps) / 1e9,
@@ -507,6 +508,8 @@ def main():
     ap.add_argument("--no-gemm", dest="gemm", action="store_false")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="issue every launch from Python instead of replaying a CUDA graph of the step")
+    ap.add_argument("--fused-update", dest="fused_update", action="store_true",
+                    help="weight gradient and weight update in one library call (default: two calls)")
     ap.add_argument("--gemm-shape", default=None,
                     help="MxNxK: time only the fused GEMM at this shape (for profiling a small case)")
     ap.add_argument("--iters", type=int, default=10)

@@ -63,6 +63,8 @@ extern "C" {
 #define NITI_OP_CONV_DGRAD 3  /* same                              */
 #define NITI_OP_CONV_WGRAD 4  /* same                              */
 #define NITI_OP_INT_XENT 5    /* dims = {B, N}                    */
+#define NITI_OP_LINEAR_BWD_UPDATE 6 /* dims = {M, N, K}            */
+#define NITI_OP_CONV_WGRAD_UPDATE 7 /* dims as NITI_OP_CONV_FWD    */
 
 /* device status bits returned by niti_check() */
 #define NITI_DEV_TIMEOUT 1u      /* a bounded wait inside a kernel gave up     */
@@ -177,6 +179,28 @@ int niti_conv_dgrad(niti_ctx *ctx, void *stream, const int8_t *e, const int8_t *
 int niti_conv_wgrad(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
                     int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
                     int m_u, int round_mode, void *ws, size_t ws_bytes);
+
+/* Weight gradient fused with the weight update (Section 3.3: the gradient is
+ * rounded to m_u bits "and fused with the weight update"; Algorithm 1, last two
+ * lines of the reverse loop).  Same arithmetic as niti_conv_wgrad followed by
+ * niti_int_sgd_update, with w [Cout][R][S][Cin] updated in place,
+ *   w <- clamp(w - round(g32), -127, 127),
+ * and the int8 gradient never returned: where the contraction is split over
+ * CTAs (every convolution of the networks) the rounding pass over the int32
+ * sums subtracts from w directly; otherwise the gradient passes through the
+ * workspace.  b_g receives the bit-width of g32.  Workspace:
+ * NITI_OP_CONV_WGRAD_UPDATE.  w must be 16-byte aligned. */
+int niti_conv_wgrad_update(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *w,
+                           int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
+                           int m_u, int round_mode, void *ws, size_t ws_bytes);
+
+/* niti_linear_bwd with the weight update fused in: e_prev (may be NULL) is
+ * computed from the weights as they are on entry, then w [N][K] is updated in
+ * place with the rounded weight gradient, which is not returned.  Workspace:
+ * NITI_OP_LINEAR_BWD_UPDATE. */
+int niti_linear_bwd_update(niti_ctx *ctx, void *stream, const int8_t *a, const int8_t *e, int8_t *w,
+                           int8_t *e_prev, const int8_t *relu_mask_src, int32_t *b_e, int32_t *b_g,
+                           int M, int N, int K, int m_u, int round_mode, void *ws, size_t ws_bytes);
 
 /* Integer cross-entropy gradient (Section 3.5, Eq. 1-4).  Per sample r:
  *   e32[r][i] = T_i - [i == labels[r]] * sum_j T_j

@@ -16,13 +16,14 @@ _LIB_PATH = os.path.join(_HERE, "libniti_b200.so")
 OK, ERR_ARG, ERR_SHAPE, ERR_WORKSPACE, ERR_RANGE, ERR_CUDA, ERR_DEVICE = range(7)
 ROUND_PSR, ROUND_NEAREST = 0, 1
 OP_LINEAR_FWD, OP_LINEAR_BWD, OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_INT_XENT = range(6)
+OP_LINEAR_BWD_UPDATE, OP_CONV_WGRAD_UPDATE = 6, 7
 
 EXPORTS = [
     "niti_create", "niti_destroy", "niti_last_error", "niti_check", "niti_workspace_bytes",
     "niti_set_engine", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
     "niti_redo_count", "niti_selftest_timeout", "niti_profile_enable", "niti_profile_read_launches",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
-    "niti_conv_dgrad", "niti_conv_wgrad", "niti_int_xent", "niti_int_xent_noalloc", "niti_int_sgd_update",
+    "niti_conv_dgrad", "niti_conv_wgrad", "niti_conv_wgrad_update", "niti_linear_bwd_update", "niti_int_xent", "niti_int_xent_noalloc", "niti_int_sgd_update",
     "niti_relu_fwd",
     "niti_relu_bwd", "niti_maxpool2_fwd", "niti_maxpool2_bwd",
 ]
@@ -71,6 +72,8 @@ def load_library():
     lib.niti_conv_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
     lib.niti_conv_dgrad.argtypes = [vp, vp, vp, vp, vp, vp, vp] + [i32] * 9 + [vp, sz]
     lib.niti_conv_wgrad.argtypes = [vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
+    lib.niti_conv_wgrad_update.argtypes = [vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
+    lib.niti_linear_bwd_update.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, sz]
     lib.niti_int_xent.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, sz]
     lib.niti_int_xent_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32]
     lib.niti_int_sgd_update.argtypes = [vp, vp, vp, vp, i64]
@@ -249,6 +252,33 @@ class Niti:
                                           _ptr(b_g), B, H, W, Ci, Co, R, S, pad, m_u, round_mode,
                                           ws, wsb))
         return g, b_g
+
+    def conv_wgrad_update(self, x, e, w, b_g=None, pad=1, m_u=5, round_mode=ROUND_PSR):
+        """Weight gradient of the convolution subtracted from w in place (the gradient is not returned)."""
+        B, H, W, Ci = x.shape
+        Co, R, S, _ = w.shape
+        b_g = b_g if b_g is not None else self.scalar()
+        ws, wsb = self._ws_for(OP_CONV_WGRAD_UPDATE, [B, H, W, Ci, Co, R, S, pad])
+        self._ck(self.lib.niti_conv_wgrad_update(self.h, self._stream(), _ptr(x), _ptr(e), _ptr(w),
+                                                 _ptr(b_g), B, H, W, Ci, Co, R, S, pad, m_u,
+                                                 round_mode, ws, wsb))
+        return w, b_g
+
+    def linear_bwd_update(self, a, e, w, need_e_prev=True, relu_mask_src=None, e_prev=None,
+                          b_e=None, b_g=None, m_u=5, round_mode=ROUND_PSR):
+        """linear_bwd with the weight update fused in: e_prev from the old weights, then w updated in place."""
+        M, K = a.shape
+        N = e.shape[1]
+        if need_e_prev and e_prev is None:
+            e_prev = torch.empty((M, K), dtype=torch.int8, device=self.device)
+        b_e = b_e if b_e is not None else self.scalar()
+        b_g = b_g if b_g is not None else self.scalar()
+        ws, wsb = self._ws_for(OP_LINEAR_BWD_UPDATE, [M, N, K])
+        self._ck(self.lib.niti_linear_bwd_update(self.h, self._stream(), _ptr(a), _ptr(e), _ptr(w),
+                                                 _ptr(e_prev) if need_e_prev else None,
+                                                 _ptr(relu_mask_src), _ptr(b_e), _ptr(b_g), M, N, K,
+                                                 m_u, round_mode, ws, wsb))
+        return (e_prev if need_e_prev else None), b_e, b_g
 
     def int_xent(self, a, s_a, labels, e=None, b_e=None, n_correct=None, round_mode=ROUND_PSR):
         B, N = a.shape

@@ -180,6 +180,7 @@ extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
       outs = (size_t)(d[0] * d[1]);
       extra = niti_tc_scratch_bytes(p);
       break;
+    case NITI_OP_LINEAR_BWD_UPDATE:
     case NITI_OP_LINEAR_BWD: {
       if (nd != 3 || d[0] <= 0 || d[1] <= 0 || d[2] <= 0) return 0;
       size_t a = (size_t)(d[0] * d[2]), b = (size_t)(d[1] * d[2]);
@@ -189,14 +190,18 @@ extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
       size_t e1 = niti_tc_scratch_bytes(p), e2 = niti_tc_scratch_bytes(p2);
       extra = e1 > e2 ? e1 : e2;
       if (d[1] % 16) extra += round_up((size_t)d[0] * (size_t)((d[1] + 15) / 16 * 16), 256);   // e with padded rows
+      if (op == NITI_OP_LINEAR_BWD_UPDATE) extra = round_up(extra, 256) + round_up(b, 256);    // scratch gradient
       break;
     }
     case NITI_OP_CONV_FWD:
     case NITI_OP_CONV_DGRAD:
+    case NITI_OP_CONV_WGRAD_UPDATE:
     case NITI_OP_CONV_WGRAD: {
       if (nd != 8) return 0;
       for (int i = 0; i < 7; ++i)
         if (d[i] <= 0) return 0;
+      const bool upd = op == NITI_OP_CONV_WGRAD_UPDATE;
+      if (upd) op = NITI_OP_CONV_WGRAD;
       int kind = op == NITI_OP_CONV_FWD ? GK_CONV_FWD : (op == NITI_OP_CONV_DGRAD ? GK_CONV_DGRAD : GK_CONV_WGRAD);
       if (!fill_conv(p, kind, (int)d[0], (int)d[1], (int)d[2], (int)d[3], (int)d[4], (int)d[5], (int)d[6], (int)d[7]))
         return 0;
@@ -207,6 +212,7 @@ extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
         extra += round_up(M * 32, 256) + round_up((size_t)d[4] * 32, 256) + round_up((size_t)d[4] * 32 * 4, 256);
         if (op == NITI_OP_CONV_FWD && outs < M * (size_t)d[4]) outs = M * (size_t)d[4];
       }
+      if (upd) extra = round_up(extra, 256) + round_up((size_t)(p.gm * p.gn), 256);             // scratch gradient
       break;
     }
     case NITI_OP_INT_XENT:
@@ -220,11 +226,17 @@ extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
 
 static inline bool misaligned16(const void *p) { return ((uintptr_t)p & 15) != 0; }
 
+int niti_launch_sgd_update(niti_ctx *ctx, cudaStream_t st, int8_t *w, const int8_t *g, long long n);
+
 // One matrix multiply of Algorithm 1 followed by EffectiveBitwidth + ShiftAndRound.
+// update_w != null (weight gradients): the rounded gradient is not returned but subtracted from the
+// weights in place.  When the int32 accumulators exist (split contractions) the rounding pass does
+// that itself and the int8 gradient is never stored; when the multiply rounds in its own epilogue,
+// `out` is a scratch tensor and the plain update kernel follows.
 static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, void *ws, size_t ws_bytes,
                           size_t need, int8_t *out, int mbits, int round_mode, int relu,
                           const int8_t *mask, const int32_t *s_a, const int32_t *s_w, int32_t *s_out,
-                          int32_t *b_out) {
+                          int32_t *b_out, int8_t *update_w = nullptr) {
   if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
     return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
   WsHeader *hdr = (WsHeader *)ws;
@@ -236,9 +248,10 @@ static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, 
   RoundSpec rs = {out, mask, mbits, round_mode, relu, s_a, s_w, s_out, b_out};
   if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, rs, acc, hdr, &fused);
   if (rc == NITI_ERR_SHAPE) rc = niti_simt_gemm(ctx, st, p, acc, hdr);
-  if (rc != NITI_OK || fused) return rc;
+  if (rc != NITI_OK) return rc;
+  if (fused) return update_w ? niti_launch_sgd_update(ctx, st, update_w, out, p.gm * p.gn) : NITI_OK;
   return niti_launch_round(ctx, st, acc, hdr, out, p.gm * p.gn, mbits, round_mode, relu, mask, s_a, s_w,
-                           s_out, b_out);
+                           s_out, b_out, update_w);
 }
 
 extern "C" int niti_linear_fwd(niti_ctx *ctx, void *stream, const int8_t *a, const int32_t *s_a,
@@ -258,24 +271,31 @@ extern "C" int niti_linear_fwd(niti_ctx *ctx, void *stream, const int8_t *a, con
                         nullptr, s_a, s_w, s_out, b_out);
 }
 
-extern "C" int niti_linear_bwd(niti_ctx *ctx, void *stream, const int8_t *a, const int8_t *e,
-                               const int8_t *w, int8_t *e_prev, const int8_t *relu_mask_src, int8_t *g,
-                               int32_t *b_e, int32_t *b_g, int M, int N, int K, int m_u, int round_mode,
-                               void *ws, size_t ws_bytes) {
+// Backward pass of a fully connected layer; `g` receives the rounded weight gradient, or, with
+// update_w, the gradient is subtracted from update_w (= w) in place after the error of the layer
+// below has been computed from the old weights.
+static int linear_bwd_impl(niti_ctx *ctx, void *stream, const int8_t *a, const int8_t *e, const int8_t *w,
+                           int8_t *e_prev, const int8_t *relu_mask_src, int8_t *g, int8_t *update_w,
+                           int32_t *b_e, int32_t *b_g, int M, int N, int K, int m_u, int round_mode, void *ws,
+                           size_t ws_bytes, const char *who) {
   if (!ctx) return NITI_ERR_ARG;
-  if (!a || !e || !w || !g || M <= 0 || N <= 0 || K <= 0 || m_u < 1 || m_u > 7 ||
+  if (!a || !e || !w || (!g && !update_w) || M <= 0 || N <= 0 || K <= 0 || m_u < 1 || m_u > 7 ||
       (round_mode != 0 && round_mode != 1) || misaligned16(a) || misaligned16(e) || misaligned16(w) ||
-      misaligned16(g) || misaligned16(e_prev) || misaligned16(relu_mask_src))
-    return niti_fail(ctx, NITI_ERR_ARG, "niti_linear_bwd: bad argument (pointers must be 16-byte aligned)");
+      misaligned16(g) || misaligned16(e_prev) || misaligned16(relu_mask_src)) {
+    snprintf(ctx->err, sizeof(ctx->err), "%s: bad argument (pointers must be 16-byte aligned)", who);
+    return NITI_ERR_ARG;
+  }
   int64_t dims[3] = {M, N, K};
-  size_t need = niti_workspace_bytes(NITI_OP_LINEAR_BWD, dims, 3);
+  const size_t need_base = niti_workspace_bytes(NITI_OP_LINEAR_BWD, dims, 3);
+  const size_t need = update_w ? niti_workspace_bytes(NITI_OP_LINEAR_BWD_UPDATE, dims, 3) : need_base;
+  if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
+    return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+  if (update_w) g = (int8_t *)((char *)ws + need_base);       // scratch, used only if the multiply rounds by itself
   // TMA needs 16-byte row pitches: an error tensor with N % 16 != 0 (10 or 1000 classes) is copied
   // once into rows padded to the next multiple of 16 for the tensor-core engine
   const int8_t *e_tc = e;
   long long e_ld = 0;
   if ((N % 16) != 0 && N >= 32 && ctx->engine != 1) {
-    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
-      return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
     const int pitch = (N + 15) / 16 * 16;
     size_t a_out = (size_t)M * K, b_out = (size_t)N * K;
     int8_t *epad = (int8_t *)((char *)ws + NITI_WS_HEADER + round_up((a_out > b_out ? a_out : b_out) * 4, 256));
@@ -285,15 +305,39 @@ extern "C" int niti_linear_bwd(niti_ctx *ctx, void *stream, const int8_t *a, con
     e_ld = pitch;
   }
   GemmProblem p;
+  int rc;
+  if (e_prev && update_w) {                // the error below needs the weights as they were
+    fill_fc(p, GK_FC_DGRAD, M, N, K);
+    p.p0 = e_tc; p.p1 = w; p.ld0 = e_ld;
+    rc = run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, e_prev, 7, round_mode, 0,
+                        relu_mask_src, nullptr, nullptr, nullptr, b_e);
+    if (rc != NITI_OK) return rc;
+  }
   fill_fc(p, GK_FC_WGRAD, M, N, K);
   p.p0 = e_tc; p.p1 = a; p.ld0 = e_ld;
-  int rc = run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, g, m_u, round_mode, 0, nullptr,
-                          nullptr, nullptr, nullptr, b_g);
-  if (rc != NITI_OK || !e_prev) return rc;
+  rc = run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, g, m_u, round_mode, 0, nullptr,
+                      nullptr, nullptr, nullptr, b_g, update_w);
+  if (rc != NITI_OK || !e_prev || update_w) return rc;
   fill_fc(p, GK_FC_DGRAD, M, N, K);
   p.p0 = e_tc; p.p1 = w; p.ld0 = e_ld;
   return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, e_prev, 7, round_mode, 0,
                         relu_mask_src, nullptr, nullptr, nullptr, b_e);
+}
+
+extern "C" int niti_linear_bwd(niti_ctx *ctx, void *stream, const int8_t *a, const int8_t *e,
+                               const int8_t *w, int8_t *e_prev, const int8_t *relu_mask_src, int8_t *g,
+                               int32_t *b_e, int32_t *b_g, int M, int N, int K, int m_u, int round_mode,
+                               void *ws, size_t ws_bytes) {
+  if (ctx && !g) return niti_fail(ctx, NITI_ERR_ARG, "niti_linear_bwd: bad argument (g is null)");
+  return linear_bwd_impl(ctx, stream, a, e, w, e_prev, relu_mask_src, g, nullptr, b_e, b_g, M, N, K, m_u,
+                         round_mode, ws, ws_bytes, "niti_linear_bwd");
+}
+
+extern "C" int niti_linear_bwd_update(niti_ctx *ctx, void *stream, const int8_t *a, const int8_t *e, int8_t *w,
+                                      int8_t *e_prev, const int8_t *relu_mask_src, int32_t *b_e, int32_t *b_g,
+                                      int M, int N, int K, int m_u, int round_mode, void *ws, size_t ws_bytes) {
+  return linear_bwd_impl(ctx, stream, a, e, w, e_prev, relu_mask_src, nullptr, w, b_e, b_g, M, N, K, m_u,
+                         round_mode, ws, ws_bytes, "niti_linear_bwd_update");
 }
 
 static int conv_args_ok(int B, int H, int W, int Ci, int Co, int R, int S, int pad, int round_mode) {
@@ -354,22 +398,28 @@ extern "C" int niti_conv_dgrad(niti_ctx *ctx, void *stream, const int8_t *e, con
                         relu_mask_src, nullptr, nullptr, nullptr, b_e);
 }
 
-extern "C" int niti_conv_wgrad(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
-                               int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
-                               int m_u, int round_mode, void *ws, size_t ws_bytes) {
+// Weight gradient of a convolution; with update_w the rounded gradient is subtracted from the
+// weights in place instead of being returned.
+static int conv_wgrad_impl(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
+                           int8_t *update_w, int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S,
+                           int pad, int m_u, int round_mode, void *ws, size_t ws_bytes, const char *who) {
   if (!ctx) return NITI_ERR_ARG;
   GemmProblem p;
   memset(&p, 0, sizeof(p));
-  if (!x || !e || !g || m_u < 1 || m_u > 7 || !conv_args_ok(B, H, W, Cin, Cout, R, S, pad, round_mode) ||
-      misaligned16(x) || misaligned16(e) || misaligned16(g) ||
-      !fill_conv(p, GK_CONV_WGRAD, B, H, W, Cin, Cout, R, S, pad))
-    return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_wgrad: bad argument (pointers must be 16-byte aligned)");
+  if (!x || !e || (!g && !update_w) || m_u < 1 || m_u > 7 || !conv_args_ok(B, H, W, Cin, Cout, R, S, pad, round_mode) ||
+      misaligned16(x) || misaligned16(e) || misaligned16(g) || misaligned16(update_w) ||
+      !fill_conv(p, GK_CONV_WGRAD, B, H, W, Cin, Cout, R, S, pad)) {
+    snprintf(ctx->err, sizeof(ctx->err), "%s: bad argument (pointers must be 16-byte aligned)", who);
+    return NITI_ERR_ARG;
+  }
   p.p0 = e; p.p1 = x;
   int64_t dims[8] = {B, H, W, Cin, Cout, R, S, pad};
-  const size_t need = niti_workspace_bytes(NITI_OP_CONV_WGRAD, dims, 8);
+  const size_t need_base = niti_workspace_bytes(NITI_OP_CONV_WGRAD, dims, 8);
+  const size_t need = update_w ? niti_workspace_bytes(NITI_OP_CONV_WGRAD_UPDATE, dims, 8) : need_base;
+  if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
+    return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+  if (update_w) g = (int8_t *)((char *)ws + need_base);       // scratch, used only where the rounding stores int8
   if (few_channel_conv(Cin, R, S) && ctx->engine != 1 && (Cout % 16) == 0) {
-    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
-      return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
     // g32[co][k] = sum_pix e[pix][co] * xcol[pix][k] over the gathered rows (k < 32), then the first
     // R*S*Cin columns are rounded into g
     cudaStream_t st = (cudaStream_t)stream;
@@ -393,8 +443,26 @@ extern "C" int niti_conv_wgrad(niti_ctx *ctx, void *stream, const int8_t *x, con
     ctx->engine = saved;
     if (rc == NITI_ERR_SHAPE) rc = niti_simt_gemm(ctx, st, q, acc32, hdr);
     if (rc != NITI_OK) return rc;
-    return niti_launch_round_compact32(ctx, st, acc32, hdr, g, Cout, R * S * Cin, m_u, round_mode, b_g);
+    rc = niti_launch_round_compact32(ctx, st, acc32, hdr, g, Cout, R * S * Cin, m_u, round_mode, b_g);
+    if (rc != NITI_OK || !update_w) return rc;
+    return niti_launch_sgd_update(ctx, st, update_w, g, (long long)Cout * R * S * Cin);
   }
   return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, g, m_u, round_mode, 0, nullptr,
-                        nullptr, nullptr, nullptr, b_g);
+                        nullptr, nullptr, nullptr, b_g, update_w);
+}
+
+extern "C" int niti_conv_wgrad(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
+                               int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
+                               int m_u, int round_mode, void *ws, size_t ws_bytes) {
+  if (ctx && !g) return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_wgrad: bad argument (g is null)");
+  return conv_wgrad_impl(ctx, stream, x, e, g, nullptr, b_g, B, H, W, Cin, Cout, R, S, pad, m_u, round_mode, ws,
+                         ws_bytes, "niti_conv_wgrad");
+}
+
+extern "C" int niti_conv_wgrad_update(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *w,
+                                      int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
+                                      int m_u, int round_mode, void *ws, size_t ws_bytes) {
+  if (ctx && !w) return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_wgrad_update: bad argument (w is null)");
+  return conv_wgrad_impl(ctx, stream, x, e, nullptr, w, b_g, B, H, W, Cin, Cout, R, S, pad, m_u, round_mode, ws,
+                         ws_bytes, "niti_conv_wgrad_update");
 }

@@ -128,4 +128,4 @@ size_t niti_tc_scratch_bytes(const GemmProblem &p);
 int niti_launch_round(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, const WsHeader *hdr,
                       int8_t *out, long long n, int mbits, int round_mode, int relu,
                       const int8_t *mask, const int32_t *s_a, const int32_t *s_w, int32_t *s_out,
-                      int32_t *b_out);
+                      int32_t *b_out, int8_t *upd_w = nullptr);

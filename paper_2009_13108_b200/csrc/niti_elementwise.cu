@@ -7,12 +7,17 @@
 // Shift-and-round pass over an int32 accumulator tensor (Algorithm 2, with Algorithm 3 rounding).
 // Every thread handles 16 consecutive elements: four 16-byte loads, one 16-byte store.
 // ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned sat_sub_clamp127(unsigned w, unsigned g) {
+  // per byte: clamp(w - g, -127, 127): saturating subtract gives [-128, 127]; lift -128 to -127
+  return __vmaxs4(__vsubss4(w, g), 0x81818181u);
+}
+
 __global__ void __launch_bounds__(256)
 round_i32_kernel(const int32_t *__restrict__ acc, const WsHeader *__restrict__ hdr,
                  int8_t *__restrict__ out, long long n, int mbits, int round_mode, int relu,
                  const int8_t *__restrict__ mask, const int32_t *__restrict__ s_a,
                  const int32_t *__restrict__ s_w, int32_t *__restrict__ s_out,
-                 int32_t *__restrict__ b_out, uint32_t *__restrict__ status) {
+                 int32_t *__restrict__ b_out, uint32_t *__restrict__ status, int8_t *__restrict__ upd_w) {
   const int b = niti_bitlen32(hdr->maxabs32);
   const int bp = b > mbits ? b - mbits : 0;
   const unsigned qmax = (1u << mbits) - 1u;
@@ -50,7 +55,16 @@ round_i32_kernel(const int32_t *__restrict__ acc, const WsHeader *__restrict__ h
       o[w] = word;
     }
     int4 ov = make_int4(o[0] & mk.x, o[1] & mk.y, o[2] & mk.z, o[3] & mk.w);
-    *(reinterpret_cast<int4 *>(out) + v) = ov;
+    if (upd_w) {
+      // weight update fused with the rounding of the weight gradient (Section 3.3: the rounded
+      // gradient is never stored): w <- clamp(w - q, -127, 127)
+      int4 wv = *(reinterpret_cast<int4 *>(upd_w) + v);
+      wv.x = sat_sub_clamp127(wv.x, ov.x); wv.y = sat_sub_clamp127(wv.y, ov.y);
+      wv.z = sat_sub_clamp127(wv.z, ov.z); wv.w = sat_sub_clamp127(wv.w, ov.w);
+      *(reinterpret_cast<int4 *>(upd_w) + v) = wv;
+    } else {
+      *(reinterpret_cast<int4 *>(out) + v) = ov;
+    }
   }
   // ragged tail (fewer than 16 elements)
   long long t = (nvec << 4) + (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -58,21 +72,26 @@ round_i32_kernel(const int32_t *__restrict__ acc, const WsHeader *__restrict__ h
     int q = niti_round_i32(acc[t], bp, qmax, round_mode);
     if (relu && q < 0) q = 0;
     if (mask && mask[t] <= 0) q = 0;
-    out[t] = (int8_t)q;
+    if (upd_w) {
+      int d = (int)upd_w[t] - q;
+      upd_w[t] = (int8_t)(d > 127 ? 127 : (d < -127 ? -127 : d));
+    } else {
+      out[t] = (int8_t)q;
+    }
   }
 }
 
 int niti_launch_round(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, const WsHeader *hdr,
                       int8_t *out, long long n, int mbits, int round_mode, int relu,
                       const int8_t *mask, const int32_t *s_a, const int32_t *s_w, int32_t *s_out,
-                      int32_t *b_out) {
+                      int32_t *b_out, int8_t *upd_w) {
   long long nvec = n >> 4;
   long long blocks = (nvec + 255) / 256;
   long long cap = (long long)ctx->sm_count * 16;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   round_i32_kernel<<<(unsigned)blocks, 256, 0, st>>>(acc, hdr, out, n, mbits, round_mode, relu, mask,
-                                                     s_a, s_w, s_out, b_out, ctx->d_status);
+                                                     s_a, s_w, s_out, b_out, ctx->d_status, upd_w);
   ctx->launches++;
   NITI_CUDA_TRY(ctx, cudaGetLastError());
   return NITI_OK;
@@ -648,10 +667,6 @@ extern "C" int niti_int_xent_noalloc(void *stream, const int8_t *a, const int32_
 // ---------------------------------------------------------------------------------------------
 // Byte-wise SIMD elementwise ops: 16 int8 per thread per iteration (one 16-byte load per operand).
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned sat_sub_clamp127(unsigned w, unsigned g) {
-  // per byte: clamp(w - g, -127, 127): saturating subtract gives [-128, 127]; lift -128 to -127
-  return __vmaxs4(__vsubss4(w, g), 0x81818181u);
-}
 
 __global__ void __launch_bounds__(256)
 sgd_update_kernel(int8_t *__restrict__ w, const int8_t *__restrict__ g, long long n) {
@@ -805,6 +820,13 @@ static inline unsigned ew_blocks(niti_ctx *ctx, long long work_items) {
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   return (unsigned)blocks;
+}
+
+int niti_launch_sgd_update(niti_ctx *ctx, cudaStream_t st, int8_t *w, const int8_t *g, long long n) {
+  sgd_update_kernel<<<ew_blocks(ctx, (n >> 4) + 16), 256, 0, st>>>(w, g, n);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
 }
 
 extern "C" int niti_int_sgd_update(niti_ctx *ctx, void *stream, int8_t *w, const int8_t *g, int64_t n) {

@@ -136,6 +136,58 @@ def test_conv_ops(niti, oref, B, H, W, Ci, Co, engine):
     niti.check()
 
 
+UPDATE_CONV_SHAPES = [(2, 16, 16, 64, 64), (4, 8, 8, 128, 256), (3, 20, 36, 3, 32), (2, 12, 20, 96, 160),
+                      (1, 6, 5, 16, 32)]
+
+
+@pytest.mark.parametrize("engine", [0, 1, 4])
+@pytest.mark.parametrize("B,H,W,Ci,Co", UPDATE_CONV_SHAPES)
+def test_conv_wgrad_update(niti, oref, B, H, W, Ci, Co, engine):
+    """Weight gradient fused with the update = the oracle's wgrad followed by its weight update."""
+    rng = np.random.default_rng(B + H * 3 + W * 5 + Ci * 7 + Co * 13)
+    x, e = _i8(rng, (B, H, W, Ci)), _i8(rng, (B, H, W, Co))
+    w = rng.integers(-127, 128, size=(Co, 3, 3, Ci), dtype=np.int8)       # extremes: the clamp is exercised
+    niti.set_engine(engine)
+    try:
+        for m_u in (5, 7):
+            wg, bg = oref.conv_wgrad(x, e, (3, 3), 1, m_u)
+            want = oref.sgd_update(w, wg)
+            wt = _T(niti, w.copy())
+            got, b_g = niti.conv_wgrad_update(_T(niti, x), _T(niti, e), wt, m_u=m_u)
+            assert got.data_ptr() == wt.data_ptr()
+            _eq(wt, want)
+            assert int(b_g) == bg
+    finally:
+        niti.set_engine(0)
+    niti.check()
+
+
+@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("M,N,K", [(64, 256, 784), (32, 10, 256), (128, 1000, 512), (300, 384, 640)])
+def test_linear_bwd_update(niti, oref, M, N, K, engine):
+    rng = np.random.default_rng(M + 3 * N + 7 * K)
+    a, e = _i8(rng, (M, K)), _i8(rng, (M, N))
+    w = rng.integers(-127, 128, size=(N, K), dtype=np.int8)
+    am = np.maximum(a, 0)
+    niti.set_engine(engine)
+    try:
+        we, wg, be, bg = oref.linear_bwd(am, e, w, True, am, 5)
+        want_w = oref.sgd_update(w, wg)
+        wt = _T(niti, w.copy())
+        e_prev, b_e, b_g = niti.linear_bwd_update(_T(niti, am), _T(niti, e), wt, relu_mask_src=_T(niti, am))
+        _eq(e_prev, we)                      # from the weights before the update
+        _eq(wt, want_w)
+        assert (int(b_e), int(b_g)) == (be, bg)
+        # without the error of the layer below
+        wt2 = _T(niti, w.copy())
+        none, _, b_g2 = niti.linear_bwd_update(_T(niti, am), _T(niti, e), wt2, need_e_prev=False)
+        assert none is None and int(b_g2) == bg
+        _eq(wt2, want_w)
+    finally:
+        niti.set_engine(0)
+    niti.check()
+
+
 def test_tensor_core_engine_is_the_one_that_runs(niti):
     rng = np.random.default_rng(1)
     before = niti.tc_launch_count()

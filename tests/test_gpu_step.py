@@ -18,12 +18,12 @@ def niti():
     n.close()
 
 
-def _run_both(niti, net, steps):
+def _run_both(niti, net, steps, fused_update=False):
     from oracle import OracleNetState, oracle_train_step
     from paper_2009_13108_b200 import NitiTrainer
     x, labels, weights = make_net_inputs(net)
     st = OracleNetState([w.copy() for w in weights])
-    tr = NitiTrainer(niti, net, weights)
+    tr = NitiTrainer(niti, net, weights, fused_update=fused_update)
     tr.load_batch(x, labels)
     for step in range(steps):
         rec = oracle_train_step(net, x, labels, st)
@@ -65,6 +65,13 @@ def test_nearest_rounding_and_smaller_update_width(niti):
 
 def test_config0_mlp_full_size(niti):
     _run_both(niti, config_net(0), steps=5)
+
+
+def test_steps_with_the_weight_update_fused_into_the_weight_gradient(niti):
+    """Same weights, bit-widths and hit counts as the oracle when the trainer uses the fused calls."""
+    _run_both(niti, config_net(0), steps=3, fused_update=True)
+    _run_both(niti, config_net(2, batch=32), steps=2, fused_update=True)
+    _run_both(niti, config_net(3, batch=8), steps=2, fused_update=True)
 
 
 def test_config2_mnist_cnn_reduced_batch(niti):
