@@ -94,6 +94,32 @@ class NitiTrainer:
         self.x.copy_(torch.as_tensor(x).reshape(self.x.shape), non_blocking=True)
         self.labels.copy_(torch.as_tensor(labels), non_blocking=True)
 
+    def prefetch_batch(self, x, labels):
+        """Starts the host-to-device copy of the NEXT batch (pinned host tensors) on a copy stream
+        into staging buffers, so that it overlaps the step running on the current stream;
+        ``commit_batch`` makes it the current batch."""
+        dev = self.n.device
+        if not hasattr(self, "_copy_stream"):
+            self._copy_stream = torch.cuda.Stream(device=dev)
+            self._x_stage = torch.empty_like(self.x)
+            self._labels_stage = torch.empty_like(self.labels)
+            self._staged = torch.cuda.Event()
+            self._stage_free = torch.cuda.Event()
+            self._stage_free.record(torch.cuda.current_stream(dev))
+        self._copy_stream.wait_event(self._stage_free)       # the previous commit has read the staging buffers
+        with torch.cuda.stream(self._copy_stream):
+            self._x_stage.copy_(torch.as_tensor(x).reshape(self.x.shape), non_blocking=True)
+            self._labels_stage.copy_(torch.as_tensor(labels), non_blocking=True)
+            self._staged.record(self._copy_stream)
+
+    def commit_batch(self):
+        """Makes the prefetched batch the resident one (device-to-device, on the current stream)."""
+        cur = torch.cuda.current_stream(self.n.device)
+        cur.wait_event(self._staged)
+        self.x.copy_(self._x_stage, non_blocking=True)
+        self.labels.copy_(self._labels_stage, non_blocking=True)
+        self._stage_free.record(cur)
+
     def _view(self, buf, shape):
         n = 1
         for d in shape:
