@@ -63,6 +63,31 @@ def test_nearest_rounding_and_smaller_update_width(niti):
                 assert np.array_equal(wg.cpu().numpy(), wo)
 
 
+def test_prefetched_batches_give_the_same_steps(niti):
+    """prefetch_batch / commit_batch (copy stream, staging buffers) against load_batch."""
+    import torch
+    from paper_2009_13108_b200 import NitiTrainer
+    net = config_net(2, batch=32)
+    x, labels, weights = make_net_inputs(net)
+    x2 = np.ascontiguousarray(x[::-1])
+    l2 = np.ascontiguousarray(labels[::-1])
+    a = NitiTrainer(niti, net, weights)
+    b = NitiTrainer(niti, net, weights)
+    hx, hl, hx2, hl2 = (torch.from_numpy(v).pin_memory() for v in (x, labels, x2, l2))
+    b.prefetch_batch(hx, hl)
+    for xb, lb, nx, nl in ((hx, hl, hx2, hl2), (hx2, hl2, hx, hl), (hx, hl, None, None)):
+        a.load_batch(xb, lb)
+        a.step()
+        b.commit_batch()
+        if nx is not None:
+            b.prefetch_batch(nx, nl)          # overlaps the step below
+        b.step()
+        niti.check()
+        assert int(a.n_correct) == int(b.n_correct)
+        for wa, wb in zip(a.weights, b.weights):
+            assert torch.equal(wa, wb)
+
+
 def test_config0_mlp_full_size(niti):
     _run_both(niti, config_net(0), steps=5)
 
