@@ -374,7 +374,7 @@ def run_ours(args):
     input_digests = {"x": hashlib.sha256(memoryview(x).cast("B")).hexdigest()[:16],
                      "labels": hashlib.sha256(memoryview(labels).cast("B")).hexdigest()[:16],
                      "weights": wh.hexdigest()[:16]}      # guards against drift of the seeded generator
-    tr = NitiTrainer(niti, net, weights, fused_update=args.fused_update)
+    tr = NitiTrainer(niti, net, weights, fused_update=args.fused_update, pool_codes=args.pool_codes)
     xh = torch.from_numpy(x).pin_memory()
     lh = torch.from_numpy(labels).pin_memory()
     tr.load_batch(xh, lh)
@@ -519,6 +519,8 @@ def main():
     ap.add_argument("--no-gemm", dest="gemm", action="store_false")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="issue every launch from Python instead of replaying a CUDA graph of the step")
+    ap.add_argument("--pool-codes", dest="pool_codes", action="store_true",
+                    help="max-pool forward records its routing; backward reads the codes instead of the pooled tensor")
     ap.add_argument("--fused-update", dest="fused_update", action="store_true",
                     help="weight gradient and weight update in one library call (default: two calls)")
     ap.add_argument("--gemm-shape", default=None,

@@ -259,6 +259,22 @@ int niti_maxpool2_fwd(niti_ctx *ctx, void *stream, const int8_t *x, int8_t *y, i
 int niti_maxpool2_bwd(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e_out,
                       int8_t *e_in, int B, int H, int W, int C, int relu);
 
+/* The same max-pool with the routing recorded in the forward pass, so that the
+ * backward pass does not read the pooled tensor again (it reads the error and
+ * half a byte per output element instead of four input bytes).
+ *   maxpool2_fwd_idx: y as niti_maxpool2_fwd, and idx [B][H/2][W/2][C/2]
+ *     bytes: per output element a 4-bit code, channel c in the low (c even) or
+ *     high (c odd) nibble; bits 0-1 = position of the first maximum in
+ *     (row, col) order, bit 2 = that maximum is > 0.
+ *   maxpool2_bwd_idx: e_in as niti_maxpool2_bwd(x, e_out, relu) for the x the
+ *     codes were recorded from.
+ * C must be a multiple of 16, x / y / e_out / e_in 16-byte and idx 8-byte
+ * aligned (NITI_ERR_SHAPE otherwise: use the plain calls). */
+int niti_maxpool2_fwd_idx(niti_ctx *ctx, void *stream, const int8_t *x, int8_t *y, uint8_t *idx, int B, int H,
+                          int W, int C);
+int niti_maxpool2_bwd_idx(niti_ctx *ctx, void *stream, const int8_t *e_out, const uint8_t *idx, int8_t *e_in,
+                          int B, int H, int W, int C, int relu);
+
 #ifdef __cplusplus
 }
 #endif

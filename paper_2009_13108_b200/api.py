@@ -25,7 +25,7 @@ EXPORTS = [
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
     "niti_conv_dgrad", "niti_conv_wgrad", "niti_conv_wgrad_update", "niti_linear_bwd_update", "niti_int_xent", "niti_int_xent_noalloc", "niti_int_sgd_update",
     "niti_relu_fwd",
-    "niti_relu_bwd", "niti_maxpool2_fwd", "niti_maxpool2_bwd",
+    "niti_relu_bwd", "niti_maxpool2_fwd", "niti_maxpool2_bwd", "niti_maxpool2_fwd_idx", "niti_maxpool2_bwd_idx",
 ]
 
 
@@ -81,6 +81,8 @@ def load_library():
     lib.niti_relu_bwd.argtypes = [vp, vp, vp, vp, vp, i64]
     lib.niti_maxpool2_fwd.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
     lib.niti_maxpool2_bwd.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32]
+    lib.niti_maxpool2_fwd_idx.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32]
+    lib.niti_maxpool2_bwd_idx.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32]
     return lib
 
 
@@ -320,6 +322,25 @@ class Niti:
                                                 device=self.device)
         self._ck(self.lib.niti_maxpool2_fwd(self.h, self._stream(), _ptr(x), _ptr(y), B, H, W, Cc))
         return y
+
+    def maxpool2_fwd_idx(self, x, y=None, idx=None):
+        """Max-pool that also records the routing codes (half a byte per output element)."""
+        B, H, W, Cc = x.shape
+        y = y if y is not None else torch.empty((B, H // 2, W // 2, Cc), dtype=torch.int8,
+                                                device=self.device)
+        idx = idx if idx is not None else torch.empty((B, H // 2, W // 2, Cc // 2), dtype=torch.uint8,
+                                                      device=self.device)
+        self._ck(self.lib.niti_maxpool2_fwd_idx(self.h, self._stream(), _ptr(x), _ptr(y), _ptr(idx),
+                                                B, H, W, Cc))
+        return y, idx
+
+    def maxpool2_bwd_idx(self, e_out, idx, in_shape, e_in=None, relu=False):
+        B, H, W, Cc = in_shape
+        e_in = e_in if e_in is not None else torch.empty(tuple(in_shape), dtype=torch.int8,
+                                                         device=self.device)
+        self._ck(self.lib.niti_maxpool2_bwd_idx(self.h, self._stream(), _ptr(e_out), _ptr(idx),
+                                                _ptr(e_in), B, H, W, Cc, int(relu)))
+        return e_in
 
     def maxpool2_bwd(self, x, e_out, e_in=None, relu=False):
         B, H, W, Cc = x.shape

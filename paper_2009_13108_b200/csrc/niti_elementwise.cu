@@ -814,6 +814,103 @@ maxpool2_bwd_kernel(const int8_t *__restrict__ x, const int8_t *__restrict__ eo,
   }
 }
 
+// ---- max-pool that records where the maximum was --------------------------------------------
+// The backward pass of a 2x2 max-pool needs, per output element, the position of the first maximum
+// of its window and (behind a ReLU) whether that maximum was positive: four bits.  Recording them in
+// the forward pass (half a byte per output element) lets the backward pass read the error and the
+// codes instead of the whole input tensor: 1.25 + 0.5/4 bytes per input element instead of 2.25.
+// Code of one element: bits 0-1 = position (0: (0,0), 1: (0,1), 2: (1,0), 3: (1,1)), bit 2 = max > 0.
+// Layout: [B][H/2][W/2][C/2] bytes, channel c in the low (c even) or high (c odd) nibble.
+__device__ __forceinline__ unsigned pool_codes_word(unsigned x0, unsigned x1, unsigned x2, unsigned x3, unsigned &m) {
+  m = __vmaxs4(__vmaxs4(x0, x1), __vmaxs4(x2, x3));
+  const unsigned s0 = __vcmpeq4(x0, m);
+  const unsigned s1 = __vcmpeq4(x1, m) & ~s0;
+  const unsigned s2 = __vcmpeq4(x2, m) & ~(s0 | s1);
+  const unsigned s3 = ~(s0 | s1 | s2);
+  const unsigned pos = __vcmpgts4(m, 0);
+  return (s1 & 0x01010101u) | (s2 & 0x02020202u) | (s3 & 0x03030303u) | (pos & 0x04040404u);
+}
+// four byte codes (one per byte) -> 16 bits of nibbles, and back
+__device__ __forceinline__ unsigned pool_pack_nibbles(unsigned w) {
+  const unsigned t = (w | (w >> 4)) & 0x00ff00ffu;
+  return (t | (t >> 8)) & 0xffffu;
+}
+__device__ __forceinline__ unsigned pool_unpack_nibbles(unsigned p16) {
+  const unsigned t = (p16 | (p16 << 8)) & 0x00ff00ffu;
+  return (t | (t << 4)) & 0x0f0f0f0fu;
+}
+
+__global__ void __launch_bounds__(256)
+maxpool2_fwd_idx_kernel(const int8_t *__restrict__ x, int8_t *__restrict__ y, uint8_t *__restrict__ idx, int B, int H,
+                        int W, int C) {
+  const int Ho = H >> 1, Wo = W >> 1, Cv = C / 16;
+  const long long total = (long long)B * Ho * Wo * Cv;
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (long long)gridDim.x * blockDim.x) {
+    const int cv = (int)(t % Cv);
+    const long long pix = t / Cv;
+    const int j = (int)(pix % Wo);
+    const long long bi = pix / Wo;
+    const int i = (int)(bi % Ho);
+    const long long b = bi / Ho;
+    const long long base = (((b * H + 2 * i) * W + 2 * j) * (long long)C) + (long long)cv * 16;
+    const long long rs = (long long)W * C;
+    const int4 v0 = *reinterpret_cast<const int4 *>(x + base);
+    const int4 v1 = *reinterpret_cast<const int4 *>(x + base + C);
+    const int4 v2 = *reinterpret_cast<const int4 *>(x + base + rs);
+    const int4 v3 = *reinterpret_cast<const int4 *>(x + base + rs + C);
+    int4 m;
+    const unsigned c0 = pool_codes_word(v0.x, v1.x, v2.x, v3.x, (unsigned &)m.x);
+    const unsigned c1 = pool_codes_word(v0.y, v1.y, v2.y, v3.y, (unsigned &)m.y);
+    const unsigned c2 = pool_codes_word(v0.z, v1.z, v2.z, v3.z, (unsigned &)m.z);
+    const unsigned c3 = pool_codes_word(v0.w, v1.w, v2.w, v3.w, (unsigned &)m.w);
+    *reinterpret_cast<int4 *>(y + pix * C + (long long)cv * 16) = m;
+    uint2 packed;
+    packed.x = pool_pack_nibbles(c0) | (pool_pack_nibbles(c1) << 16);
+    packed.y = pool_pack_nibbles(c2) | (pool_pack_nibbles(c3) << 16);
+    *reinterpret_cast<uint2 *>(idx + (pix * C >> 1) + (long long)cv * 8) = packed;
+  }
+}
+
+__device__ __forceinline__ void pool_route_word(unsigned codes, unsigned e, int relu, unsigned &o0, unsigned &o1,
+                                                unsigned &o2, unsigned &o3) {
+  const unsigned pos2 = codes & 0x03030303u;
+  if (relu) e &= __vcmpne4(codes & 0x04040404u, 0u);
+  o0 = e & __vcmpeq4(pos2, 0u);
+  o1 = e & __vcmpeq4(pos2, 0x01010101u);
+  o2 = e & __vcmpeq4(pos2, 0x02020202u);
+  o3 = e & __vcmpeq4(pos2, 0x03030303u);
+}
+
+__global__ void __launch_bounds__(256)
+maxpool2_bwd_idx_kernel(const int8_t *__restrict__ eo, const uint8_t *__restrict__ idx, int8_t *__restrict__ ei, int B,
+                        int H, int W, int C, int relu) {
+  const int Ho = H >> 1, Wo = W >> 1, Cv = C / 16;
+  const long long total = (long long)B * Ho * Wo * Cv;
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (long long)gridDim.x * blockDim.x) {
+    const int cv = (int)(t % Cv);
+    const long long pix = t / Cv;
+    const int j = (int)(pix % Wo);
+    const long long bi = pix / Wo;
+    const int i = (int)(bi % Ho);
+    const long long b = bi / Ho;
+    const long long base = (((b * H + 2 * i) * W + 2 * j) * (long long)C) + (long long)cv * 16;
+    const long long rs = (long long)W * C;
+    const int4 e = __ldcs(reinterpret_cast<const int4 *>(eo + pix * C + (long long)cv * 16));
+    const uint2 packed = __ldcs(reinterpret_cast<const uint2 *>(idx + (pix * C >> 1) + (long long)cv * 8));
+    int4 o0, o1, o2, o3;
+    pool_route_word(pool_unpack_nibbles(packed.x & 0xffffu), e.x, relu, (unsigned &)o0.x, (unsigned &)o1.x, (unsigned &)o2.x, (unsigned &)o3.x);
+    pool_route_word(pool_unpack_nibbles(packed.x >> 16), e.y, relu, (unsigned &)o0.y, (unsigned &)o1.y, (unsigned &)o2.y, (unsigned &)o3.y);
+    pool_route_word(pool_unpack_nibbles(packed.y & 0xffffu), e.z, relu, (unsigned &)o0.z, (unsigned &)o1.z, (unsigned &)o2.z, (unsigned &)o3.z);
+    pool_route_word(pool_unpack_nibbles(packed.y >> 16), e.w, relu, (unsigned &)o0.w, (unsigned &)o1.w, (unsigned &)o2.w, (unsigned &)o3.w);
+    *reinterpret_cast<int4 *>(ei + base) = o0;
+    *reinterpret_cast<int4 *>(ei + base + C) = o1;
+    *reinterpret_cast<int4 *>(ei + base + rs) = o2;
+    *reinterpret_cast<int4 *>(ei + base + rs + C) = o3;
+  }
+}
+
 static inline unsigned ew_blocks(niti_ctx *ctx, long long work_items) {
   long long blocks = (work_items + 255) / 256;
   long long cap = (long long)ctx->sm_count * 16;
@@ -872,6 +969,34 @@ extern "C" int niti_maxpool2_fwd(niti_ctx *ctx, void *stream, const int8_t *x, i
     maxpool2_fwd_kernel<16><<<ew_blocks(ctx, items), 256, 0, (cudaStream_t)stream>>>(x, y, B, H, W, C);
   else
     maxpool2_fwd_kernel<1><<<ew_blocks(ctx, items), 256, 0, (cudaStream_t)stream>>>(x, y, B, H, W, C);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+extern "C" int niti_maxpool2_fwd_idx(niti_ctx *ctx, void *stream, const int8_t *x, int8_t *y, uint8_t *idx, int B,
+                                     int H, int W, int C) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!x || !y || !idx || B <= 0 || H <= 0 || W <= 0 || C <= 0 || (H & 1) || (W & 1))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_maxpool2_fwd_idx: bad argument (H and W must be even)");
+  if ((C % 16) != 0 || (((uintptr_t)x | (uintptr_t)y) & 15) || ((uintptr_t)idx & 7))
+    return niti_fail(ctx, NITI_ERR_SHAPE, "niti_maxpool2_fwd_idx: C must be a multiple of 16 and the tensors aligned");
+  const long long items = (long long)B * (H / 2) * (W / 2) * (C / 16);
+  maxpool2_fwd_idx_kernel<<<ew_blocks(ctx, items), 256, 0, (cudaStream_t)stream>>>(x, y, idx, B, H, W, C);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
+extern "C" int niti_maxpool2_bwd_idx(niti_ctx *ctx, void *stream, const int8_t *e_out, const uint8_t *idx,
+                                     int8_t *e_in, int B, int H, int W, int C, int relu) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!e_out || !idx || !e_in || B <= 0 || H <= 0 || W <= 0 || C <= 0 || (H & 1) || (W & 1))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_maxpool2_bwd_idx: bad argument (H and W must be even)");
+  if ((C % 16) != 0 || (((uintptr_t)e_out | (uintptr_t)e_in) & 15) || ((uintptr_t)idx & 7))
+    return niti_fail(ctx, NITI_ERR_SHAPE, "niti_maxpool2_bwd_idx: C must be a multiple of 16 and the tensors aligned");
+  const long long items = (long long)B * (H / 2) * (W / 2) * (C / 16);
+  maxpool2_bwd_idx_kernel<<<ew_blocks(ctx, items), 256, 0, (cudaStream_t)stream>>>(e_out, idx, e_in, B, H, W, C, relu);
   ctx->launches++;
   NITI_CUDA_TRY(ctx, cudaGetLastError());
   return NITI_OK;

@@ -402,6 +402,23 @@ def test_maxpool(niti, oref, B, H, W, C):
     _eq(niti.maxpool2_bwd(_T(niti, xs), _T(niti, e)), oref.maxpool2_bwd(xs, e))
 
 
+@pytest.mark.parametrize("B,H,W,C", [(2, 8, 8, 16), (3, 6, 10, 64), (1, 28, 28, 32), (2, 4, 4, 512)])
+def test_maxpool_with_recorded_routing(niti, oref, B, H, W, C):
+    """Forward records position and positivity of each window's first maximum; backward uses only
+    the codes and the error.  Few distinct values: many ties; negative maxima: the ReLU gate."""
+    rng = np.random.default_rng(B + H + W + C)
+    for lo, hi in ((-3, 4), (-127, 128), (-5, 1)):
+        x = rng.integers(lo, hi, size=(B, H, W, C), dtype=np.int8)
+        e = _i8(rng, (B, H // 2, W // 2, C))
+        y, idx = niti.maxpool2_fwd_idx(_T(niti, x))
+        _eq(y, oref.maxpool2_fwd(x))
+        assert tuple(idx.shape) == (B, H // 2, W // 2, C // 2)
+        routed = oref.maxpool2_bwd(x, e)
+        _eq(niti.maxpool2_bwd_idx(_T(niti, e), idx, x.shape, relu=False), routed)
+        _eq(niti.maxpool2_bwd_idx(_T(niti, e), idx, x.shape, relu=True), oref.relu_bwd(x, routed))
+    niti.check()
+
+
 def test_argument_errors(niti):
     from paper_2009_13108_b200 import NitiError
     a = torch.zeros((4, 32), dtype=torch.int8, device=niti.device)

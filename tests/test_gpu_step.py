@@ -18,12 +18,12 @@ def niti():
     n.close()
 
 
-def _run_both(niti, net, steps, fused_update=False):
+def _run_both(niti, net, steps, fused_update=False, pool_codes=False):
     from oracle import OracleNetState, oracle_train_step
     from paper_2009_13108_b200 import NitiTrainer
     x, labels, weights = make_net_inputs(net)
     st = OracleNetState([w.copy() for w in weights])
-    tr = NitiTrainer(niti, net, weights, fused_update=fused_update)
+    tr = NitiTrainer(niti, net, weights, fused_update=fused_update, pool_codes=pool_codes)
     tr.load_batch(x, labels)
     for step in range(steps):
         rec = oracle_train_step(net, x, labels, st)
@@ -97,6 +97,11 @@ def test_steps_with_the_weight_update_fused_into_the_weight_gradient(niti):
     _run_both(niti, config_net(0), steps=3, fused_update=True)
     _run_both(niti, config_net(2, batch=32), steps=2, fused_update=True)
     _run_both(niti, config_net(3, batch=8), steps=2, fused_update=True)
+
+
+def test_steps_with_recorded_pool_routing(niti):
+    _run_both(niti, config_net(2, batch=32), steps=2, pool_codes=True)
+    _run_both(niti, config_net(3, batch=8), steps=2, pool_codes=True)
 
 
 def test_config2_mnist_cnn_reduced_batch(niti):
