@@ -188,6 +188,40 @@ def test_linear_bwd_update(niti, oref, M, N, K, engine):
     niti.check()
 
 
+def test_outputs_and_masks_aligned_to_16_but_not_32_bytes(niti, oref):
+    """The epilogue's whole-chunk loop needs 32-byte aligned rows; 16-byte aligned tensors take the
+    general loop (16-byte stores) and must give the same bytes."""
+    import torch
+    rng = np.random.default_rng(77)
+    B, H, W, Ci, Co = 2, 16, 24, 64, 64
+    x, w, e = _i8(rng, (B, H, W, Ci)), _i8(rng, (Co, 3, 3, Ci)), _i8(rng, (B, H, W, Co))
+    xm = np.maximum(x, 0)
+
+    def off16(shape):
+        n = int(np.prod(shape))
+        buf = torch.empty(n + 64, dtype=torch.int8, device=niti.device)
+        skew = (16 - buf.data_ptr() % 32) % 32          # 16 mod 32
+        return buf[skew:skew + n].view(shape)
+
+    wy, s, b = oref.conv_fwd(x, -7, w, -9, 1, True)
+    y = off16((B, H, W, Co))
+    assert y.data_ptr() % 32 == 16
+    niti.conv_fwd(_T(niti, x), niti.scalar(-7), _T(niti, w), niti.scalar(-9), y=y, relu=True)
+    _eq(y, wy)
+    wd, bd = oref.conv_dgrad(e, w, (H, W), 1, xm)
+    mask = off16((B, H, W, Ci))
+    mask.copy_(_T(niti, xm))
+    ep, b_e = niti.conv_dgrad(_T(niti, e), _T(niti, w), (H, W), relu_mask_src=mask)
+    _eq(ep, wd)
+    assert int(b_e) == bd
+    a, wl = _i8(rng, (300, 256)), _i8(rng, (192, 256))
+    want, s2, b2 = oref.linear_fwd(a, -7, wl, -9, True)
+    out = off16((300, 192))
+    niti.linear_fwd(_T(niti, a), niti.scalar(-7), _T(niti, wl), niti.scalar(-9), out=out, relu=True)
+    _eq(out, want)
+    niti.check()
+
+
 def test_tensor_core_engine_is_the_one_that_runs(niti):
     rng = np.random.default_rng(1)
     before = niti.tc_launch_count()
