@@ -202,6 +202,28 @@ int niti_linear_bwd_update(niti_ctx *ctx, void *stream, const int8_t *a, const i
                            int8_t *e_prev, const int8_t *relu_mask_src, int32_t *b_e, int32_t *b_g,
                            int M, int N, int K, int m_u, int round_mode, void *ws, size_t ws_bytes);
 
+/* Exact data-parallel training over several GPUs (one process per GPU, each with its share of
+ * the batch): the method shards over the batch, and the only quantities that couple the samples
+ * are (a) the max magnitude that fixes the bit-width b of a tensor, and (b) the int32 sums of the
+ * weight gradient, which contract over the batch (Algorithm 1).  With a hook installed the
+ * library calls it, in stream order, wherever one of them must be combined over the ranks before
+ * the rounding uses it:
+ *   NITI_REDUCE_MAX_U32: dev_ptr -> count (= 1) unsigned 32-bit values, combine with max;
+ *   NITI_REDUCE_MAX_U64: the same, 64-bit (integer cross-entropy);
+ *   NITI_REDUCE_SUM_I32: dev_ptr -> count int32 sums (a whole weight-gradient tensor), add.
+ * dev_ptr points into the workspace of the running call.  The hook must order its work after what
+ * is already on `stream` and before what follows (e.g. an NCCL all-reduce on that stream) and
+ * return 0.  Every rank must make the same sequence of library calls.  With the combined values
+ * every rank rounds exactly as one process holding the whole batch would, so activations, errors
+ * and updated weights equal the single-process result bit for bit.  Multiplies that would round
+ * in their own epilogue from partial sums (weight gradients) take the int32 path instead.
+ * fn == NULL removes the hook.  niti_int_xent_noalloc has no context and calls no hook. */
+#define NITI_REDUCE_MAX_U32 0
+#define NITI_REDUCE_MAX_U64 1
+#define NITI_REDUCE_SUM_I32 2
+typedef int (*niti_reduce_fn)(void *user, void *stream, void *dev_ptr, int64_t count, int kind);
+int niti_set_reduce_hook(niti_ctx *ctx, niti_reduce_fn fn, void *user);
+
 /* Integer cross-entropy gradient (Section 3.5, Eq. 1-4).  Per sample r:
  *   e32[r][i] = T_i - [i == labels[r]] * sum_j T_j
  * with T_i = 2^(1-2s) + a_i 2^(1-s) + a_i^2 when s = *s_a <= -7 (Eq. 2), else

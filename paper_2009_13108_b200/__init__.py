@@ -6,5 +6,5 @@ training step (Algorithm 1 of the paper) together for a feed-forward net.  There
 fallback: importing works without a GPU, but constructing ``Niti`` requires the built library
 and a CUDA device.
 """
-from .api import Niti, NitiError, library_path  # noqa: F401
+from .api import Niti, NitiError, dist_reducer, library_path  # noqa: F401
 from .trainer import NitiTrainer  # noqa: F401

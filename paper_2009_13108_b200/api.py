@@ -17,10 +17,12 @@ OK, ERR_ARG, ERR_SHAPE, ERR_WORKSPACE, ERR_RANGE, ERR_CUDA, ERR_DEVICE = range(7
 ROUND_PSR, ROUND_NEAREST = 0, 1
 OP_LINEAR_FWD, OP_LINEAR_BWD, OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_INT_XENT = range(6)
 OP_LINEAR_BWD_UPDATE, OP_CONV_WGRAD_UPDATE = 6, 7
+REDUCE_MAX_U32, REDUCE_MAX_U64, REDUCE_SUM_I32 = 0, 1, 2
+_REDUCE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int)
 
 EXPORTS = [
     "niti_create", "niti_destroy", "niti_last_error", "niti_check", "niti_workspace_bytes",
-    "niti_set_engine", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
+    "niti_set_engine", "niti_set_reduce_hook", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
     "niti_redo_count", "niti_selftest_timeout", "niti_profile_enable", "niti_profile_read_launches",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
     "niti_conv_dgrad", "niti_conv_wgrad", "niti_conv_wgrad_update", "niti_linear_bwd_update", "niti_int_xent", "niti_int_xent_noalloc", "niti_int_sgd_update",
@@ -53,6 +55,7 @@ def load_library():
     lib.niti_workspace_bytes.argtypes = [i32, C.POINTER(i64), i32]
     lib.niti_workspace_bytes.restype = sz
     lib.niti_set_engine.argtypes = [vp, i32]
+    lib.niti_set_reduce_hook.argtypes = [vp, _REDUCE_FN, vp]
     lib.niti_launch_count.argtypes = [vp]
     lib.niti_launch_count.restype = C.c_uint64
     lib.niti_tc_launch_count.argtypes = [vp]
@@ -127,6 +130,32 @@ class Niti:
     def workspace_bytes(self, op, dims) -> int:
         arr = (C.c_int64 * len(dims))(*dims)
         return int(self.lib.niti_workspace_bytes(op, arr, len(dims)))
+
+    def set_reduce_hook(self, fn):
+        """Exact data parallelism: ``fn(view, kind)`` combines the device tensor ``view`` (a slice of
+        the workspace: int32 for REDUCE_MAX_U32 / REDUCE_SUM_I32, int64 for REDUCE_MAX_U64; the values
+        to maximise are non-negative) in place over the ranks, ordered on the current stream.
+        ``None`` removes the hook.  See ``dist_reducer`` for torch.distributed."""
+        if fn is None:
+            self._ck(self.lib.niti_set_reduce_hook(self.h, None, None))
+            self._reduce_cb = None
+            return
+
+        def cb(user, stream, ptr, count, kind):
+            try:
+                dtype, size = {REDUCE_MAX_U32: (torch.int32, 4), REDUCE_MAX_U64: (torch.int64, 8),
+                               REDUCE_SUM_I32: (torch.int32, 4)}[kind]
+                off = ptr - self._ws.data_ptr()
+                if off < 0 or off + count * size > self._ws.numel():
+                    return 2
+                fn(self._ws[off:off + count * size].view(dtype), kind)
+                return 0
+            except Exception as exc:          # an exception must not cross the C boundary
+                self._reduce_error = exc
+                return 1
+
+        self._reduce_cb = _REDUCE_FN(cb)      # keep the callback object alive
+        self._ck(self.lib.niti_set_reduce_hook(self.h, self._reduce_cb, None))
 
     def reserve_workspace(self, nbytes: int):
         if self._ws.numel() < nbytes:
@@ -348,3 +377,15 @@ class Niti:
         self._ck(self.lib.niti_maxpool2_bwd(self.h, self._stream(), _ptr(x), _ptr(e_out),
                                             _ptr(e_in), B, H, W, Cc, int(relu)))
         return e_in
+
+
+def dist_reducer(group=None):
+    """A reduction hook for ``Niti.set_reduce_hook`` over a torch.distributed process group (NCCL: the
+    all-reduce is ordered on the current stream; gloo: through the host)."""
+    import torch.distributed as dist
+
+    def reduce(view, kind):
+        op = dist.ReduceOp.SUM if kind == REDUCE_SUM_I32 else dist.ReduceOp.MAX
+        dist.all_reduce(view, op=op, group=group)
+
+    return reduce

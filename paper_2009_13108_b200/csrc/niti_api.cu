@@ -69,6 +69,13 @@ extern "C" int niti_set_engine(niti_ctx *ctx, int engine) {
   return old;
 }
 
+extern "C" int niti_set_reduce_hook(niti_ctx *ctx, niti_reduce_fn fn, void *user) {
+  if (!ctx) return NITI_ERR_ARG;
+  ctx->reduce_fn = fn;
+  ctx->reduce_user = fn ? user : nullptr;
+  return NITI_OK;
+}
+
 extern "C" uint64_t niti_launch_count(niti_ctx *ctx) { return ctx ? ctx->launches : 0; }
 extern "C" uint64_t niti_tc_launch_count(niti_ctx *ctx) { return ctx ? ctx->tc_launches : 0; }
 extern "C" uint64_t niti_tc_pair_launch_count(niti_ctx *ctx) { return ctx ? ctx->tc2_launches : 0; }
@@ -228,6 +235,19 @@ static inline bool misaligned16(const void *p) { return ((uintptr_t)p & 15) != 0
 
 int niti_launch_sgd_update(niti_ctx *ctx, cudaStream_t st, int8_t *w, const int8_t *g, long long n);
 
+// Data parallelism (niti_set_reduce_hook), after a multiply has left its int32 accumulators in acc and
+// their max magnitude in the header: a weight gradient is summed over the ranks and its max taken
+// again from the sums; any other tensor only shares the max.
+int niti_reduce_after_gemm(niti_ctx *ctx, cudaStream_t st, int kind, int32_t *acc, long long n, WsHeader *hdr) {
+  if (!ctx->reduce_fn) return NITI_OK;
+  if (!niti_is_wgrad(kind)) return niti_reduce(ctx, st, &hdr->maxabs32, 1, NITI_REDUCE_MAX_U32);
+  int rc = niti_reduce(ctx, st, acc, n, NITI_REDUCE_SUM_I32);
+  if (rc != NITI_OK) return rc;
+  NITI_CUDA_TRY(ctx, cudaMemsetAsync(&hdr->maxabs32, 0, sizeof(unsigned int), st));
+  ctx->launches++;
+  return niti_launch_maxabs(ctx, st, acc, n, hdr);
+}
+
 // One matrix multiply of Algorithm 1 followed by EffectiveBitwidth + ShiftAndRound.
 // update_w != null (weight gradients): the rounded gradient is not returned but subtracted from the
 // weights in place.  When the int32 accumulators exist (split contractions) the rounding pass does
@@ -247,7 +267,10 @@ static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, 
   bool fused = false;
   RoundSpec rs = {out, mask, mbits, round_mode, relu, s_a, s_w, s_out, b_out};
   if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, rs, acc, hdr, &fused);
-  if (rc == NITI_ERR_SHAPE) rc = niti_simt_gemm(ctx, st, p, acc, hdr);
+  if (rc == NITI_ERR_SHAPE) {
+    rc = niti_simt_gemm(ctx, st, p, acc, hdr);
+    if (rc == NITI_OK) rc = niti_reduce_after_gemm(ctx, st, p.kind, acc, p.gm * p.gn, hdr);
+  }
   if (rc != NITI_OK) return rc;
   if (fused) return update_w ? niti_launch_sgd_update(ctx, st, update_w, out, p.gm * p.gn) : NITI_OK;
   return niti_launch_round(ctx, st, acc, hdr, out, p.gm * p.gn, mbits, round_mode, relu, mask, s_a, s_w,
@@ -441,7 +464,10 @@ static int conv_wgrad_impl(niti_ctx *ctx, void *stream, const int8_t *x, const i
     if (saved == 0) ctx->engine = 4;               // int32 accumulators are needed here, not a fused store
     rc = niti_tc_gemm(ctx, st, q, none, acc32, hdr, &fused);
     ctx->engine = saved;
-    if (rc == NITI_ERR_SHAPE) rc = niti_simt_gemm(ctx, st, q, acc32, hdr);
+    if (rc == NITI_ERR_SHAPE) {
+      rc = niti_simt_gemm(ctx, st, q, acc32, hdr);
+      if (rc == NITI_OK) rc = niti_reduce_after_gemm(ctx, st, q.kind, acc32, (long long)Cout * 32, hdr);
+    }
     if (rc != NITI_OK) return rc;
     rc = niti_launch_round_compact32(ctx, st, acc32, hdr, g, Cout, R * S * Cin, m_u, round_mode, b_g);
     if (rc != NITI_OK || !update_w) return rc;

@@ -24,7 +24,13 @@ struct niti_ctx {
   double *prof_ops;         // algorithmic int8 operations (2*M*N*K) of each recorded launch
   // cuTensorMapEncodeTiled, fetched through the runtime so that libcuda is not a link dependency
   void *encode_tiled;
+  // data-parallel training (niti_set_reduce_hook): called where a tensor-wide quantity has to be
+  // combined over the ranks before the rounding may use it
+  niti_reduce_fn reduce_fn;
+  void *reduce_user;
 };
+
+
 
 #define NITI_PROF_MAX 8192
 #define NITI_WS_HEADER 256  // bytes reserved at the start of every workspace for reduction scalars
@@ -56,6 +62,17 @@ static inline int niti_fail(niti_ctx *ctx, int code, const char *msg) {
   if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s", msg);
   return code;
 }
+
+// Runs the caller's reduction over the ranks on a device buffer, ordered on the stream.
+static inline int niti_reduce(niti_ctx *ctx, cudaStream_t st, void *dev_ptr, long long count, int kind) {
+  if (!ctx->reduce_fn) return NITI_OK;
+  if (ctx->reduce_fn(ctx->reduce_user, (void *)st, dev_ptr, (int64_t)count, kind) != 0)
+    return niti_fail(ctx, NITI_ERR_ARG, "the reduction hook reported a failure");
+  return NITI_OK;
+}
+// (weight gradients contract over the batch: under data parallelism their int32 sums are added
+// over the ranks; every other multiply only shares its max magnitude)
+static inline bool niti_is_wgrad(int kind) { return kind == 2 || kind == 5; }   // GK_FC_WGRAD, GK_CONV_WGRAD
 
 // ---- rounding arithmetic (Algorithm 3 and round-to-nearest), on the magnitude ----------------
 template <typename U>
@@ -92,6 +109,7 @@ enum NitiGemmKind {
   GK_CONV_DGRAD,   // A(pix, (r,s,co)) = e shifted, B(ci, (r,s,co)) = w[co][r][s][ci]
   GK_CONV_WGRAD    // A(co, pix) = e[pix][co],      B((r,s,ci), pix) = x shifted
 };
+static_assert(GK_FC_WGRAD == 2 && GK_CONV_WGRAD == 5, "niti_is_wgrad");
 
 struct GemmProblem {
   int kind;
@@ -106,6 +124,8 @@ struct GemmProblem {
   long long ld0;
 };
 
+int niti_reduce_after_gemm(niti_ctx *ctx, cudaStream_t st, int kind, int32_t *acc, long long n, WsHeader *hdr);
+int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr);
 // Plain CUDA-core engine: writes int32 accumulators to acc[gm][gn] and max|acc| to hdr->maxabs32.
 int niti_simt_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t *acc, WsHeader *hdr);
 // What follows the multiply: rounding target and the scalars of Algorithm 2.

@@ -583,18 +583,22 @@ xent_round_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__
 }
 
 // both passes; the packed path needs whole words per row
-static void launch_xent(cudaStream_t st, const int8_t *a, const int32_t *s_a, const int32_t *labels,
-                        long long *rowinfo, WsHeader *hdr, int8_t *e, int32_t *b_e, int32_t *n_correct, int B, int N,
-                        int round_mode, uint32_t *status) {
+// (ctx may be null: the variant without a context; with one, the max magnitude of the 64-bit
+// gradients is combined over the ranks between the two passes when a reduction hook is installed)
+static int launch_xent(niti_ctx *ctx, cudaStream_t st, const int8_t *a, const int32_t *s_a, const int32_t *labels,
+                       long long *rowinfo, WsHeader *hdr, int8_t *e, int32_t *b_e, int32_t *n_correct, int B, int N,
+                       int round_mode, uint32_t *status) {
   const unsigned blocks = (unsigned)((B + XENT_WARPS - 1) / XENT_WARPS);
   const bool packed = (N & 3) == 0 && N >= 64 && (((uintptr_t)a | (uintptr_t)e) & 3) == 0;
-  if (packed) {
-    xent_row_fast_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
-    xent_round_fast_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
-  } else {
-    xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
-    xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
+  if (packed) xent_row_fast_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
+  else xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
+  if (ctx) {
+    int rc = niti_reduce(ctx, st, &hdr->maxabs64, 1, NITI_REDUCE_MAX_U64);
+    if (rc != NITI_OK) return rc;
   }
+  if (packed) xent_round_fast_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
+  else xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
+  return NITI_OK;
 }
 
 extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const int32_t *s_a,
@@ -615,7 +619,8 @@ extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st));
     ctx->launches++;
   }
-  launch_xent(st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, ctx->d_status);
+  int rcx = launch_xent(ctx, st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, ctx->d_status);
+  if (rcx != NITI_OK) return rcx;
   ctx->launches += 2;
   NITI_CUDA_TRY(ctx, cudaGetLastError());
   return NITI_OK;
@@ -659,7 +664,7 @@ extern "C" int niti_int_xent_noalloc(void *stream, const int8_t *a, const int32_
   uint32_t *status = (uint32_t *)((char *)base + NITI_WS_HEADER - sizeof(uint32_t));
   if (cudaMemsetAsync(base, 0, NITI_WS_HEADER, st) != cudaSuccess) return NITI_ERR_CUDA;
   if (n_correct && cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st) != cudaSuccess) return NITI_ERR_CUDA;
-  launch_xent(st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, status);
+  launch_xent(nullptr, st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, status);
   if (cudaGetLastError() != cudaSuccess) return NITI_ERR_CUDA;
   return NITI_OK;
 }

@@ -2170,7 +2170,10 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
     double f = (n_s > 16.0 && frac < 1.0) ? sqrt(log(n_all) / log(n_s)) : 1.0;
     p.spec_mul256 = (unsigned)(f * 256.0 + 0.5);
   }
-  p.single_wave = (p.items <= (p.ctas == 2 ? tc_units<2>(ctx) : tc_units<1>(ctx)) && p.spec_mul256 == 256) ? 1 : 0;
+  // data parallelism (niti_set_reduce_hook): the max magnitude is combined over the ranks between the
+  // two launches, so there is always a second launch; weight gradients keep their int32 sums
+  const bool dp = ctx->reduce_fn != nullptr, dp_sum = dp && niti_is_wgrad(g.kind);
+  p.single_wave = (!dp && p.items <= (p.ctas == 2 ? tc_units<2>(ctx) : tc_units<1>(ctx)) && p.spec_mul256 == 256) ? 1 : 0;
   {
     const long long units = p.ctas == 2 ? tc_units<2>(ctx) : tc_units<1>(ctx);
     const long long grid = (p.items < units ? p.items : units) * p.ctas;
@@ -2179,7 +2182,7 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
   p.mbits = r.mbits;
   p.round_mode = r.round_mode;
   p.relu = r.relu;
-  p.epi_mode = (p.splits > 1 || p.halo == 2) ? EPI_ATOMIC : (ctx->engine == 4 ? EPI_SPILL : EPI_SPECULATE);
+  p.epi_mode = (p.splits > 1 || p.halo == 2) ? EPI_ATOMIC : ((ctx->engine == 4 || dp_sum) ? EPI_SPILL : EPI_SPECULATE);
   if (p.epi_mode == EPI_ATOMIC) {
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(acc, 0, sizeof(int32_t) * (size_t)(g.gm * g.gn), st));
     ctx->launches++;
@@ -2192,6 +2195,10 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
     *fused = true;                     // exact shift, scalars published by the last CTA: no second launch
   } else if (p.epi_mode == EPI_SPECULATE) {
     // publishes b and the exponent; recomputes with the true bit-width only if the guess was low
+    if (dp) {
+      rc = niti_reduce(ctx, st, &hdr->maxabs32, 1, NITI_REDUCE_MAX_U32);
+      if (rc != NITI_OK) return rc;
+    }
     p.epi_mode = EPI_KNOWN_B;
     rc = p.ctas == 2 ? launch_tc<2>(ctx, st, p, ma, mb, acc, hdr, r) : launch_tc<1>(ctx, st, p, ma, mb, acc, hdr, r);
     if (rc != NITI_OK) return rc;
@@ -2202,6 +2209,15 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
     ctx->prof_ops[ctx->prof_used] = 2.0 * (double)g.gm * (double)g.gn * (double)g.gk;
     ctx->prof_used++;
   }
-  if (p.epi_mode == EPI_ATOMIC) return niti_launch_maxabs(ctx, st, acc, g.gm * g.gn, hdr);
+  if (p.epi_mode == EPI_ATOMIC) {
+    if (dp_sum) {                      // sums over the ranks first, then their max
+      rc = niti_reduce(ctx, st, acc, g.gm * g.gn, NITI_REDUCE_SUM_I32);
+      if (rc != NITI_OK) return rc;
+    }
+    rc = niti_launch_maxabs(ctx, st, acc, g.gm * g.gn, hdr);
+    if (rc != NITI_OK || !dp || dp_sum) return rc;
+    return niti_reduce(ctx, st, &hdr->maxabs32, 1, NITI_REDUCE_MAX_U32);
+  }
+  if (p.epi_mode == EPI_SPILL && dp) return niti_reduce_after_gemm(ctx, st, g.kind, acc, g.gm * g.gn, hdr);
   return NITI_OK;
 }

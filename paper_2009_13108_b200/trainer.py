@@ -13,7 +13,7 @@ from .api import Niti, ROUND_PSR
 
 class NitiTrainer:
     def __init__(self, niti: Niti, net, weights, round_mode: int = ROUND_PSR, fused_update: bool = False,
-                 pool_codes: bool = False):
+                 pool_codes: bool = False, dist_group=None, data_parallel: bool = False):
         """``net``: an object with ``batch``, ``in_shape``, ``s_in``, ``m_u`` and ``layers`` (dicts
         with op in {"conv", "pool", "fc"}); ``weights``: int8 host arrays / tensors per weight
         layer ([Cout,3,3,Cin] or [N,K]).  ``fused_update``: weight gradient and weight update in one
@@ -29,6 +29,14 @@ class NitiTrainer:
         self.net = net
         self.round_mode = round_mode
         self.fused_update = fused_update
+        # exact data parallelism: ``net.batch`` is this rank's share of the batch; bit-widths and
+        # weight-gradient sums are combined over the ranks of ``dist_group`` (None = the default group),
+        # so every rank holds the weights one process with the whole batch would have
+        self.data_parallel = data_parallel
+        if data_parallel:
+            from .api import dist_reducer
+            niti.set_reduce_hook(dist_reducer(dist_group))
+            self._dist_group = dist_group
         dev = niti.device
         i8 = dict(dtype=torch.int8, device=dev)
         self.weights = [torch.as_tensor(w).to(dev).contiguous() for w in weights]
@@ -71,6 +79,14 @@ class NitiTrainer:
         self.b_loss = niti.scalar()
         self.n_correct = niti.scalar()
         self.first_weight_layer = next(i for i, L in enumerate(net.layers) if L["op"] != "pool")
+
+    def global_hits(self):
+        """Hit count of the last step over all ranks (data parallel), as a device tensor."""
+        hits = self.n_correct.clone()
+        if self.data_parallel:
+            import torch.distributed as dist
+            dist.all_reduce(hits, op=dist.ReduceOp.SUM, group=self._dist_group)
+        return hits
 
     def snapshot_weights(self):
         """Keeps a device copy of the current weights for reset_weights()."""
