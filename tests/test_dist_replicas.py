@@ -1,5 +1,6 @@
-"""The N > 1 path of the benchmark is replicas only: its plumbing (max-over-ranks timing, whole-job
-throughput, per-rank seeds) is covered here with two gloo ranks on CPU."""
+"""The N > 1 paths with two gloo ranks on CPU: the benchmark's replicas (max-over-ranks timing, whole-job
+throughput, per-rank seeds) and the reducer that the exact data-parallel mode hands its max / sum
+words to (the two-rank run of the kernels themselves is tests/test_gpu_dp.py)."""
 import os
 import socket
 
@@ -52,3 +53,42 @@ def test_two_gloo_ranks_reduce_timing_and_draw_distinct_batches():
 def test_single_process_is_the_identity():
     assert max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
     assert aggregate_throughput(64, 5.0, 1) == 12800.0
+
+
+def _reducer_worker(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2009_13108_b200.api import REDUCE_MAX_U32, REDUCE_MAX_U64, REDUCE_SUM_I32, dist_reducer
+    reduce = dist_reducer()
+    # the three quantities the exact data-parallel mode combines, as the library hands them over:
+    # slices of a byte workspace viewed as int32 / int64
+    ws = torch.zeros(256 + 64, dtype=torch.uint8)
+    m32 = ws[0:4].view(torch.int32)
+    m64 = ws[8:16].view(torch.int64)
+    acc = ws[256:256 + 16].view(torch.int32)
+    m32[0] = 1000 + 7 * rank
+    m64[0] = (1 << 40) + (3 - rank)
+    acc.copy_(torch.tensor([5, -6, 7 * (rank + 1), -2147483000 * rank], dtype=torch.int32))
+    reduce(m32, REDUCE_MAX_U32)
+    reduce(m64, REDUCE_MAX_U64)
+    reduce(acc, REDUCE_SUM_I32)
+    q.put((rank, int(m32[0]), int(m64[0]), acc.tolist()))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_the_data_parallel_reducer_combines_max_and_sum_over_two_gloo_ranks():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_reducer_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, m32, m64, acc in res:                       # the same on every rank
+        assert m32 == 1007
+        assert m64 == (1 << 40) + 3
+        assert acc == [10, -12, 21, -2147483000]
