@@ -224,7 +224,8 @@ extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
     }
     case NITI_OP_INT_XENT:
       if (nd != 2 || d[0] <= 0 || d[1] <= 0) return 0;
-      return NITI_WS_HEADER + round_up((size_t)d[0] * 16, 256);   // two 64-bit scalars per sample
+      // two 64-bit scalars per sample + the tables of many-row calls (256 x 256 x (2 + 1) + 256 bytes)
+      return NITI_WS_HEADER + round_up((size_t)d[0] * 16, 256) + 196864;
     default:
       return 0;
   }

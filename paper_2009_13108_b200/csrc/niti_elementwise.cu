@@ -436,13 +436,62 @@ __device__ __forceinline__ int warp_sum_i(int v) {
   return v;
 }
 
+// Tables for many rows (B >= XENT_TAB_MIN_ROWS).  The offset p of Eq. 4 is x-hat of one of the 256
+// logit values, so there are at most 256 different T tables and, once the shared binary point is
+// known, 256 different tables of rounded results: they are computed once per call (two launches of
+// 256 x 256 threads) and a row copies the 512- or 256-byte line it needs instead of evaluating
+// 2 x 256 64-bit expressions of its own.  ttab[i][v] = T(v - 128) with p = x-hat(i - 128) (16 bits:
+// entries a row can use are at most 2^9); thr[t] = 128 + the smallest logit whose x-hat exceeds
+// x-hat(t - 128) - 10; qtab[i][v] = T rounded with the shared binary point.  With tables the first
+// scalar of a row is p * 256 + (index of its line).
+constexpr int XENT_TAB_MIN_ROWS = 1024;
+struct XentTables {
+  unsigned short *ttab;
+  unsigned char *qtab;
+  unsigned char *thr;
+};
+
+__global__ void __launch_bounds__(256)
+xent_ttab_kernel(const int32_t *__restrict__ s_a_ptr, XentTables t) {
+  const int s = *s_a_ptr;
+  if (s < -22 || s > 24 || s <= -7) return;             // (Eq. 2 needs no table of T)
+  const long long sh_amt = 15 - (long long)s;
+  const int i = blockIdx.x, v = threadIdx.x;
+  const long long p = xent_xhat(i - 128, sh_amt);
+  t.ttab[i * 256 + v] = (unsigned short)xent_T(v - 128, s, sh_amt, p);
+  if (i == 0) {
+    const long long mx = xent_xhat(v - 128, sh_amt);
+    int lo = -128, hi = v - 128;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (xent_xhat(mid, sh_amt) > mx - 10) hi = mid; else lo = mid + 1;
+    }
+    t.thr[v] = (unsigned char)(lo + 128);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+xent_qtab_kernel(const int32_t *__restrict__ s_a_ptr, const WsHeader *__restrict__ hdr, XentTables t, int round_mode) {
+  const int s = *s_a_ptr;
+  if (s < -22 || s > 24) return;
+  const unsigned long long mxv = hdr->maxabs64;
+  const int b = 64 - __clzll((long long)mxv);
+  const int bp = b > 7 ? b - 7 : 0;
+  const long long sh_amt = 15 - (long long)s;
+  const int i = blockIdx.x, v = threadIdx.x;
+  const long long p = s <= -7 ? 0 : xent_xhat(i - 128, sh_amt);
+  const unsigned long long T = (unsigned long long)xent_T(v - 128, s, sh_amt, p);
+  t.qtab[i * 256 + v] = (unsigned char)niti_round_mag<unsigned long long>(T, bp, 127ull, round_mode);
+}
+
+template <bool TAB>
 __global__ void __launch_bounds__(32 * XENT_WARPS)
 xent_row_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
                      const int32_t *__restrict__ labels, long long *__restrict__ rowinfo, WsHeader *hdr,
-                     int32_t *__restrict__ n_correct, int B, int N, uint32_t *__restrict__ status) {
+                     int32_t *__restrict__ n_correct, int B, int N, uint32_t *__restrict__ status, XentTables tabs) {
   __shared__ unsigned long long sh_max[XENT_WARPS];
   __shared__ int sh_hit[XENT_WARPS];
-  __shared__ unsigned short sh_T[XENT_WARPS][256];     // T(a) of Eq. 4 for a = -128 .. 127 (at most 2^9)
+  __shared__ __align__(16) unsigned short sh_T[XENT_WARPS][256];     // T(a) of Eq. 4 for a = -128 .. 127 (at most 2^9)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * XENT_WARPS + warp;
   const int s = *s_a_ptr;
@@ -482,6 +531,7 @@ xent_row_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s
       const int row_top = max(max_other, a_label);
       hit = (a_label > max_before && a_label >= max_after) ? 1 : 0;   // the first arg-max is the label
       long long p = 0, csum, t_other, t_label;
+      int line = 0;                                     // (TAB) the table line of this row
       if (s <= -7) {
         sum_a = warp_sum_i(sum_a);
         sum_q = warp_sum_i(sum_q);
@@ -489,12 +539,17 @@ xent_row_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s
         t_other = N > 1 ? xent_T(max_other, s, sh_amt, 0) : 0;     // T is increasing in the logit
         t_label = xent_T(a_label, s, sh_amt, 0);
       } else {
-        const long long mx = xent_xhat(row_top, sh_amt);
         // smallest logit value whose x-hat exceeds mx - 10 (x-hat is non-decreasing in the logit)
-        int lo = -128, hi = row_top;
-        while (lo < hi) {
-          const int mid = (lo + hi) >> 1;          // floor for negative sums as well
-          if (xent_xhat(mid, sh_amt) > mx - 10) hi = mid; else lo = mid + 1;
+        int lo = -128;
+        if (TAB) {
+          lo = (int)tabs.thr[row_top + 128] - 128;
+        } else {
+          const long long mx = xent_xhat(row_top, sh_amt);
+          int hi = row_top;
+          while (lo < hi) {
+            const int mid = (lo + hi) >> 1;          // floor for negative sums as well
+            if (xent_xhat(mid, sh_amt) > mx - 10) hi = mid; else lo = mid + 1;
+          }
         }
         const unsigned thr4 = (unsigned)(lo & 0xff) * 0x01010101u;
         // sweep 2: the smallest logit of the row that is at least that value
@@ -507,7 +562,13 @@ xent_row_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s
         const int a_star = warp_min_i(hmin_s8x4(mn));
         p = xent_xhat(a_star, sh_amt);
         // table of T over the logit values, then sweep 3: the sum
-        for (int v = lane; v < 256; v += 32) sh_T[warp][v] = (unsigned short)xent_T(v - 128, s, sh_amt, p);
+        if (TAB) {
+          reinterpret_cast<uint4 *>(sh_T[warp])[lane] =
+              reinterpret_cast<const uint4 *>(tabs.ttab + (a_star + 128) * 256)[lane];
+          line = a_star + 128;
+        } else {
+          for (int v = lane; v < 256; v += 32) sh_T[warp][v] = (unsigned short)xent_T(v - 128, s, sh_amt, p);
+        }
         __syncwarp();
         int acc = 0;
         for (int wi = lane; wi < words; wi += 32) {
@@ -522,7 +583,7 @@ xent_row_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s
       const long long on_label = csum - t_label;
       row_max = (unsigned long long)(t_other > on_label ? t_other : on_label);
       if (lane == 0) {
-        rowinfo[2 * (long long)r] = p;
+        rowinfo[2 * (long long)r] = TAB ? p * 256 + line : p;
         rowinfo[2 * (long long)r + 1] = csum;
       }
     }
@@ -538,12 +599,13 @@ xent_row_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s
   }
 }
 
+template <bool TAB>
 __global__ void __launch_bounds__(32 * XENT_WARPS)
 xent_round_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
                        const int32_t *__restrict__ labels, const long long *__restrict__ rowinfo,
                        const WsHeader *__restrict__ hdr, int8_t *__restrict__ out, int B, int N, int round_mode,
-                       int32_t *__restrict__ b_out) {
-  __shared__ unsigned char sh_q[XENT_WARPS][256];        // rounded T(a) for a = -128 .. 127
+                       int32_t *__restrict__ b_out, XentTables tabs) {
+  __shared__ __align__(8) unsigned char sh_q[XENT_WARPS][256];        // rounded T(a) for a = -128 .. 127
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * XENT_WARPS + warp;
   const unsigned long long mxv = hdr->maxabs64;
@@ -561,11 +623,17 @@ xent_round_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__
     return;
   }
   const long long sh_amt = 15 - (long long)s;
-  const long long p = rowinfo[2 * (long long)r], csum = rowinfo[2 * (long long)r + 1];
+  const long long info = rowinfo[2 * (long long)r], csum = rowinfo[2 * (long long)r + 1];
+  const long long p = TAB ? (info >> 8) : info;
   // off the label e32 = T(a) > 0: one rounded value per logit value
-  for (int v = lane; v < 256; v += 32) {
-    const unsigned long long T = (unsigned long long)xent_T(v - 128, s, sh_amt, p);
-    sh_q[warp][v] = (unsigned char)niti_round_mag<unsigned long long>(T, bp, 127ull, round_mode);
+  if (TAB) {
+    reinterpret_cast<uint2 *>(sh_q[warp])[lane] =
+        reinterpret_cast<const uint2 *>(tabs.qtab + (int)(info & 0xff) * 256)[lane];
+  } else {
+    for (int v = lane; v < 256; v += 32) {
+      const unsigned long long T = (unsigned long long)xent_T(v - 128, s, sh_amt, p);
+      sh_q[warp][v] = (unsigned char)niti_round_mag<unsigned long long>(T, bp, 127ull, round_mode);
+    }
   }
   // on the label e32 = T - sum <= 0
   const int a_label = (int)a[(long long)r * N + label];
@@ -585,19 +653,38 @@ xent_round_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__
 // both passes; the packed path needs whole words per row
 // (ctx may be null: the variant without a context; with one, the max magnitude of the 64-bit
 // gradients is combined over the ranks between the two passes when a reduction hook is installed)
+// tab_mem: 196864 bytes of scratch for the tables of many-row calls, or null
 static int launch_xent(niti_ctx *ctx, cudaStream_t st, const int8_t *a, const int32_t *s_a, const int32_t *labels,
                        long long *rowinfo, WsHeader *hdr, int8_t *e, int32_t *b_e, int32_t *n_correct, int B, int N,
-                       int round_mode, uint32_t *status) {
+                       int round_mode, uint32_t *status, void *tab_mem) {
   const unsigned blocks = (unsigned)((B + XENT_WARPS - 1) / XENT_WARPS);
   const bool packed = (N & 3) == 0 && N >= 64 && (((uintptr_t)a | (uintptr_t)e) & 3) == 0;
-  if (packed) xent_row_fast_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
-  else xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
+  const bool tab = packed && tab_mem != nullptr && B >= XENT_TAB_MIN_ROWS;
+  XentTables t = {nullptr, nullptr, nullptr};
+  if (tab) {
+    t.ttab = (unsigned short *)tab_mem;
+    t.qtab = (unsigned char *)tab_mem + 256 * 256 * 2;
+    t.thr = t.qtab + 256 * 256;
+    xent_ttab_kernel<<<256, 256, 0, st>>>(s_a, t);
+    xent_row_fast_kernel<true><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status, t);
+  } else if (packed) {
+    xent_row_fast_kernel<false><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status, t);
+  } else {
+    xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
+  }
   if (ctx) {
     int rc = niti_reduce(ctx, st, &hdr->maxabs64, 1, NITI_REDUCE_MAX_U64);
     if (rc != NITI_OK) return rc;
   }
-  if (packed) xent_round_fast_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
-  else xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
+  if (tab) {
+    xent_qtab_kernel<<<256, 256, 0, st>>>(s_a, hdr, t, round_mode);
+    xent_round_fast_kernel<true><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e, t);
+    if (ctx) ctx->launches += 2;
+  } else if (packed) {
+    xent_round_fast_kernel<false><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e, t);
+  } else {
+    xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
+  }
   return NITI_OK;
 }
 
@@ -619,7 +706,8 @@ extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st));
     ctx->launches++;
   }
-  int rcx = launch_xent(ctx, st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, ctx->d_status);
+  void *tab_mem = (char *)ws + NITI_WS_HEADER + ((size_t)B * 16 + 255) / 256 * 256;
+  int rcx = launch_xent(ctx, st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, ctx->d_status, tab_mem);
   if (rcx != NITI_OK) return rcx;
   ctx->launches += 2;
   NITI_CUDA_TRY(ctx, cudaGetLastError());
@@ -664,7 +752,7 @@ extern "C" int niti_int_xent_noalloc(void *stream, const int8_t *a, const int32_
   uint32_t *status = (uint32_t *)((char *)base + NITI_WS_HEADER - sizeof(uint32_t));
   if (cudaMemsetAsync(base, 0, NITI_WS_HEADER, st) != cudaSuccess) return NITI_ERR_CUDA;
   if (n_correct && cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st) != cudaSuccess) return NITI_ERR_CUDA;
-  launch_xent(nullptr, st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, status);
+  launch_xent(nullptr, st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, status, nullptr);
   if (cudaGetLastError() != cudaSuccess) return NITI_ERR_CUDA;
   return NITI_OK;
 }

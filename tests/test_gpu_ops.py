@@ -394,6 +394,30 @@ def test_int_xent_packed_rows(niti, oref, s_a):
     niti.check()
 
 
+@pytest.mark.parametrize("s_a", [-22, -9, -7, -6, -4, -2, 0, 3, 9, 24])
+@pytest.mark.parametrize("B,N", [(1024, 64), (1500, 1000), (4096, 128)])
+def test_int_xent_many_rows_use_precomputed_tables(niti, oref, s_a, B, N):
+    """From 1024 rows on, the T and rounded-T tables are computed once per call (one line per
+    possible offset p) and the rows copy their line: same bytes as the oracle, rows with narrow,
+    constant and extreme logits included."""
+    rng = np.random.default_rng(9000 + s_a + B + N)
+    a = _i8(rng, (B, N))
+    labels = rng.integers(0, N, size=B).astype(np.int32)
+    a[0] = 0
+    a[1] = rng.integers(-2, 3, size=N)
+    a[2] = -127; a[2, 5] = 127; labels[2] = 5
+    a[3] = -127; a[3, 6] = 127; labels[3] = 7
+    a[4] = 127
+    a[5] = -128 + (np.arange(N) % 3 == 0)
+    a[6:70] = np.clip(a[6:70] // 16, -8, 7)               # few distinct values: every threshold line gets used
+    for mode in (0, 1):
+        want, b, nc = oref.int_xent(a, s_a, labels, mode)
+        e, b_e, n_correct = niti.int_xent(_T(niti, a), niti.scalar(s_a), _T(niti, labels), round_mode=mode)
+        _eq(e, want)
+        assert (int(b_e), int(n_correct)) == (b, nc)
+    niti.check()
+
+
 def test_int_xent_flags_bad_domain(niti):
     from paper_2009_13108_b200 import NitiError
     a = torch.zeros((4, 8), dtype=torch.int8, device=niti.device)
