@@ -178,8 +178,10 @@ im2col32_rgb3x3_kernel(const int8_t *__restrict__ x, int8_t *__restrict__ xcol, 
         }
         o[wd] = v;
       }
-      dst[2 * px] = make_int4(o[0], o[1], o[2], o[3]);
-      dst[2 * px + 1] = make_int4(o[4], o[5], o[6], o[7]);
+      // one gathered row = one 32-byte sector: a single 256-bit store per pixel
+      asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                   ::"l"(dst + 2 * px), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                   : "memory");
     }
   }
 }
@@ -227,7 +229,8 @@ __global__ void round_compact32_kernel(const int32_t *__restrict__ acc, const Ws
 
 int niti_launch_im2col32(niti_ctx *ctx, cudaStream_t st, const int8_t *x, int8_t *xcol, int B, int H, int W,
                          int Ci, int R, int S, int pad, int Ho, int Wo) {
-  if (Ci == 3 && R == 3 && S == 3 && pad == 1 && (W % 4) == 0 && (long long)B * H < (1LL << 31)) {
+  if (Ci == 3 && R == 3 && S == 3 && pad == 1 && (W % 4) == 0 && (long long)B * H < (1LL << 31) &&
+      ((uintptr_t)xcol & 31) == 0) {
     const int threads = W / 4 >= 128 ? 128 : (W / 4 > 32 ? 64 : 32);
     const size_t smem = (size_t)3 * (W * 3 / 4 + 2) * sizeof(unsigned);
     if (smem <= 48 * 1024) {
