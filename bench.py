@@ -498,9 +498,10 @@ def run_ours(args):
                      "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
                      "peak_source": "2 x %s bf16 sustained (int8 : bf16 = 2 : 1 nominal); nominal int8 4500" % pk["source"],
                      "frac_of_nominal": achieved / 4500.0, "launches": k_n,
-                     # DRAM bytes per multiply, from one ncu capture of the config-4 step
-                     # (profiles/tc_gemm_dram_traffic_vgg16_step.md): 4.60 GB over the step's 47 multiplies,
-                     # against 5.13 GB algorithmic (operands once + int8 result once); null for other configs
+                     # DRAM bytes per multiply, from one single-pass ncu capture (dram__bytes_read.sum +
+                     # dram__bytes_write.sum of every launch of the kernel) of the config-4 step run eagerly:
+                     # 4.60 GB over the step's 47 multiplies, against 5.13 GB algorithmic (operands once +
+                     # int8 result once); null for other configs
                      "traffic": (4.60e9 / 47.0 if args.config == 4 else None),
                      "traffic_unit": "bytes per multiply (mean over the 47 multiplies of the step)",
                      "algorithmic_bytes": (5.13e9 / 47.0 if args.config == 4 else None),
