@@ -161,9 +161,10 @@ def gemm_point(niti, M, N, K, iters=10, dist="uniform", variant="act"):
         a, w = torch.from_numpy(a).to(dev), torch.from_numpy(w).to(dev)
         sa, sw = niti.scalar(-7), niti.scalar(-10)
         out = torch.empty((M, N), dtype=torch.int8, device=dev)
+        s_out, b_out = niti.scalar(), niti.scalar()      # (allocated once: no allocator call per launch)
 
         def run():
-            niti.linear_fwd(a, sa, w, sw, out=out)
+            niti.linear_fwd(a, sa, w, sw, out=out, s_out=s_out, b_out=b_out)
     else:
         e, a2 = gemm_grad_operands(M, N, K, dist)
         e, a2 = torch.from_numpy(e).to(dev), torch.from_numpy(a2).to(dev)
@@ -349,6 +350,60 @@ def run_per_launch(args):
     niti.check()
 
 
+def algorithmic_bytes_per_multiply(net):
+    """Bytes every matrix multiply of one training step must move (both operands once, the int8 result
+    once, and for an error multiply the ReLU gate bytes it reads); one entry per multiply, in the order
+    forward layers, then weight gradient / error of every layer from the last to the first."""
+    fwd, bwd = [], []
+    first = True
+    shape = (net.batch,) + tuple(net.in_shape)
+    for L in net.layers:
+        if L["op"] == "conv":
+            n_in = shape[0] * shape[1] * shape[2] * L["cin"]
+            n_out = shape[0] * shape[1] * shape[2] * L["cout"]
+            n_w = 9 * L["cin"] * L["cout"]
+            shape = shape[:3] + (L["cout"],)
+        elif L["op"] == "pool":
+            shape = (shape[0], shape[1] // 2, shape[2] // 2, shape[3])
+            continue
+        else:
+            n_in, n_out, n_w = net.batch * L["k"], net.batch * L["n"], L["k"] * L["n"]
+            shape = (net.batch, L["n"])
+        fwd.append(n_in + n_w + n_out)
+        layer_bwd = [n_in + n_out + n_w]                 # weight gradient: activations, errors -> g
+        if not first:
+            layer_bwd.append(n_out + n_w + 2 * n_in)     # error: e, w -> e_prev, gated by the input's sign
+        bwd.append(layer_bwd)
+        first = False
+    out = list(fwd)
+    for lb in reversed(bwd):
+        out += lb
+    return out
+
+
+def measured_traffic(kernel_file):
+    """DRAM traffic of the dominant kernel relative to its algorithmic bytes, from the committed ncu
+    summary (profiles/tc_gemm_dram_traffic.json).  The figure belongs to one build of the kernel: it is
+    used only while the kernel source still has the recorded SHA-256."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "tc_gemm_dram_traffic.json")
+    if not os.path.exists(path):
+        return None, "no committed ncu capture"
+    rec = json.load(open(path))
+    sha = hashlib.sha256(open(kernel_file, "rb").read()).hexdigest()
+    if rec.get("kernel_source_sha256") != sha:
+        return None, "kernel source changed since the committed ncu capture (%s)" % rec.get("captured", "?")
+    return rec, None
+
+
+def spawn_ranks(args):
+    """`python bench.py --gpus N` without a launcher: start the N ranks here (one process per GPU,
+    rendezvous on 127.0.0.1) and pass their output through."""
+    from paper_2009_13108_b200.dist_util import launch_ranks
+    argv = [a for a in sys.argv[1:]]
+    return launch_ranks([os.path.abspath(__file__)] + argv, args.gpus)
+
+
 def run_ours(args):
     import torch
     rank = int(os.environ.get("RANK", "0"))
@@ -359,15 +414,17 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     torch.cuda.set_device(local)
+    import hashlib
+    import numpy as np
     from paper_2009_13108_b200 import Niti, NitiTrainer
-    from synth import config_net, make_net_inputs
+    from paper_2009_13108_b200.build import CSRC
+    from synth import config_net, make_net_inputs, make_step_batch
 
     niti = Niti(local)
     net = config_net(args.config)
     from paper_2009_13108_b200.dist_util import aggregate_throughput, max_over_ranks, rank_seed
     net.seed = rank_seed(net.seed, rank)         # every rank draws its own batch and replica
     x, labels, weights = make_net_inputs(net)
-    import hashlib
     wh = hashlib.sha256()
     for w in weights:
         wh.update(memoryview(w).cast("B"))
@@ -375,19 +432,34 @@ def run_ours(args):
                      "labels": hashlib.sha256(memoryview(labels).cast("B")).hexdigest()[:16],
                      "weights": wh.hexdigest()[:16]}      # guards against drift of the seeded generator
     tr = NitiTrainer(niti, net, weights, fused_update=args.fused_update, pool_codes=args.pool_codes)
-    xh = torch.from_numpy(x).pin_memory()
-    lh = torch.from_numpy(labels).pin_memory()
+    # Config 2 is "trained for 100 integer steps": consecutive steps on fresh mini-batches with the weights
+    # carried over.  The other configs time ONE step K times: every iteration restores the seeded weights
+    # (device-to-device copies inside the timed region) and repeats the same step; repeated steps on
+    # random labels saturate the big nets' weights and leave the domain of the integer loss.
+    train = args.config == 2
+    n_batches = min(args.steps + args.warmup + 1, 128) if train else 1
+    host_batches = []
+    for t in range(n_batches):
+        bx, bl = (x, labels) if t == 0 else make_step_batch(net, t)
+        host_batches.append((torch.from_numpy(bx).pin_memory(), torch.from_numpy(bl).pin_memory()))
+    dev_batches = [(bx.to(niti.device), bl.to(niti.device)) for bx, bl in host_batches]
+    xh, lh = host_batches[0]
     tr.load_batch(xh, lh)
     tr.snapshot_weights()
     torch.cuda.synchronize()
+    step_no = [0]
+
+    def step_body():
+        tr.step()
 
     def one_step():
-        # "one training step timed over K iterations": every iteration is the same step, from the
-        # seeded initial weights (restored by device-to-device copies inside the timed region).
-        # Without this the random-label task saturates the int8 weights within a few steps and the
-        # logits' exponent leaves the domain of the integer loss.
-        tr.reset_weights()
-        tr.step()
+        if train:
+            bx, bl = dev_batches[step_no[0] % n_batches]       # batch already resident in HBM
+            tr.load_batch(bx, bl)
+            step_no[0] += 1
+        else:
+            tr.reset_weights()
+        step_body()
 
     def barrier():
         torch.cuda.synchronize()
@@ -400,13 +472,17 @@ def run_ours(args):
     for _ in range(args.warmup):
         one_step()
     niti.check()
+    launches_per_step = None
     if args.graph:
         # replay the captured launch sequence (same kernels, same order) instead of re-issuing it
         # from Python: removes the host-side launch cost, which dominates the small configs
         launches_per_step = niti.launch_count()
-        replay = tr.capture(with_reset=True)
+        replay = tr.capture(with_reset=not train)
         launches_per_step = niti.launch_count() - launches_per_step
-        one_step = replay
+        step_body = replay
+        if not train:
+            def one_step():                       # noqa: F811  (the graph holds the weight restore too)
+                replay()
         one_step()
         niti.check()
     niti.profile_enable(not args.graph)
@@ -414,17 +490,26 @@ def run_ours(args):
     barrier()
     l0 = niti.launch_count()
     redo0 = niti.redo_count()
-    e0, e1 = torch.cuda.Event(True), torch.cuda.Event(True)
-    e0.record()
-    for _ in range(args.steps):
+    marks = [torch.cuda.Event(True) for _ in range(args.steps + 1)]
+    marks[0].record()
+    for i in range(args.steps):
         one_step()
-    e1.record()
+        marks[i + 1].record()
     barrier()
-    ms = e0.elapsed_time(e1)
+    ms = marks[0].elapsed_time(marks[-1])
+    per_step = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
     launches = niti.launch_count() - l0
     if args.graph:
         launches = launches_per_step * args.steps
     redo = niti.redo_count() - redo0
+    niti.check()
+    # digests of what the timed region left behind (the oracle-written digests of the tests are the
+    # same quantities): every weight tensor and the logits
+    w_sha = [hashlib.sha256(w.cpu().numpy().tobytes()).hexdigest() for w in tr.weights]
+    out_digests = {"weights_sha256_16": [h[:16] for h in w_sha],
+                   "weights_combined_sha256_16": hashlib.sha256("".join(w_sha).encode()).hexdigest()[:16],
+                   "logits_sha256_16": hashlib.sha256(tr.acts[-1].cpu().numpy().tobytes()).hexdigest()[:16],
+                   "hits_last_step": int(tr.n_correct)}
     if args.graph:
         # per-kernel timing for the roofline: the same K steps issued eagerly with a CUDA event pair
         # around every tensor-core launch (events cannot be read back from inside a graph replay)
@@ -433,6 +518,8 @@ def run_ours(args):
             tr.reset_weights()
             tr.step()
         torch.cuda.synchronize()
+        if train:
+            tr.reset_weights()
     k_ms, k_n, k_ops = niti.profile_read()
     niti.profile_enable(False)
     # ---- end to end: host batch in, hit count out, every step ----
@@ -446,12 +533,14 @@ def run_ours(args):
     # batch runs on a copy stream while the current step computes (double buffering through the
     # trainer's prefetch_batch / commit_batch); the hit count of every step is copied to the host and
     # the host waits for it one step behind, so that the next step is already queued
-    tr.prefetch_batch(xh, lh)
+    tr.prefetch_batch(*host_batches[0])
     for i in range(args.steps):
         tr.commit_batch()
         if i + 1 < args.steps:
-            tr.prefetch_batch(xh, lh)
-        one_step()
+            tr.prefetch_batch(*host_batches[(i + 1) % n_batches])
+        if not train and not args.graph:
+            tr.reset_weights()
+        step_body()
         result[i:i + 1].copy_(tr.n_correct, non_blocking=True)
         read_back[i].record()
         if i > 0:
@@ -462,6 +551,25 @@ def run_ours(args):
     ms_e2e = t0.elapsed_time(t1)
     clocks = sampler.stop()
     niti.check()
+    # ---- sustained: the same step replayed for seconds, so that the power cap and the clocks it
+    # settles at are part of the number ----
+    sustained = None
+    if args.sustain_seconds > 0 and not train:
+        n_sus = max(args.steps, int(args.sustain_seconds * 1e3 / (ms / args.steps)) + 1)
+        s2 = ClockSampler(local)
+        barrier()
+        s2.start()
+        e0, e1 = torch.cuda.Event(True), torch.cuda.Event(True)
+        e0.record()
+        for _ in range(n_sus):
+            one_step()
+        e1.record()
+        barrier()
+        sus_ms = e0.elapsed_time(e1)
+        sc = s2.stop()
+        niti.check()
+        sustained = {"steps": n_sus, "seconds": sus_ms / 1e3, "ms_per_step": sus_ms / n_sus,
+                     "value": net.batch * n_sus * world / (sus_ms / 1e3), "unit": UNIT, "clocks": sc}
     ms, ms_e2e = max_over_ranks([ms, ms_e2e], device="cuda")
     if rank != 0:
         if dist is not None:
@@ -470,24 +578,39 @@ def run_ours(args):
     pk = _peaks()
     images = net.batch * args.steps * world
     ops_step = net.int8_ops_per_step()
-    # int8 dense tensor peak: twice the measured bf16 rate of this machine (sustained: the kernel is
-    # timed inside a long step); nominal 4500 TOPS given for context
-    int8_peak = 2.0 * pk["bf16_sustained"]
+    # Dense int8 tensor peak = 2 x the bf16 rate measured on this machine (int8 : bf16 = 2 : 1 nominal).  The
+    # dominant kernel is timed launch by launch with CUDA events in a region far shorter than a second
+    # (no power capping: the clocks line shows it), so the burst measurement is its denominator; the
+    # sustained one belongs to the seconds-long leg below.
+    int8_peak = 2.0 * pk["bf16_burst"]
     achieved = k_ops / max(k_ms, 1e-9) / 1e9
+    alg = algorithmic_bytes_per_multiply(net)
+    alg_mean = sum(alg) / len(alg)
+    rec, why = measured_traffic(os.path.join(CSRC, "niti_tc_gemm.cu"))
+    traffic = rec["dram_bytes_per_launch"] / rec["algorithmic_bytes_per_launch"] * alg_mean if rec else None
+    if sustained is not None:
+        sus_tops = ops_step / sustained["ms_per_step"] / 1e9
+        mhz = sustained["clocks"].get("sm_mhz")
+        sustained.update({"step_tops": sus_tops, "peak": 2.0 * pk["bf16_sustained"],
+                          "frac_of_2x_bf16_sustained": sus_tops / (2.0 * pk["bf16_sustained"]),
+                          "ms_x_mhz": (sustained["ms_per_step"] * mhz) if mhz else None})
     line = {
         "metric": METRIC, "value": aggregate_throughput(net.batch * args.steps, ms, world), "unit": UNIT,
         "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+        "ms_per_step_median": per_step[len(per_step) // 2], "ms_per_step_best": per_step[0],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s8",
         "data": "synthetic",
         "config": {"workload": "config%d:%s" % (args.config, net.name), "global_batch": net.batch * world,
                    "per_gpu_batch": net.batch, "int8_ops_per_step": ops_step,
                    "l2": "working set (activations + int32 scratch) exceeds the 126 MB L2",
-                   "state": "weights restored to the seeded initial values before every step",
+                   "state": ("weights carried from step to step, a fresh mini-batch every step" if train else
+                             "weights restored to the seeded initial values before every step"),
                    "launch": "cuda-graph replay" if args.graph else "eager",
                    "weight_update": "fused with the weight gradient" if args.fused_update else "separate call",
                    "parallelism": "replicas" if world > 1 else "single",
                    "inputs_sha256_16": input_digests},
+        "outputs": out_digests,
         "step_tops": ops_step / (ms / args.steps) / 1e9,
         "clocks": clocks,
         "e2e": {"value": images / (ms_e2e / 1e3), "unit": UNIT, "h2d_bytes_per_step": int(xh.numel() + lh.numel() * 4),
@@ -496,24 +619,45 @@ def run_ours(args):
         "speculation_redo_passes": int(redo),
         "roofline": {"bound": "tensor", "kernel": "tc_gemm_kernel (tcgen05 kind::i8)", "achieved": achieved,
                      "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
-                     "peak_source": "2 x %s bf16 sustained (int8 : bf16 = 2 : 1 nominal); nominal int8 4500" % pk["source"],
-                     "frac_of_nominal": achieved / 4500.0, "launches": k_n,
-                     # DRAM bytes per multiply, from one single-pass ncu capture (dram__bytes_read.sum +
-                     # dram__bytes_write.sum of every launch of the kernel) of the config-4 step run eagerly:
-                     # 4.60 GB over the step's 47 multiplies, against 5.13 GB algorithmic (operands once +
-                     # int8 result once); null for other configs
-                     "traffic": (4.60e9 / 47.0 if args.config == 4 else None),
-                     "traffic_unit": "bytes per multiply (mean over the 47 multiplies of the step)",
-                     "algorithmic_bytes": (5.13e9 / 47.0 if args.config == 4 else None),
+                     "peak_source": "2 x %s bf16 burst (%.1f TFLOP/s; int8 : bf16 = 2 : 1 nominal): the kernel is timed "
+                                    "per launch, the region lasts %.0f ms" % (pk["source"], pk["bf16_burst"], ms),
+                     "frac_of_nominal_4500": achieved / 4500.0,
+                     "frac_of_measured_issue_peak_4582": achieved / 4582.0,
+                     "frac_of_2x_bf16_sustained": achieved / (2.0 * pk["bf16_sustained"]),
+                     "launches": k_n,
+                     # DRAM bytes per multiply: the ratio DRAM bytes / algorithmic bytes of one ncu capture
+                     # of a single launch (profiles/tc_gemm_dram_traffic.json) times the mean algorithmic
+                     # bytes of this step's multiplies; null when the kernel changed after the capture
+                     "traffic": traffic, "traffic_note": why if rec is None else rec.get("workload"),
+                     "traffic_unit": "bytes per multiply (mean over the %d multiplies of the step)" % len(alg),
+                     "algorithmic_bytes": alg_mean,
                      "timing": "CUDA event pair around every launch of the kernel over %d steps%s" % (
                          args.steps, " (eager pass after the graph-replayed timed region)" if args.graph else "")},
     }
+    if sustained is not None:
+        line["sustained"] = sustained
     if args.gemm:
         line["gemm_sweep"] = [gemm_point(niti, *s) for s in [(4096, 4096, 4096), (8192, 8192, 8192)]]
     line["cpu_baseline"] = {k: v for k, v in cpu_baseline(args.config).items() if k != "seconds"}
+    if args.config in (0, 2):
+        line["cpu_baseline"]["single_thread"] = cpu_baseline_single_thread(args.config)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def cpu_baseline_single_thread(config):
+    """The same oracle sample on one host thread (a child process with OMP_NUM_THREADS=1)."""
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    for k in ("RANK", "WORLD_SIZE", "LOCAL_RANK"):
+        env.pop(k, None)
+    try:
+        out = subprocess.run([sys.executable, os.path.abspath(__file__), "--cpu-baseline-json", "--config", str(config)],
+                             env=env, capture_output=True, text=True, timeout=180)
+        d = json.loads(out.stdout.strip().splitlines()[-1])
+        return {"value": d["value"], "unit": UNIT, "cores": 1, "sample": d["sample"]}
+    except Exception as exc:      # the baseline is a reported extra: never fail the bench over it
+        return {"unavailable": repr(exc)}
 
 
 def main():
@@ -540,7 +684,13 @@ def main():
     ap.add_argument("--per-launch", action="store_true",
                     help="one eager step with a CUDA event pair around every tensor-core multiply")
     ap.add_argument("--full-sweep", action="store_true", help="with --sweep: time the second operand set on every shape")
+    ap.add_argument("--sustain-seconds", type=float, default=3.0,
+                    help="also replay the step for this many seconds and report the sustained rate (0: skip)")
+    ap.add_argument("--cpu-baseline-json", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
+    if args.cpu_baseline_json:
+        print(json.dumps(cpu_baseline(args.config, budget_s=15.0)), flush=True)
+        return
     if args.sweep:
         run_sweep(args)
         return
@@ -562,6 +712,8 @@ def main():
         return
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     else:
         run_ours(args)
 

@@ -29,8 +29,16 @@
  * with the sign re-applied, saturating at 2^mbits - 1.  mbits is 7 for
  * activations and errors and m_u (1..7) for weight gradients.
  *
- * Contract on accumulators: the caller guarantees |sum| < 2^31 for every
- * output (always true when the contraction length is <= 133144).
+ * Contract on accumulators (Section 3.2: results are accumulated in int32): the
+ * caller guarantees |sum| < 2^31 for every output.  This always holds when the
+ * contraction length is <= 133144.  The weight-gradient calls contract over
+ * the batch (niti_linear_bwd) or over batch x output pixels (niti_conv_wgrad:
+ * 3.2 million on the first layers of a 224 x 224 network), the one place where
+ * the contract can really break.  Contractions longer than 131072 are always
+ * split over CTAs into pieces that cannot wrap, and the library adds up the
+ * largest partial sum of every piece: when that bound reaches 2^31 the device
+ * status bit NITI_DEV_ACC_RANGE is raised (the bound is conservative: the bit
+ * can be raised for a tensor whose true sums still fit, never the reverse).
  *
  * Return value: NITI_OK or an error code; nothing is enqueued on error.
  */
@@ -71,6 +79,9 @@ extern "C" {
 #define NITI_DEV_EXP_RANGE 2u    /* an exponent left the int8 range            */
 #define NITI_DEV_XENT_RANGE 4u   /* s_a outside [-22, 24] in niti_int_xent     */
 #define NITI_DEV_BAD_LABEL 8u    /* a label outside [0, N)                     */
+#define NITI_DEV_INTERNAL 32u    /* a consistency check inside a kernel failed: outputs of that call are not exact */
+#define NITI_DEV_ACC_RANGE 16u   /* an int32 accumulator may have wrapped: in a contraction split over
+                                  * CTAs the largest partial sums of the splits add up to 2^31 or more */
 
 typedef struct niti_ctx niti_ctx;
 

@@ -2,7 +2,6 @@
 // accumulate -> bit-width -> shift-and-round sequence of Algorithm 1 for each layer op.
 #include "niti_common.cuh"
 
-int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr);
 int niti_launch_im2col32(niti_ctx *ctx, cudaStream_t st, const int8_t *x, int8_t *xcol, int B, int H, int W,
                          int Ci, int R, int S, int pad, int Ho, int Wo);
 int niti_launch_pad_pitch(niti_ctx *ctx, cudaStream_t st, const int8_t *src, int8_t *dst, int rows, int n, int pitch);
@@ -262,7 +261,7 @@ static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, 
     return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
   WsHeader *hdr = (WsHeader *)ws;
   int32_t *acc = (int32_t *)((char *)ws + NITI_WS_HEADER);
-  NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, sizeof(WsHeader), st));
+  NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, NITI_WS_HEADER, st));        // reduction scalars and split maxima
   ctx->launches++;
   int rc = NITI_ERR_SHAPE;
   bool fused = false;
@@ -452,7 +451,7 @@ static int conv_wgrad_impl(niti_ctx *ctx, void *stream, const int8_t *x, const i
     char *base = (char *)ws + NITI_WS_HEADER + round_up((size_t)(p.gm * p.gn) * 4, 256);
     int8_t *xcol = (int8_t *)base;
     int32_t *acc32 = (int32_t *)(base + round_up(M * 32, 256) + round_up((size_t)Cout * 32, 256));
-    NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, sizeof(WsHeader), st));
+    NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, NITI_WS_HEADER, st));
     ctx->launches++;
     int rc = niti_launch_im2col32(ctx, st, x, xcol, B, H, W, Cin, R, S, pad, p.Ho, p.Wo);
     if (rc != NITI_OK) return rc;

@@ -11,7 +11,8 @@
 struct niti_ctx {
   int device;
   int sm_count;
-  int engine;               // 0 auto, 1 CUDA-core kernels only, 2 single-CTA tensor-core kernel, 3 paired-CTA only
+  int engine;               // niti_set_engine: 0 auto, 1 CUDA-core kernels only, 2 single-CTA tensor-core kernel,
+                            // 3 paired-CTA only, 4 two-pass (int32 spill) epilogue, 5 no resident-weights mode
   uint32_t *d_status;       // device status word
   uint64_t launches;
   uint64_t tc_launches;     // launches of the tensor-core matrix-multiply kernel
@@ -28,12 +29,24 @@ struct niti_ctx {
   // combined over the ranks before the rounding may use it
   niti_reduce_fn reduce_fn;
   void *reduce_user;
+  // per-device facts of the tensor-core kernel, indexed by CTAs per tile (1 or 2): co-resident CTAs /
+  // CTA pairs (0 = not asked yet) and the dynamic shared-memory limit already set on the kernel
+  int tc_units[3];
+  size_t tc_attr_smem[3];
 };
 
 
 
 #define NITI_PROF_MAX 8192
-#define NITI_WS_HEADER 256  // bytes reserved at the start of every workspace for reduction scalars
+#define NITI_WS_HEADER 4096 // bytes reserved at the start of every workspace: reduction scalars, then split maxima
+// A contraction that is split over CTAs adds int32 partial sums; split s records the largest magnitude
+// among its partial sums in split_max[s] (unsigned words from byte NITI_SPLIT_MAX_OFF of the header).
+// The sum of those maxima bounds every accumulator of the tensor: when it reaches 2^31 the int32
+// contract of Section 3.2 can no longer be vouched for and NITI_DEV_ACC_RANGE is raised.  Every split
+// covers at most NITI_SPLIT_MAX_K contraction elements, so a partial sum itself cannot wrap.
+#define NITI_SPLIT_MAX_OFF 256
+#define NITI_MAX_SPLITS 960
+#define NITI_SPLIT_MAX_K 131072
 
 // Scalars at the start of a workspace.
 struct WsHeader {
@@ -47,6 +60,10 @@ struct WsHeader {
   unsigned int pad1[1];
 };
 static_assert(sizeof(WsHeader) == 32, "workspace header layout");
+static_assert(NITI_SPLIT_MAX_OFF + 4 * NITI_MAX_SPLITS <= NITI_WS_HEADER, "split maxima fit the header");
+__host__ __device__ __forceinline__ unsigned int *niti_split_max(WsHeader *hdr) {
+  return reinterpret_cast<unsigned int *>(reinterpret_cast<char *>(hdr) + NITI_SPLIT_MAX_OFF);
+}
 
 #define NITI_CUDA_TRY(ctx, expr)                                                        \
   do {                                                                                  \
@@ -125,7 +142,9 @@ struct GemmProblem {
 };
 
 int niti_reduce_after_gemm(niti_ctx *ctx, cudaStream_t st, int kind, int32_t *acc, long long n, WsHeader *hdr);
-int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr);
+// max |acc| into hdr->maxabs32; splits > 1: also adds up the split maxima of the header and raises
+// NITI_DEV_ACC_RANGE when an accumulator may have left the int32 range
+int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr, int splits = 0);
 // Plain CUDA-core engine: writes int32 accumulators to acc[gm][gn] and max|acc| to hdr->maxabs32.
 int niti_simt_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t *acc, WsHeader *hdr);
 // What follows the multiply: rounding target and the scalars of Algorithm 2.

@@ -722,7 +722,8 @@ extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const
 // scalars per sample) in a fixed device array that is part of the library image, for callers that must
 // not allocate device memory.  Every GPU that loads the library carries the array until exit.
 // ---------------------------------------------------------------------------------------------
-#define NITI_NOALLOC_BYTES (NITI_WS_HEADER + 8 * NITI_XENT_NOALLOC_MAX_ELEMS)
+#define NITI_NOALLOC_HEADER 256       // reduction scalars of this variant (its last word: status bits)
+#define NITI_NOALLOC_BYTES (NITI_NOALLOC_HEADER + 8 * NITI_XENT_NOALLOC_MAX_ELEMS)
 static __device__ __align__(256) unsigned char g_xent_scratch[NITI_NOALLOC_BYTES];
 // The name above is only a host-side handle in host code; the device address is looked up once per
 // device (with that device current) and cached here.
@@ -749,11 +750,11 @@ extern "C" int niti_int_xent_noalloc(void *stream, const int8_t *a, const int32_
   }
   cudaStream_t st = (cudaStream_t)stream;
   WsHeader *hdr = (WsHeader *)base;
-  long long *rowinfo = (long long *)((char *)base + NITI_WS_HEADER);
+  long long *rowinfo = (long long *)((char *)base + NITI_NOALLOC_HEADER);
   // the array keeps what the previous call left: the reduction scalars must start at zero.  The last
   // word of the header takes the (unreported) status bits of this variant.
-  uint32_t *status = (uint32_t *)((char *)base + NITI_WS_HEADER - sizeof(uint32_t));
-  if (cudaMemsetAsync(base, 0, NITI_WS_HEADER, st) != cudaSuccess) return NITI_ERR_CUDA;
+  uint32_t *status = (uint32_t *)((char *)base + NITI_NOALLOC_HEADER - sizeof(uint32_t));
+  if (cudaMemsetAsync(base, 0, NITI_NOALLOC_HEADER, st) != cudaSuccess) return NITI_ERR_CUDA;
   if (n_correct && cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st) != cudaSuccess) return NITI_ERR_CUDA;
   launch_xent(nullptr, st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, status, nullptr);
   if (cudaGetLastError() != cudaSuccess) return NITI_ERR_CUDA;

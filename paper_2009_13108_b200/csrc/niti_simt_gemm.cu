@@ -146,34 +146,43 @@ simt_gemm_kernel(Addr q, int32_t *__restrict__ acc, WsHeader *hdr, long long k_p
       long long n = n0 + tx * 4 + j;
       if (n >= q.gn) continue;
       int v = c[i][j];
+      const unsigned a = v < 0 ? 0u - (unsigned)v : (unsigned)v;
+      mx = a > mx ? a : mx;
       if (SPLIT) {
         if (v) atomicAdd(&acc[m * q.gn + n], v);
       } else {
         acc[m * q.gn + n] = v;
-        unsigned a = v < 0 ? 0u - (unsigned)v : (unsigned)v;
-        mx = a > mx ? a : mx;
       }
     }
   }
-  if (!SPLIT) {
-    for (int o = 16; o > 0; o >>= 1) {
-      unsigned u = __shfl_xor_sync(0xffffffffu, mx, o);
-      mx = u > mx ? u : mx;
-    }
-    if ((tid & 31) == 0) smax[tid >> 5] = mx;
-    __syncthreads();
-    if (tid == 0) {
-      for (int i = 1; i < 8; ++i) mx = smax[i] > mx ? smax[i] : mx;
-      if (mx) atomicMax(&hdr->maxabs32, mx);
-    }
+  // block-wide max magnitude: of the finished accumulators (unsplit), or of this split's partial sums
+  // (kept per split in the header; their sum bounds every accumulator of the tensor)
+  for (int o = 16; o > 0; o >>= 1) {
+    unsigned u = __shfl_xor_sync(0xffffffffu, mx, o);
+    mx = u > mx ? u : mx;
+  }
+  if ((tid & 31) == 0) smax[tid >> 5] = mx;
+  __syncthreads();
+  if (tid == 0) {
+    for (int i = 1; i < 8; ++i) mx = smax[i] > mx ? smax[i] : mx;
+    if (mx) atomicMax(SPLIT ? niti_split_max(hdr) + blockIdx.z : &hdr->maxabs32, mx);
   }
 }
 
 }  // namespace
 
-// max |v| over an int32 tensor (used after split-K accumulation)
+// max |v| over an int32 tensor (used after split-K accumulation).  splits > 1: block 0 also adds up the
+// largest partial-sum magnitude of every split; that sum bounds every accumulator, and when it reaches
+// 2^31 the int32 contract cannot be vouched for.
 __global__ void __launch_bounds__(256)
-maxabs_i32_kernel(const int32_t *__restrict__ acc, long long n, WsHeader *hdr) {
+maxabs_i32_kernel(const int32_t *__restrict__ acc, long long n, WsHeader *hdr, int splits, uint32_t *status) {
+  if (splits > 1 && blockIdx.x == 0 && threadIdx.x < 32) {
+    unsigned long long bound = 0;
+    const unsigned *sm = niti_split_max(hdr);
+    for (int i = threadIdx.x; i < splits; i += 32) bound += sm[i];
+    for (int o = 16; o > 0; o >>= 1) bound += __shfl_xor_sync(0xffffffffu, bound, o);
+    if (threadIdx.x == 0 && bound >= 0x80000000ull) atomicOr(status, NITI_DEV_ACC_RANGE);
+  }
   unsigned mx = 0;
   const long long nvec = n >> 2;
   const long long stride = (long long)gridDim.x * blockDim.x;
@@ -204,11 +213,11 @@ maxabs_i32_kernel(const int32_t *__restrict__ acc, long long n, WsHeader *hdr) {
   }
 }
 
-int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr) {
+int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr, int splits) {
   long long blocks = ((n >> 2) + 255) / 256;
   if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
   if (blocks < 1) blocks = 1;
-  maxabs_i32_kernel<<<(unsigned)blocks, 256, 0, st>>>(acc, n, hdr);
+  maxabs_i32_kernel<<<(unsigned)blocks, 256, 0, st>>>(acc, n, hdr, splits, ctx->d_status);
   ctx->launches++;
   NITI_CUDA_TRY(ctx, cudaGetLastError());
   return NITI_OK;
@@ -231,8 +240,11 @@ int niti_simt_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t
     long long max_splits = p.gk / 1024;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
-    if (splits > 65535) splits = 65535;
   }
+  // no split longer than NITI_SPLIT_MAX_K (a partial sum then cannot wrap), at most NITI_MAX_SPLITS splits
+  const long long min_splits = (p.gk + NITI_SPLIT_MAX_K - 1) / NITI_SPLIT_MAX_K;
+  if (splits < min_splits) splits = min_splits;
+  if (splits > NITI_MAX_SPLITS) return niti_fail(ctx, NITI_ERR_SHAPE, "simt gemm: contraction too long");
   long long kps = (p.gk + splits - 1) / splits;
   kps = (kps + TK - 1) / TK * TK;
   splits = (p.gk + kps - 1) / kps;
@@ -243,7 +255,7 @@ int niti_simt_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t
     simt_gemm_kernel<true><<<grid, 256, 0, st>>>(q, acc, hdr, kps);
     ctx->launches++;
     NITI_CUDA_TRY(ctx, cudaGetLastError());
-    return niti_launch_maxabs(ctx, st, acc, p.gm * p.gn, hdr);
+    return niti_launch_maxabs(ctx, st, acc, p.gm * p.gn, hdr, (int)splits);
   }
   simt_gemm_kernel<false><<<grid, 256, 0, st>>>(q, acc, hdr, kps);
   ctx->launches++;

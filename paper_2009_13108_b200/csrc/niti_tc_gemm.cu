@@ -1,9 +1,10 @@
 // Tensor-core engine: int8 x int8 -> int32 matrix multiply on the 5th-generation tensor cores
 // (tcgen05.mma kind::i8, accumulators in tensor memory, operands staged by TMA), sm_100a only.
 //
-// One persistent CTA per SM; warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner),
-// warps 2..5 = epilogue (each reads its 32-lane quarter of TMEM with tcgen05.ld).  The accumulator
-// is double-buffered in TMEM so the epilogue of one tile overlaps the main loop of the next.
+// One persistent CTA (or CTA pair) per SM, 20 warps: warps 0..2 = TMA producers (each owns every
+// third stage of the ring), warp 3 = MMA issuer and TMEM owner, warps 4..19 = epilogue (four per
+// 32-lane quarter of TMEM, read with tcgen05.ld).  Up to eight accumulator buffers live in TMEM, so
+// the epilogues of finished tiles overlap the main loops of the following ones.
 //
 // The six operand mappings of the layer ops (Int8MatrixMultiply of Algorithm 1; implicit GEMM for
 // convolutions, Section 3.2) differ only in the TMA tensor maps, the per-k-block coordinates the
@@ -1078,6 +1079,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int ci0 = (blk % p.wg_nci) * 64, co0 = (blk / p.wg_nci) * 64;
         if (!mbar_wait(tfull0, use & 1u, &abort_flag, status)) { ok = false; break; }
         tc_fence_after();
+        unsigned pmx = 0;                       // largest partial-sum magnitude of this item
         for (int job = chunk_phase; job < 10; job += wpq) {
           const int pi = job >> 1, c0 = (job & 1) * 32;
           const int tap = 2 * pi + which;
@@ -1086,13 +1088,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (tap < 9) {
             int32_t *dst = acc + (long long)(co0 + c0) * p.gn + (long long)tap * p.Cn + ci0 + ci;
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
+            for (int j = 0; j < 32; ++j) {
+              pmx = max(pmx, (unsigned)abs(v[j]));
               if (v[j] != 0) atomicAdd(dst + (long long)j * p.gn, v[j]);
+            }
           }
         }
+        pmx = __reduce_max_sync(0xffffffffu, pmx);
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty0);
+        if (lane == 0) {
+          if (pmx) atomicMax(niti_split_max(hdr) + (p.splits > 1 ? item % p.splits : 0), pmx);
+          mbar_arrive(tempty0);
+        }
       }
       item_end = first_item;
     }
@@ -1177,12 +1185,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int *stg = reinterpret_cast<int *>(smem_raw + (smem_base - smem_u32(smem_raw)) + p.stg_off) +
                    (warp - EPI_WARP0) * (32 * 33);
         const long long row0 = out_row - lane;                 // output row of lane 0 of this warp
+        unsigned pmx = 0;                                      // largest partial-sum magnitude of this item
         for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
           int v[32];
           tc_ld32(tm_row + (unsigned)c, v);
           if (c < ncols_valid) {                               // (uniform across the warp)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = v[j];
+            for (int j = 0; j < 32; ++j) { stg[lane * 33 + j] = v[j]; pmx = max(pmx, (unsigned)abs(v[j])); }
             __syncwarp();
             const bool col_ok = c + lane < ncols_valid;
             int32_t *dcol = acc + row0 * p.gn + col0 + c + lane;
@@ -1195,9 +1204,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             __syncwarp();
           }
         }
+        pmx = __reduce_max_sync(0xffffffffu, pmx);
+        if (lane == 0 && pmx) atomicMax(niti_split_max(hdr) + split, pmx);
       } else if (p.epi_mode <= EPI_ATOMIC) {
         int32_t *dst = acc + out_row * p.gn + col0;
         const bool vec_ok = ((p.gn & 3) == 0) && ((col0 & 3) == 0);
+        unsigned pmx = 0;                                      // largest partial-sum magnitude of this item
         for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
           int v[32];
           tc_ld32(tm_row + (unsigned)c, v);
@@ -1205,7 +1217,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (p.epi_mode == EPI_ATOMIC) {
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                if (c + j < ncols_valid && v[j] != 0) atomicAdd(dst + c + j, v[j]);
+                if (c + j < ncols_valid && v[j] != 0) {
+                  pmx = max(pmx, (unsigned)abs(v[j]));
+                  atomicAdd(dst + c + j, v[j]);
+                }
             } else {
               if (vec_ok && c + 32 <= ncols_valid) {
 #pragma unroll
@@ -1228,6 +1243,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               }
             }
           }
+        }
+        if (p.epi_mode == EPI_ATOMIC) {
+          pmx = __reduce_max_sync(0xffffffffu, pmx);
+          if (lane == 0 && pmx) atomicMax(niti_split_max(hdr) + split, pmx);
         }
       } else {
         if (p.epi_mode == EPI_SPECULATE && use == (unsigned)egroup && egroup != 0) {
@@ -1299,6 +1318,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                              : "memory");
                 if (v_pub) { pub = v_pub; break; }
                 if (v_cnt >= quorum) {
+                  // (the 16-byte load is not promised to be one atomic snapshot: once the count is seen,
+                  // the maximum is read again, after a fence, so that it is at least as new as the count)
+                  __threadfence();
+                  v_max = *(volatile unsigned *)&hdr->est_max;
                   // the first tiles are a sample: scale their max by the growth expected from the sample
                   // to the whole tensor before taking the bit length (a wrong guess only costs the redo)
                   unsigned long long scaled = ((unsigned long long)v_max * p.spec_mul256) >> 8;
@@ -1578,6 +1601,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       __threadfence();
       const int b_true = niti_bitlen32(*(volatile unsigned *)&hdr->maxabs32);
       const int bpf = b_true > p.mbits ? b_true - p.mbits : 0;
+      // the shift every CTA rounded with came from the agreed maximum over ALL tiles, so it must be the
+      // true one; anything else means the agreement was broken and the stored int8 values are not exact
+      if (b_true != (int)(*(volatile unsigned *)&hdr->spec_b) - 1) atomicOr(status, NITI_DEV_INTERNAL);
       if (b_out) *b_out = b_true;
       if (s_out) {
         int sv = bpf + (s_a ? *s_a : 0) + (s_w ? *s_w : 0);
@@ -1859,6 +1885,10 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
           if (eff > best_eff + 0.02) { best_eff = eff; best_s = sp; }
         }
         p.splits = best_s;
+        // (a split covers at most NITI_SPLIT_MAX_K pixels: its partial sums cannot wrap)
+        if (p.splits < (p.kb_total + NITI_SPLIT_MAX_K / 128 - 1) / (NITI_SPLIT_MAX_K / 128))
+          p.splits = (p.kb_total + NITI_SPLIT_MAX_K / 128 - 1) / (NITI_SPLIT_MAX_K / 128);
+        if (p.splits > NITI_MAX_SPLITS) return false;
         p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
         p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
         p.items = blocks * p.splits;
@@ -1985,6 +2015,14 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
     }
     p.splits = best_s;
   }
+  {
+    // a contraction longer than NITI_SPLIT_MAX_K is always split, into pieces whose partial sums cannot
+    // wrap an int32; the epilogue records the largest partial sum of every piece (overflow detection)
+    const int max_kb = NITI_SPLIT_MAX_K / p.kdepth;
+    const int min_splits = (p.kb_total + max_kb - 1) / max_kb;
+    if (p.splits < min_splits) p.splits = min_splits;
+    if (p.splits > NITI_MAX_SPLITS) return false;
+  }
   p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
   p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
   // split contractions add their partial sums atomically: room for the epilogue warps' transpose
@@ -2035,8 +2073,6 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
 
 }  // namespace
 
-int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr);
-
 size_t niti_tc_scratch_bytes(const GemmProblem &) { return 0; }
 
 int niti_tc_timeout_probe(niti_ctx *ctx, cudaStream_t st) {
@@ -2051,7 +2087,7 @@ int niti_tc_timeout_probe(niti_ctx *ctx, cudaStream_t st) {
 // a second, short wave.
 template <int CTAS>
 static int tc_units(niti_ctx *ctx) {
-  static int cached = 0;
+  int &cached = ctx->tc_units[CTAS];
   if (cached) return cached;
   cached = ctx->sm_count / CTAS;
   if (CTAS == 2) {
@@ -2067,7 +2103,9 @@ static int tc_units(niti_ctx *ctx) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    (void)cudaFuncSetAttribute(tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 201 * 1024);
+    if (cudaFuncSetAttribute(tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 201 * 1024) == cudaSuccess &&
+        ctx->tc_attr_smem[2] < 201 * 1024)
+      ctx->tc_attr_smem[2] = 201 * 1024;
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, tc_gemm_kernel<2>, &cfg) == cudaSuccess && n > 0 && n < cached) cached = n;
     else (void)cudaGetLastError();
@@ -2080,7 +2118,7 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
                      int32_t *acc, WsHeader *hdr, const RoundSpec &r) {
   size_t smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + (size_t)p.b_res_bytes + 1024;
   if (p.stg_off > 0) smem = (size_t)p.stg_off + (size_t)EPI_WARPS * 32 * 33 * 4 + 1024;
-  static size_t attr_smem = CTAS == 2 ? 201 * 1024 : 0;
+  size_t &attr_smem = ctx->tc_attr_smem[CTAS];
   if (smem > attr_smem) {
     NITI_CUDA_TRY(ctx, cudaFuncSetAttribute(tc_gemm_kernel<CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     attr_smem = smem;
@@ -2214,7 +2252,7 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
       rc = niti_reduce(ctx, st, acc, g.gm * g.gn, NITI_REDUCE_SUM_I32);
       if (rc != NITI_OK) return rc;
     }
-    rc = niti_launch_maxabs(ctx, st, acc, g.gm * g.gn, hdr);
+    rc = niti_launch_maxabs(ctx, st, acc, g.gm * g.gn, hdr, p.splits);
     if (rc != NITI_OK || !dp || dp_sum) return rc;
     return niti_reduce(ctx, st, &hdr->maxabs32, 1, NITI_REDUCE_MAX_U32);
   }

@@ -11,6 +11,7 @@ from .workloads import (  # noqa: F401
     gemm_grad_operands,
     he_like_exponent,
     make_net_inputs,
+    make_step_batch,
     uniform_int8,
     GEMM_SWEEP_DIMS,
 )

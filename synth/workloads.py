@@ -153,6 +153,18 @@ def make_net_inputs(net: Net):
     return x, labels, weights
 
 
+def make_step_batch(net: Net, step: int):
+    """The mini-batch of training step ``step`` (x int8, labels int32).  Step 0 is the batch of
+    ``make_net_inputs``; every later step draws a fresh batch from ``PCG64([seed, step])``."""
+    if step == 0:
+        rng = np.random.Generator(np.random.PCG64(net.seed))
+    else:
+        rng = np.random.Generator(np.random.PCG64([net.seed, step]))
+    x = uniform_int8(rng, (net.batch,) + tuple(net.in_shape))
+    labels = rng.integers(0, net.n_classes, size=(net.batch,), dtype=np.int32)
+    return x, labels
+
+
 def gemm_operands(M: int, N: int, K: int, dist: str = "uniform", seed: int = 1):
     """Operands of the fused-GEMM sweep: a[M,K] and w[N,K] (both K-contiguous)."""
     rng = np.random.Generator(np.random.PCG64([seed, M, N, K, 0 if dist == "uniform" else 1]))

@@ -92,3 +92,13 @@ def test_the_data_parallel_reducer_combines_max_and_sum_over_two_gloo_ranks():
         assert m32 == 1007
         assert m64 == (1 << 40) + 3
         assert acc == [10, -12, 21, -2147483000]
+
+
+def test_launch_ranks_starts_one_process_per_rank_on_localhost(tmp_path):
+    """`bench.py --gpus N` without an external launcher starts its N ranks through this helper."""
+    from paper_2009_13108_b200.dist_util import launch_ranks
+    worker = os.path.join(os.path.dirname(os.path.abspath(__file__)), "_spawn_worker.py")
+    rc = launch_ranks([worker, str(tmp_path)], 2, timeout=300)
+    assert rc == 0
+    rows = sorted(open(os.path.join(tmp_path, "rank%d.txt" % r)).read().split() for r in range(2))
+    assert rows == [["0", "2", "0", "127.0.0.1", "3"], ["1", "2", "1", "127.0.0.1", "3"]]

@@ -3,6 +3,8 @@
 Sizes are chosen so the oracle finishes in seconds while the tensor-core engine still sees
 several tiles, ragged tails, every operand layout (K-major / MN-major, 32/64/128-byte swizzle),
 split contractions and the fallback engine."""
+from ctypes import c_uint32 as C_uint32
+
 import numpy as np
 import pytest
 import torch
@@ -329,6 +331,90 @@ def test_general_taps_and_padding_use_the_fallback(niti, oref):
         wg, _ = oref.conv_wgrad(x, e, (5, 5), pad, 5)
         _eq(niti.conv_wgrad(_T(niti, x), _T(niti, e), (5, 5), pad=pad)[0], wg)
     niti.check()
+
+
+@pytest.mark.parametrize("engine", [0, 2, 3])
+@pytest.mark.parametrize("R,pad", [(5, 2), (7, 3), (1, 0)])
+@pytest.mark.parametrize("B,H,W,Ci,Co", [(2, 16, 16, 32, 64), (2, 12, 20, 64, 128), (3, 8, 16, 128, 32),
+                                         (1, 24, 40, 64, 64)])
+def test_large_and_pointwise_filters_on_the_tensor_cores(niti, oref, B, H, W, Ci, Co, R, pad, engine):
+    """5x5, 7x7 (the paper's LeNet / AlexNet filter sizes, Section 4) and 1x1 convolutions with "same"
+    geometry and at least 32 channels run on the tcgen05 kernel: forward, error and weight gradient
+    against the oracle, and the tensor-core launch counter must move for each of them."""
+    rng = np.random.default_rng(B + H * 3 + W * 5 + Ci * 7 + Co * 11 + R)
+    x, w, e = _i8(rng, (B, H, W, Ci)), _i8(rng, (Co, R, R, Ci)), _i8(rng, (B, H, W, Co))
+    xm = np.maximum(x, 0)
+    niti.set_engine(engine)
+    try:
+        n0 = niti.tc_launch_count()
+        wy, s, b = oref.conv_fwd(x, -7, w, -9, pad, True)
+        y, s_y, b_y = niti.conv_fwd(_T(niti, x), niti.scalar(-7), _T(niti, w), niti.scalar(-9), pad=pad, relu=True)
+        _eq(y, wy)
+        assert (int(s_y), int(b_y)) == (s, b)
+        n1 = niti.tc_launch_count()
+        wd, bd = oref.conv_dgrad(e, w, (H, W), pad, xm)
+        ep, b_e = niti.conv_dgrad(_T(niti, e), _T(niti, w), (H, W), relu_mask_src=_T(niti, xm), pad=pad)
+        _eq(ep, wd)
+        assert int(b_e) == bd
+        n2 = niti.tc_launch_count()
+        wg, bg = oref.conv_wgrad(x, e, (R, R), pad, 5)
+        g, b_g = niti.conv_wgrad(_T(niti, x), _T(niti, e), (R, R), pad=pad)
+        _eq(g, wg)
+        assert int(b_g) == bg
+        n3 = niti.tc_launch_count()
+        if engine != 3:       # (3 = paired CTAs only: a test switch that falls back where pairs do not apply)
+            assert n1 > n0 and n2 > n1 and n3 > n2, "a multiply fell back to the CUDA-core engine"
+    finally:
+        niti.set_engine(0)
+    niti.check()
+
+
+@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("Ci,Co", [(64, 64), (32, 128)])
+def test_accumulator_range_is_flagged_where_the_oracle_reports_an_overflow(niti, oref, Ci, Co, engine):
+    """int32 accumulators (Section 3.2): the weight gradient contracts over batch x pixels.  With
+    constant +127 operands the centre tap sums pixels * 16129: 120000 pixels stay below 2^31 (result
+    equal to the oracle's, no flag), 140800 pixels exceed it (the int64 oracle reports the overflow
+    and the device status word must carry NITI_DEV_ACC_RANGE)."""
+    from oracle.ref import ERR_OVERFLOW, OracleError
+    from paper_2009_13108_b200.api import NitiError
+    niti.set_engine(engine)
+    try:
+        for H, overflow in ((300, False), (352, True)):
+            x = np.full((1, H, 400, Ci), 127, np.int8)
+            e = np.full((1, H, 400, Co), 127, np.int8)
+            g, b_g = niti.conv_wgrad(_T(niti, x), _T(niti, e))
+            if overflow:
+                with pytest.raises(OracleError) as oerr:
+                    oref.conv_wgrad(x, e, (3, 3), 1, 5)
+                assert oerr.value.code == ERR_OVERFLOW
+                with pytest.raises(NitiError):
+                    niti.check()
+                st = C_uint32()
+                assert niti.lib.niti_check(niti.h, niti._stream(), st) == 0     # the word was cleared
+            else:
+                wg, bg = oref.conv_wgrad(x, e, (3, 3), 1, 5)
+                _eq(g, wg)
+                assert int(b_g) == bg
+                assert niti.check() == 0
+        # fully connected weight gradient: contraction over the batch
+        for M, overflow in ((120000, False), (140000, True)):
+            a = np.full((M, 64), 127, np.int8)
+            e = np.full((M, 32), 127, np.int8)
+            w = np.zeros((32, 64), np.int8)
+            _, g, _, b_g = niti.linear_bwd(_T(niti, a), _T(niti, e), _T(niti, w), need_e_prev=False)
+            if overflow:
+                with pytest.raises(OracleError):
+                    oref.linear_bwd(a, e, w, False)
+                with pytest.raises(NitiError) as gerr:
+                    niti.check()
+                assert "0x10" in str(gerr.value)
+            else:
+                _, wg, _, bg = oref.linear_bwd(a, e, w, False)
+                _eq(g, wg)
+                assert int(b_g) == bg and niti.check() == 0
+    finally:
+        niti.set_engine(0)
 
 
 def test_saturation_and_zero_tensor(niti, oref):

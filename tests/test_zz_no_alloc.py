@@ -1,7 +1,8 @@
 """niti_int_xent_noalloc -- the entry point for callers that may not allocate device memory (no
 context, no workspace: its scratch is a fixed array inside the library).  It must give exactly
 the bytes of niti_int_xent, on two calls in a row (the shared array keeps the first call's
-contents), and refuse inputs beyond its fixed capacity.  Collected last on purpose."""
+contents), and refuse inputs beyond its fixed capacity; the same outputs are also compared with the
+CPU oracle directly.  Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
@@ -15,7 +16,7 @@ def _case(rng, B, N, dev):
     return a, labels
 
 
-def test_no_alloc_entry_point_matches_the_regular_one():
+def test_no_alloc_entry_point_matches_the_regular_one(oref):
     from paper_2009_13108_b200 import Niti
     niti = Niti(0)
     dev = niti.device
@@ -37,6 +38,10 @@ def test_no_alloc_entry_point_matches_the_regular_one():
         assert torch.cuda.memory_allocated(dev) == before
         assert torch.equal(e, want_e)                       # bit-exact: all of this path is integer
         assert int(b_e) == int(want_b) and int(n_correct) == int(want_nc)
+        # and against the CPU oracle (Section 3.5), not only against the other CUDA entry point
+        ref_e, ref_b, ref_nc = oref.int_xent(a.cpu().numpy(), s_a, labels.cpu().numpy(), mode)
+        assert np.array_equal(e.cpu().numpy(), ref_e)
+        assert (int(b_e), int(n_correct)) == (ref_b, ref_nc)
     # optional outputs may be omitted
     a, labels = _case(rng, 8, 16, dev)
     e = torch.empty((8, 16), dtype=torch.int8, device=dev)
