@@ -67,7 +67,7 @@ extern "C" {
 /* op ids for niti_workspace_bytes(); dims as listed */
 #define NITI_OP_LINEAR_FWD 0  /* dims = {M, N, K}                 */
 #define NITI_OP_LINEAR_BWD 1  /* dims = {M, N, K}                 */
-#define NITI_OP_CONV_FWD 2    /* dims = {B, H, W, Cin, Cout, R, S, pad} */
+#define NITI_OP_CONV_FWD 2    /* dims = {B, H, W, Cin, Cout, R, S, pad} or {..., pad, stride} */
 #define NITI_OP_CONV_DGRAD 3  /* same                              */
 #define NITI_OP_CONV_WGRAD 4  /* same                              */
 #define NITI_OP_INT_XENT 5    /* dims = {B, N}                    */
@@ -86,8 +86,10 @@ extern "C" {
 typedef struct niti_ctx niti_ctx;
 
 /* Creates a context on CUDA device `device` (the device must be sm_100).
- * Allocates a few bytes of device memory for the status word.  The caller
- * destroys it with niti_destroy().  Not thread-safe per context. */
+ * Allocates 33 KB of device memory (status words; a table in which the
+ * speculative epilogue remembers, per call site, how far its last bit-width
+ * estimate was off).  The caller destroys it with niti_destroy().  Not
+ * thread-safe per context. */
 int niti_create(niti_ctx **out, int device);
 int niti_destroy(niti_ctx *ctx);
 
@@ -122,8 +124,11 @@ uint64_t niti_tc_pair_launch_count(niti_ctx *ctx);
 
 /* The fused epilogue of the tensor-core kernel rounds with a bit-width guessed from the first
  * tile of every CTA and recomputes the multiply when the whole tensor turns out to need a larger
- * shift (results are exact either way).  Returns how many such recomputations this context has
- * run so far (synchronises `stream`; -1 on error). */
+ * shift (results are exact either way).  A call that passes a bit-width scalar (b_out / b_e / b_g)
+ * is recognised by that scalar's address when it comes again (the same layer in the next training
+ * step): the estimate is then corrected by what it missed last time, which removes the recomputations
+ * of tensors whose extremes the sample systematically misses.  Returns how many recomputations this
+ * context has run so far (synchronises `stream`; -1 on error). */
 int64_t niti_redo_count(niti_ctx *ctx, void *stream);
 
 /* Self-test of the failure detection: every wait inside the kernels is bounded; this enqueues a
@@ -166,7 +171,7 @@ int niti_linear_bwd(niti_ctx *ctx, void *stream, const int8_t *a, const int8_t *
                     size_t ws_bytes);
 
 /* Convolution forward as an implicit matrix multiply (Section 3.2), stride 1,
- * zero padding `pad`, R x S taps:
+ * zero padding `pad`, R x S taps (any R, S, pad; 3 x 3 / pad 1 has tuned modes):
  *   acc[b][i][j][co] = sum_{r,s,ci} x[b][i+r-pad][j+s-pad][ci] * w[co][r][s][ci]
  * followed by the same bit-width / shift / round / exponent rule as
  * niti_linear_fwd.  x [B][H][W][Cin], y [B][H+2pad-R+1][W+2pad-S+1][Cout]. */
@@ -190,6 +195,30 @@ int niti_conv_dgrad(niti_ctx *ctx, void *stream, const int8_t *e, const int8_t *
 int niti_conv_wgrad(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
                     int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
                     int m_u, int round_mode, void *ws, size_t ws_bytes);
+
+/* The same three convolution ops with a stride (the first layer of the paper's
+ * AlexNet is 11 x 11 with stride 4, Section 4):
+ *   acc[b][i][j][co] = sum_{r,s,ci} x[b][i*stride+r-pad][j*stride+s-pad][ci] * w[co][r][s][ci]
+ * with output size Ho = (H + 2 pad - R) / stride + 1 (integer division), Wo
+ * likewise; the error and weight-gradient calls are its exact transposes with
+ * respect to x and w.  H, W are always the INPUT sizes of the forward
+ * convolution; y / e have the [B][Ho][Wo][Cout] shape.  Workspace: the same op
+ * ids with the stride as a ninth entry of dims.  stride = 1 is the call
+ * without the suffix.  Forward and weight gradient of strided layers with at
+ * least 32 channels on both sides run on the tensor cores (the stride becomes
+ * the element stride of the operand copies); the error of a strided layer and
+ * layers with other channel counts run on the CUDA-core engine. */
+int niti_conv_fwd_strided(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x,
+                          const int8_t *w, const int32_t *s_w, int8_t *y, int32_t *s_y, int32_t *b_y, int B,
+                          int H, int W, int Cin, int Cout, int R, int S, int pad, int stride, int relu,
+                          int round_mode, void *ws, size_t ws_bytes);
+int niti_conv_dgrad_strided(niti_ctx *ctx, void *stream, const int8_t *e, const int8_t *w, int8_t *e_prev,
+                            const int8_t *relu_mask_src, int32_t *b_e, int B, int H, int W, int Cin,
+                            int Cout, int R, int S, int pad, int stride, int round_mode, void *ws,
+                            size_t ws_bytes);
+int niti_conv_wgrad_strided(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
+                            int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
+                            int stride, int m_u, int round_mode, void *ws, size_t ws_bytes);
 
 /* Weight gradient fused with the weight update (Section 3.3: the gradient is
  * rounded to m_u bits "and fused with the weight update"; Algorithm 1, last two

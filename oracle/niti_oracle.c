@@ -176,15 +176,20 @@ void niti_ref_fc_wgrad_acc(const int8_t *a, const int8_t *e, int64_t *acc, int64
 }
 
 /* ------------------------------------------------------------------------- */
-/* Convolution, stride 1, zero padding `pad`, R x S taps, NHWC / [Co][R][S][Ci]*/
-/* Direct loops over the definition (Section 3.2 reduces it to a matrix       */
-/* multiply; the oracle deliberately does not).                               */
-/*   y[b][i][j][co] = sum_{r,s,ci} x[b][i+r-pad][j+s-pad][ci] * w[co][r][s][ci]*/
-/* Output spatial size: Ho = H + 2*pad - R + 1, Wo = W + 2*pad - S + 1.       */
+/* Convolution with stride `stride`, zero padding `pad`, R x S taps, NHWC /    */
+/* [Co][R][S][Ci].  Direct loops over the definition (Section 3.2 reduces it   */
+/* to a matrix multiply; the oracle deliberately does not).                    */
+/*   y[b][i][j][co] = sum_{r,s,ci} x[b][i*stride+r-pad][j*stride+s-pad][ci]    */
+/*                                 * w[co][r][s][ci]                           */
+/* Output spatial size: Ho = (H + 2*pad - R) / stride + 1 (integer division),  */
+/* Wo likewise.  The paper's measured layer has stride 1 (Section 5); its      */
+/* networks also use stride 4 (AlexNet's first layer, Section 4).  The         */
+/* functions without the _s suffix are the stride-1 case.                      */
 /* ------------------------------------------------------------------------- */
-void niti_ref_conv_fwd_acc(const int8_t *x, const int8_t *w, int64_t *acc, int64_t B, int64_t H,
-                           int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S, int64_t pad) {
-  int64_t Ho = H + 2 * pad - R + 1, Wo = W + 2 * pad - S + 1;
+void niti_ref_conv_fwd_acc_s(const int8_t *x, const int8_t *w, int64_t *acc, int64_t B, int64_t H,
+                             int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S, int64_t pad,
+                             int64_t stride) {
+  int64_t Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - S) / stride + 1;
 #pragma omp parallel for collapse(3) schedule(static)
   for (int64_t b = 0; b < B; ++b)
     for (int64_t i = 0; i < Ho; ++i)
@@ -193,7 +198,7 @@ void niti_ref_conv_fwd_acc(const int8_t *x, const int8_t *w, int64_t *acc, int64
           int64_t s = 0;
           for (int64_t r = 0; r < R; ++r)
             for (int64_t t = 0; t < S; ++t) {
-              int64_t ii = i + r - pad, jj = j + t - pad;
+              int64_t ii = i * stride + r - pad, jj = j * stride + t - pad;
               if (ii < 0 || ii >= H || jj < 0 || jj >= W) continue;
               for (int64_t ci = 0; ci < Ci; ++ci)
                 s += (int64_t)x[((b * H + ii) * W + jj) * Ci + ci] *
@@ -204,12 +209,14 @@ void niti_ref_conv_fwd_acc(const int8_t *x, const int8_t *w, int64_t *acc, int64
 }
 
 /* Error back-propagation through the convolution: the exact transpose of the */
-/* forward map with respect to x.                                              */
-/*   ex[b][ii][jj][ci] = sum_{r,s,co} e[b][ii-r+pad][jj-s+pad][co]*w[co][r][s][ci] */
-void niti_ref_conv_dgrad_acc(const int8_t *e, const int8_t *w, int64_t *acc, int64_t B, int64_t H,
-                             int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S,
-                             int64_t pad) {
-  int64_t Ho = H + 2 * pad - R + 1, Wo = W + 2 * pad - S + 1;
+/* forward map with respect to x:                                              */
+/*   ex[b][ii][jj][ci] = sum over (r, s, co) and the output pixels (i, j) with */
+/*   i*stride + r - pad == ii, j*stride + s - pad == jj of                     */
+/*   e[b][i][j][co] * w[co][r][s][ci]                                          */
+void niti_ref_conv_dgrad_acc_s(const int8_t *e, const int8_t *w, int64_t *acc, int64_t B, int64_t H,
+                               int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S, int64_t pad,
+                               int64_t stride) {
+  int64_t Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - S) / stride + 1;
 #pragma omp parallel for collapse(3) schedule(static)
   for (int64_t b = 0; b < B; ++b)
     for (int64_t ii = 0; ii < H; ++ii)
@@ -218,8 +225,10 @@ void niti_ref_conv_dgrad_acc(const int8_t *e, const int8_t *w, int64_t *acc, int
           int64_t s = 0;
           for (int64_t r = 0; r < R; ++r)
             for (int64_t t = 0; t < S; ++t) {
-              int64_t i = ii - r + pad, j = jj - t + pad;
-              if (i < 0 || i >= Ho || j < 0 || j >= Wo) continue;
+              int64_t ti = ii - r + pad, tj = jj - t + pad;
+              if (ti < 0 || tj < 0 || ti % stride || tj % stride) continue;
+              int64_t i = ti / stride, j = tj / stride;
+              if (i >= Ho || j >= Wo) continue;
               for (int64_t co = 0; co < Co; ++co)
                 s += (int64_t)e[((b * Ho + i) * Wo + j) * Co + co] *
                      (int64_t)w[((co * R + r) * S + t) * Ci + ci];
@@ -229,30 +238,53 @@ void niti_ref_conv_dgrad_acc(const int8_t *e, const int8_t *w, int64_t *acc, int
 }
 
 /* Weight gradient: the exact transpose of the forward map with respect to w. */
-/*   g[co][r][s][ci] = sum_{b,i,j} e[b][i][j][co] * x[b][i+r-pad][j+s-pad][ci] */
+/*   g[co][r][s][ci] = sum_{b,i,j} e[b][i][j][co]                              */
+/*                                 * x[b][i*stride+r-pad][j*stride+s-pad][ci]  */
+/* Loop nest: one output channel per OpenMP iteration; inside it the pixels    */
+/* are the outer loops and (r, s, ci) the inner ones, so that x and e are read */
+/* front to back once per output channel (with the pixel loops innermost every */
+/* single output element streamed both tensors in full, which at 224 x 224,    */
+/* batch 64 does not finish).  Each output is still the plain sum above; the   */
+/* order of integer additions does not change it.                              */
+void niti_ref_conv_wgrad_acc_s(const int8_t *x, const int8_t *e, int64_t *acc, int64_t B, int64_t H,
+                               int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S, int64_t pad,
+                               int64_t stride) {
+  int64_t Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - S) / stride + 1;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t co = 0; co < Co; ++co) {
+    int64_t *g = acc + co * R * S * Ci;
+    for (int64_t q = 0; q < R * S * Ci; ++q) g[q] = 0;
+    for (int64_t b = 0; b < B; ++b)
+      for (int64_t i = 0; i < Ho; ++i)
+        for (int64_t j = 0; j < Wo; ++j) {
+          int64_t ev = (int64_t)e[((b * Ho + i) * Wo + j) * Co + co];
+          for (int64_t r = 0; r < R; ++r) {
+            int64_t ii = i * stride + r - pad;
+            if (ii < 0 || ii >= H) continue;
+            for (int64_t t = 0; t < S; ++t) {
+              int64_t jj = j * stride + t - pad;
+              if (jj < 0 || jj >= W) continue;
+              for (int64_t ci = 0; ci < Ci; ++ci)
+                g[(r * S + t) * Ci + ci] += ev * (int64_t)x[((b * H + ii) * W + jj) * Ci + ci];
+            }
+          }
+        }
+  }
+}
+
+void niti_ref_conv_fwd_acc(const int8_t *x, const int8_t *w, int64_t *acc, int64_t B, int64_t H,
+                           int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S, int64_t pad) {
+  niti_ref_conv_fwd_acc_s(x, w, acc, B, H, W, Ci, Co, R, S, pad, 1);
+}
+void niti_ref_conv_dgrad_acc(const int8_t *e, const int8_t *w, int64_t *acc, int64_t B, int64_t H,
+                             int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S,
+                             int64_t pad) {
+  niti_ref_conv_dgrad_acc_s(e, w, acc, B, H, W, Ci, Co, R, S, pad, 1);
+}
 void niti_ref_conv_wgrad_acc(const int8_t *x, const int8_t *e, int64_t *acc, int64_t B, int64_t H,
                              int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S,
                              int64_t pad) {
-  int64_t Ho = H + 2 * pad - R + 1, Wo = W + 2 * pad - S + 1;
-#pragma omp parallel for collapse(3) schedule(static)
-  for (int64_t co = 0; co < Co; ++co)
-    for (int64_t r = 0; r < R; ++r)
-      for (int64_t t = 0; t < S; ++t)
-        for (int64_t ci = 0; ci < Ci; ++ci) {
-          int64_t s = 0;
-          for (int64_t b = 0; b < B; ++b)
-            for (int64_t i = 0; i < Ho; ++i) {
-              int64_t ii = i + r - pad;
-              if (ii < 0 || ii >= H) continue;
-              for (int64_t j = 0; j < Wo; ++j) {
-                int64_t jj = j + t - pad;
-                if (jj < 0 || jj >= W) continue;
-                s += (int64_t)e[((b * Ho + i) * Wo + j) * Co + co] *
-                     (int64_t)x[((b * H + ii) * W + jj) * Ci + ci];
-              }
-            }
-          acc[((co * R + r) * S + t) * Ci + ci] = s;
-        }
+  niti_ref_conv_wgrad_acc_s(x, e, acc, B, H, W, Ci, Co, R, S, pad, 1);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -439,14 +471,15 @@ int niti_ref_linear_bwd(const int8_t *a, const int8_t *e, const int8_t *w, int8_
   return rc;
 }
 
-int niti_ref_conv_fwd(const int8_t *x, int32_t s_x, const int8_t *w, int32_t s_w, int8_t *y,
-                      int32_t *s_y, int32_t *b_y, int64_t B, int64_t H, int64_t W, int64_t Ci,
-                      int64_t Co, int64_t R, int64_t S, int64_t pad, int relu, int round_mode) {
-  int64_t Ho = H + 2 * pad - R + 1, Wo = W + 2 * pad - S + 1;
+int niti_ref_conv_fwd_s(const int8_t *x, int32_t s_x, const int8_t *w, int32_t s_w, int8_t *y,
+                        int32_t *s_y, int32_t *b_y, int64_t B, int64_t H, int64_t W, int64_t Ci,
+                        int64_t Co, int64_t R, int64_t S, int64_t pad, int64_t stride, int relu,
+                        int round_mode) {
+  int64_t Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - S) / stride + 1;
   int64_t n = B * Ho * Wo * Co;
   int64_t *acc = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
   if (!acc) return NITI_REF_ERR_ARG;
-  niti_ref_conv_fwd_acc(x, w, acc, B, H, W, Ci, Co, R, S, pad);
+  niti_ref_conv_fwd_acc_s(x, w, acc, B, H, W, Ci, Co, R, S, pad, stride);
   int32_t bp = 0;
   int rc = finish(acc, n, 7, round_mode, y, b_y, &bp);
   if (relu) niti_ref_relu_fwd(y, y, n);
@@ -454,26 +487,44 @@ int niti_ref_conv_fwd(const int8_t *x, int32_t s_x, const int8_t *w, int32_t s_w
   return rc;
 }
 
-int niti_ref_conv_dgrad(const int8_t *e, const int8_t *w, int8_t *e_prev, const int8_t *mask,
-                        int32_t *b_e, int64_t B, int64_t H, int64_t W, int64_t Ci, int64_t Co,
-                        int64_t R, int64_t S, int64_t pad, int round_mode) {
+int niti_ref_conv_fwd(const int8_t *x, int32_t s_x, const int8_t *w, int32_t s_w, int8_t *y,
+                      int32_t *s_y, int32_t *b_y, int64_t B, int64_t H, int64_t W, int64_t Ci,
+                      int64_t Co, int64_t R, int64_t S, int64_t pad, int relu, int round_mode) {
+  return niti_ref_conv_fwd_s(x, s_x, w, s_w, y, s_y, b_y, B, H, W, Ci, Co, R, S, pad, 1, relu, round_mode);
+}
+
+int niti_ref_conv_dgrad_s(const int8_t *e, const int8_t *w, int8_t *e_prev, const int8_t *mask,
+                          int32_t *b_e, int64_t B, int64_t H, int64_t W, int64_t Ci, int64_t Co,
+                          int64_t R, int64_t S, int64_t pad, int64_t stride, int round_mode) {
   int64_t n = B * H * W * Ci;
   int64_t *acc = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
   if (!acc) return NITI_REF_ERR_ARG;
-  niti_ref_conv_dgrad_acc(e, w, acc, B, H, W, Ci, Co, R, S, pad);
+  niti_ref_conv_dgrad_acc_s(e, w, acc, B, H, W, Ci, Co, R, S, pad, stride);
   int rc = finish(acc, n, 7, round_mode, e_prev, b_e, NULL);
   if (mask) niti_ref_relu_bwd(mask, e_prev, e_prev, n);
   return rc;
 }
 
-int niti_ref_conv_wgrad(const int8_t *x, const int8_t *e, int8_t *g, int32_t *b_g, int64_t B,
-                        int64_t H, int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S,
-                        int64_t pad, int m_u, int round_mode) {
+int niti_ref_conv_dgrad(const int8_t *e, const int8_t *w, int8_t *e_prev, const int8_t *mask,
+                        int32_t *b_e, int64_t B, int64_t H, int64_t W, int64_t Ci, int64_t Co,
+                        int64_t R, int64_t S, int64_t pad, int round_mode) {
+  return niti_ref_conv_dgrad_s(e, w, e_prev, mask, b_e, B, H, W, Ci, Co, R, S, pad, 1, round_mode);
+}
+
+int niti_ref_conv_wgrad_s(const int8_t *x, const int8_t *e, int8_t *g, int32_t *b_g, int64_t B,
+                          int64_t H, int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S,
+                          int64_t pad, int64_t stride, int m_u, int round_mode) {
   int64_t n = Co * R * S * Ci;
   int64_t *acc = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
   if (!acc) return NITI_REF_ERR_ARG;
-  niti_ref_conv_wgrad_acc(x, e, acc, B, H, W, Ci, Co, R, S, pad);
+  niti_ref_conv_wgrad_acc_s(x, e, acc, B, H, W, Ci, Co, R, S, pad, stride);
   return finish(acc, n, m_u, round_mode, g, b_g, NULL);
+}
+
+int niti_ref_conv_wgrad(const int8_t *x, const int8_t *e, int8_t *g, int32_t *b_g, int64_t B,
+                        int64_t H, int64_t W, int64_t Ci, int64_t Co, int64_t R, int64_t S,
+                        int64_t pad, int m_u, int round_mode) {
+  return niti_ref_conv_wgrad_s(x, e, g, b_g, B, H, W, Ci, Co, R, S, pad, 1, m_u, round_mode);
 }
 
 int niti_ref_int_xent(const int8_t *a, int32_t s_a, const int32_t *labels, int8_t *e, int32_t *b_e,

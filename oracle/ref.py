@@ -69,9 +69,9 @@ def _declare(L):
     for f in (L.niti_ref_fc_fwd_acc, L.niti_ref_fc_dgrad_acc, L.niti_ref_fc_wgrad_acc):
         f.restype = None
         f.argtypes = [_i8p, _i8p, _i64p, _i64, _i64, _i64]
-    for f in (L.niti_ref_conv_fwd_acc, L.niti_ref_conv_dgrad_acc, L.niti_ref_conv_wgrad_acc):
+    for f in (L.niti_ref_conv_fwd_acc_s, L.niti_ref_conv_dgrad_acc_s, L.niti_ref_conv_wgrad_acc_s):
         f.restype = None
-        f.argtypes = [_i8p, _i8p, _i64p] + [_i64] * 8
+        f.argtypes = [_i8p, _i8p, _i64p] + [_i64] * 9
     L.niti_ref_xent_acc.restype = _int
     L.niti_ref_xent_acc.argtypes = [_i8p, _i32, _i32p, _i64p, _i64, _i64]
     L.niti_ref_count_correct.restype = _i32
@@ -92,13 +92,13 @@ def _declare(L):
     L.niti_ref_linear_bwd.restype = _int
     L.niti_ref_linear_bwd.argtypes = [_i8p, _i8p, _i8p, _i8p, _i8p, _i8p, _i32p, _i32p, _i64, _i64,
                                       _i64, _int, _int]
-    L.niti_ref_conv_fwd.restype = _int
-    L.niti_ref_conv_fwd.argtypes = [_i8p, _i32, _i8p, _i32, _i8p, _i32p, _i32p] + [_i64] * 8 + \
+    L.niti_ref_conv_fwd_s.restype = _int
+    L.niti_ref_conv_fwd_s.argtypes = [_i8p, _i32, _i8p, _i32, _i8p, _i32p, _i32p] + [_i64] * 9 + \
         [_int, _int]
-    L.niti_ref_conv_dgrad.restype = _int
-    L.niti_ref_conv_dgrad.argtypes = [_i8p, _i8p, _i8p, _i8p, _i32p] + [_i64] * 8 + [_int]
-    L.niti_ref_conv_wgrad.restype = _int
-    L.niti_ref_conv_wgrad.argtypes = [_i8p, _i8p, _i8p, _i32p] + [_i64] * 8 + [_int, _int]
+    L.niti_ref_conv_dgrad_s.restype = _int
+    L.niti_ref_conv_dgrad_s.argtypes = [_i8p, _i8p, _i8p, _i8p, _i32p] + [_i64] * 9 + [_int]
+    L.niti_ref_conv_wgrad_s.restype = _int
+    L.niti_ref_conv_wgrad_s.argtypes = [_i8p, _i8p, _i8p, _i32p] + [_i64] * 9 + [_int, _int]
     L.niti_ref_int_xent.restype = _int
     L.niti_ref_int_xent.argtypes = [_i8p, _i32, _i32p, _i8p, _i32p, _i32p, _i64, _i64, _int]
 
@@ -192,32 +192,40 @@ def fc_wgrad_acc(a, e):
     return acc
 
 
-def conv_fwd_acc(x, w, pad=1):
+def conv_out_hw(H, W, R, S, pad, stride=1):
+    """Output size of a convolution: (H + 2 pad - R) // stride + 1."""
+    return (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
+
+
+def conv_fwd_acc(x, w, pad=1, stride=1):
     x, w = _c8(x), _c8(w)
     B, H, W, Ci = x.shape
     Co, R, S, _ = w.shape
-    acc = np.empty((B, H + 2 * pad - R + 1, W + 2 * pad - S + 1, Co), np.int64)
-    lib().niti_ref_conv_fwd_acc(_p8(x), _p8(w), _p64(acc), B, H, W, Ci, Co, R, S, pad)
+    Ho, Wo = conv_out_hw(H, W, R, S, pad, stride)
+    acc = np.empty((B, Ho, Wo, Co), np.int64)
+    lib().niti_ref_conv_fwd_acc_s(_p8(x), _p8(w), _p64(acc), B, H, W, Ci, Co, R, S, pad, stride)
     return acc
 
 
-def conv_dgrad_acc(e, w, in_hw, pad=1):
+def conv_dgrad_acc(e, w, in_hw, pad=1, stride=1):
     e, w = _c8(e), _c8(w)
     B = e.shape[0]
     H, W = in_hw
     Co, R, S, Ci = w.shape
+    assert e.shape[1:3] == conv_out_hw(H, W, R, S, pad, stride)
     acc = np.empty((B, H, W, Ci), np.int64)
-    lib().niti_ref_conv_dgrad_acc(_p8(e), _p8(w), _p64(acc), B, H, W, Ci, Co, R, S, pad)
+    lib().niti_ref_conv_dgrad_acc_s(_p8(e), _p8(w), _p64(acc), B, H, W, Ci, Co, R, S, pad, stride)
     return acc
 
 
-def conv_wgrad_acc(x, e, rs=(3, 3), pad=1):
+def conv_wgrad_acc(x, e, rs=(3, 3), pad=1, stride=1):
     x, e = _c8(x), _c8(e)
     B, H, W, Ci = x.shape
     Co = e.shape[3]
     R, S = rs
+    assert e.shape[1:3] == conv_out_hw(H, W, R, S, pad, stride)
     acc = np.empty((Co, R, S, Ci), np.int64)
-    lib().niti_ref_conv_wgrad_acc(_p8(x), _p8(e), _p64(acc), B, H, W, Ci, Co, R, S, pad)
+    lib().niti_ref_conv_wgrad_acc_s(_p8(x), _p8(e), _p64(acc), B, H, W, Ci, Co, R, S, pad, stride)
     return acc
 
 
@@ -302,44 +310,47 @@ def linear_bwd(a, e, w, need_e_prev=True, mask=None, m_u=5, round_mode=ROUND_PSR
     return e_prev, g, int(be[0]), int(bg[0])
 
 
-def conv_fwd(x, s_x, w, s_w, pad=1, relu=False, round_mode=ROUND_PSR, allow_overflow=False):
+def conv_fwd(x, s_x, w, s_w, pad=1, relu=False, round_mode=ROUND_PSR, allow_overflow=False, stride=1):
     """Returns (y int8 NHWC, s_y, b)."""
     x, w = _c8(x), _c8(w)
     B, H, W, Ci = x.shape
     Co, R, S, _ = w.shape
-    y = np.empty((B, H + 2 * pad - R + 1, W + 2 * pad - S + 1, Co), np.int8)
+    Ho, Wo = conv_out_hw(H, W, R, S, pad, stride)
+    y = np.empty((B, Ho, Wo, Co), np.int8)
     s = np.zeros(1, np.int32)
     b = np.zeros(1, np.int32)
-    _check(lib().niti_ref_conv_fwd(_p8(x), s_x, _p8(w), s_w, _p8(y), _p32(s), _p32(b), B, H, W, Ci,
-                                   Co, R, S, pad, int(relu), round_mode), allow_overflow)
+    _check(lib().niti_ref_conv_fwd_s(_p8(x), s_x, _p8(w), s_w, _p8(y), _p32(s), _p32(b), B, H, W, Ci,
+                                     Co, R, S, pad, stride, int(relu), round_mode), allow_overflow)
     return y, int(s[0]), int(b[0])
 
 
-def conv_dgrad(e, w, in_hw, pad=1, mask=None, round_mode=ROUND_PSR, allow_overflow=False):
+def conv_dgrad(e, w, in_hw, pad=1, mask=None, round_mode=ROUND_PSR, allow_overflow=False, stride=1):
     """Returns (e_prev int8 [B,H,W,Ci], b)."""
     e, w = _c8(e), _c8(w)
     B = e.shape[0]
     H, W = in_hw
     Co, R, S, Ci = w.shape
+    assert e.shape[1:3] == conv_out_hw(H, W, R, S, pad, stride)
     e_prev = np.empty((B, H, W, Ci), np.int8)
     if mask is not None:
         mask = _c8(mask)
     b = np.zeros(1, np.int32)
-    _check(lib().niti_ref_conv_dgrad(_p8(e), _p8(w), _p8(e_prev), _p8(mask), _p32(b), B, H, W, Ci,
-                                     Co, R, S, pad, round_mode), allow_overflow)
+    _check(lib().niti_ref_conv_dgrad_s(_p8(e), _p8(w), _p8(e_prev), _p8(mask), _p32(b), B, H, W, Ci,
+                                       Co, R, S, pad, stride, round_mode), allow_overflow)
     return e_prev, int(b[0])
 
 
-def conv_wgrad(x, e, rs=(3, 3), pad=1, m_u=5, round_mode=ROUND_PSR, allow_overflow=False):
+def conv_wgrad(x, e, rs=(3, 3), pad=1, m_u=5, round_mode=ROUND_PSR, allow_overflow=False, stride=1):
     """Returns (g int8 [Co,R,S,Ci], b)."""
     x, e = _c8(x), _c8(e)
     B, H, W, Ci = x.shape
     Co = e.shape[3]
     R, S = rs
+    assert e.shape[1:3] == conv_out_hw(H, W, R, S, pad, stride)
     g = np.empty((Co, R, S, Ci), np.int8)
     b = np.zeros(1, np.int32)
-    _check(lib().niti_ref_conv_wgrad(_p8(x), _p8(e), _p8(g), _p32(b), B, H, W, Ci, Co, R, S, pad,
-                                     m_u, round_mode), allow_overflow)
+    _check(lib().niti_ref_conv_wgrad_s(_p8(x), _p8(e), _p8(g), _p32(b), B, H, W, Ci, Co, R, S, pad,
+                                       stride, m_u, round_mode), allow_overflow)
     return g, int(b[0])
 
 

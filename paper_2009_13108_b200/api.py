@@ -25,7 +25,8 @@ EXPORTS = [
     "niti_set_engine", "niti_set_reduce_hook", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
     "niti_redo_count", "niti_selftest_timeout", "niti_profile_enable", "niti_profile_read_launches",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
-    "niti_conv_dgrad", "niti_conv_wgrad", "niti_conv_wgrad_update", "niti_linear_bwd_update", "niti_int_xent", "niti_int_xent_noalloc", "niti_int_sgd_update",
+    "niti_conv_dgrad", "niti_conv_wgrad", "niti_conv_fwd_strided", "niti_conv_dgrad_strided", "niti_conv_wgrad_strided",
+    "niti_conv_wgrad_update", "niti_linear_bwd_update", "niti_int_xent", "niti_int_xent_noalloc", "niti_int_sgd_update",
     "niti_relu_fwd",
     "niti_relu_bwd", "niti_maxpool2_fwd", "niti_maxpool2_bwd", "niti_maxpool2_fwd_idx", "niti_maxpool2_bwd_idx",
 ]
@@ -75,6 +76,9 @@ def load_library():
     lib.niti_conv_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
     lib.niti_conv_dgrad.argtypes = [vp, vp, vp, vp, vp, vp, vp] + [i32] * 9 + [vp, sz]
     lib.niti_conv_wgrad.argtypes = [vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
+    lib.niti_conv_fwd_strided.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp] + [i32] * 11 + [vp, sz]
+    lib.niti_conv_dgrad_strided.argtypes = [vp, vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
+    lib.niti_conv_wgrad_strided.argtypes = [vp, vp, vp, vp, vp, vp] + [i32] * 11 + [vp, sz]
     lib.niti_conv_wgrad_update.argtypes = [vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
     lib.niti_linear_bwd_update.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, sz]
     lib.niti_int_xent.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, sz]
@@ -245,43 +249,59 @@ class Niti:
         return (e_prev if need_e_prev else None), g, b_e, b_g
 
     def conv_fwd(self, x, s_x, w, s_w, y=None, s_y=None, b_y=None, pad=1, relu=False,
-                 round_mode=ROUND_PSR):
+                 round_mode=ROUND_PSR, stride=1):
+        """niti_conv_fwd (stride 1) / niti_conv_fwd_strided."""
         B, H, W, Ci = x.shape
         Co, R, S, _ = w.shape
-        Ho, Wo = H + 2 * pad - R + 1, W + 2 * pad - S + 1
+        Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
         y = y if y is not None else torch.empty((B, Ho, Wo, Co), dtype=torch.int8, device=self.device)
         s_y = s_y if s_y is not None else self.scalar()
         b_y = b_y if b_y is not None else self.scalar()
-        ws, wsb = self._ws_for(OP_CONV_FWD, [B, H, W, Ci, Co, R, S, pad])
-        self._ck(self.lib.niti_conv_fwd(self.h, self._stream(), _ptr(x), _ptr(s_x), _ptr(w),
-                                        _ptr(s_w), _ptr(y), _ptr(s_y), _ptr(b_y), B, H, W, Ci, Co,
-                                        R, S, pad, int(relu), round_mode, ws, wsb))
+        ws, wsb = self._ws_for(OP_CONV_FWD, [B, H, W, Ci, Co, R, S, pad, stride])
+        if stride == 1:
+            self._ck(self.lib.niti_conv_fwd(self.h, self._stream(), _ptr(x), _ptr(s_x), _ptr(w),
+                                            _ptr(s_w), _ptr(y), _ptr(s_y), _ptr(b_y), B, H, W, Ci, Co,
+                                            R, S, pad, int(relu), round_mode, ws, wsb))
+        else:
+            self._ck(self.lib.niti_conv_fwd_strided(self.h, self._stream(), _ptr(x), _ptr(s_x), _ptr(w),
+                                                    _ptr(s_w), _ptr(y), _ptr(s_y), _ptr(b_y), B, H, W, Ci, Co,
+                                                    R, S, pad, stride, int(relu), round_mode, ws, wsb))
         return y, s_y, b_y
 
     def conv_dgrad(self, e, w, in_hw, e_prev=None, relu_mask_src=None, b_e=None, pad=1,
-                   round_mode=ROUND_PSR):
+                   round_mode=ROUND_PSR, stride=1):
         B = e.shape[0]
         H, W = in_hw
         Co, R, S, Ci = w.shape
         e_prev = e_prev if e_prev is not None else torch.empty((B, H, W, Ci), dtype=torch.int8,
                                                                 device=self.device)
         b_e = b_e if b_e is not None else self.scalar()
-        ws, wsb = self._ws_for(OP_CONV_DGRAD, [B, H, W, Ci, Co, R, S, pad])
-        self._ck(self.lib.niti_conv_dgrad(self.h, self._stream(), _ptr(e), _ptr(w), _ptr(e_prev),
-                                          _ptr(relu_mask_src), _ptr(b_e), B, H, W, Ci, Co, R, S,
-                                          pad, round_mode, ws, wsb))
+        ws, wsb = self._ws_for(OP_CONV_DGRAD, [B, H, W, Ci, Co, R, S, pad, stride])
+        if stride == 1:
+            self._ck(self.lib.niti_conv_dgrad(self.h, self._stream(), _ptr(e), _ptr(w), _ptr(e_prev),
+                                              _ptr(relu_mask_src), _ptr(b_e), B, H, W, Ci, Co, R, S,
+                                              pad, round_mode, ws, wsb))
+        else:
+            self._ck(self.lib.niti_conv_dgrad_strided(self.h, self._stream(), _ptr(e), _ptr(w), _ptr(e_prev),
+                                                      _ptr(relu_mask_src), _ptr(b_e), B, H, W, Ci, Co, R, S,
+                                                      pad, stride, round_mode, ws, wsb))
         return e_prev, b_e
 
-    def conv_wgrad(self, x, e, rs=(3, 3), g=None, b_g=None, pad=1, m_u=5, round_mode=ROUND_PSR):
+    def conv_wgrad(self, x, e, rs=(3, 3), g=None, b_g=None, pad=1, m_u=5, round_mode=ROUND_PSR, stride=1):
         B, H, W, Ci = x.shape
         Co = e.shape[3]
         R, S = rs
         g = g if g is not None else torch.empty((Co, R, S, Ci), dtype=torch.int8, device=self.device)
         b_g = b_g if b_g is not None else self.scalar()
-        ws, wsb = self._ws_for(OP_CONV_WGRAD, [B, H, W, Ci, Co, R, S, pad])
-        self._ck(self.lib.niti_conv_wgrad(self.h, self._stream(), _ptr(x), _ptr(e), _ptr(g),
-                                          _ptr(b_g), B, H, W, Ci, Co, R, S, pad, m_u, round_mode,
-                                          ws, wsb))
+        ws, wsb = self._ws_for(OP_CONV_WGRAD, [B, H, W, Ci, Co, R, S, pad, stride])
+        if stride == 1:
+            self._ck(self.lib.niti_conv_wgrad(self.h, self._stream(), _ptr(x), _ptr(e), _ptr(g),
+                                              _ptr(b_g), B, H, W, Ci, Co, R, S, pad, m_u, round_mode,
+                                              ws, wsb))
+        else:
+            self._ck(self.lib.niti_conv_wgrad_strided(self.h, self._stream(), _ptr(x), _ptr(e), _ptr(g),
+                                                      _ptr(b_g), B, H, W, Ci, Co, R, S, pad, stride, m_u,
+                                                      round_mode, ws, wsb))
         return g, b_g
 
     def conv_wgrad_update(self, x, e, w, b_g=None, pad=1, m_u=5, round_mode=ROUND_PSR):

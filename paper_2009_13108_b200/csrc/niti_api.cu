@@ -3,7 +3,7 @@
 #include "niti_common.cuh"
 
 int niti_launch_im2col32(niti_ctx *ctx, cudaStream_t st, const int8_t *x, int8_t *xcol, int B, int H, int W,
-                         int Ci, int R, int S, int pad, int Ho, int Wo);
+                         int Ci, int R, int S, int pad, int stride, int Ho, int Wo);
 int niti_launch_pad_pitch(niti_ctx *ctx, cudaStream_t st, const int8_t *src, int8_t *dst, int rows, int n, int pitch);
 int niti_launch_pad_rows32(niti_ctx *ctx, cudaStream_t st, const int8_t *w, int8_t *wcol, int rows, int k);
 int niti_launch_round_compact32(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, const WsHeader *hdr, int8_t *out,
@@ -32,12 +32,15 @@ extern "C" int niti_create(niti_ctx **out, int device) {
     return NITI_ERR_SHAPE;
   }
   ctx->sm_count = prop.multiProcessorCount;
-  e = cudaMalloc(&ctx->d_status, 256);
-  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
+  // one allocation: the status words, then the table of speculative-estimate errors
+  const size_t dev_bytes = 256 + sizeof(int32_t) * 2 * NITI_SPEC_SLOTS;
+  e = cudaMalloc(&ctx->d_status, dev_bytes);
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, dev_bytes);
   if (e != cudaSuccess) {
     delete ctx;
     return NITI_ERR_CUDA;
   }
+  ctx->d_spec_tab = (int32_t *)((char *)ctx->d_status + 256);
   cudaDriverEntryPointQueryResult qres;
   void *fn = nullptr;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
@@ -153,11 +156,12 @@ static inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 
 
 static bool fill_conv(GemmProblem &p, int kind, int B, int H, int W, int Ci, int Co, int R, int S,
-                      int pad) {
+                      int pad, int stride = 1) {
   p.kind = kind;
-  p.B = B; p.H = H; p.W = W; p.Ci = Ci; p.Co = Co; p.R = R; p.S = S; p.pad = pad;
-  p.Ho = H + 2 * pad - R + 1;
-  p.Wo = W + 2 * pad - S + 1;
+  p.B = B; p.H = H; p.W = W; p.Ci = Ci; p.Co = Co; p.R = R; p.S = S; p.pad = pad; p.stride = stride;
+  if (stride < 1 || H + 2 * pad < R || W + 2 * pad < S) return false;
+  p.Ho = (H + 2 * pad - R) / stride + 1;
+  p.Wo = (W + 2 * pad - S) / stride + 1;
   if (p.Ho <= 0 || p.Wo <= 0) return false;
   if (kind == GK_CONV_FWD) { p.gm = (long long)B * p.Ho * p.Wo; p.gn = Co; p.gk = (long long)R * S * Ci; }
   else if (kind == GK_CONV_DGRAD) { p.gm = (long long)B * H * W; p.gn = Ci; p.gk = (long long)R * S * Co; }
@@ -203,13 +207,15 @@ extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
     case NITI_OP_CONV_DGRAD:
     case NITI_OP_CONV_WGRAD_UPDATE:
     case NITI_OP_CONV_WGRAD: {
-      if (nd != 8) return 0;
+      if (nd != 8 && nd != 9) return 0;                  // a ninth entry is the stride (default 1)
       for (int i = 0; i < 7; ++i)
         if (d[i] <= 0) return 0;
+      const int stride = nd == 9 ? (int)d[8] : 1;
       const bool upd = op == NITI_OP_CONV_WGRAD_UPDATE;
       if (upd) op = NITI_OP_CONV_WGRAD;
       int kind = op == NITI_OP_CONV_FWD ? GK_CONV_FWD : (op == NITI_OP_CONV_DGRAD ? GK_CONV_DGRAD : GK_CONV_WGRAD);
-      if (!fill_conv(p, kind, (int)d[0], (int)d[1], (int)d[2], (int)d[3], (int)d[4], (int)d[5], (int)d[6], (int)d[7]))
+      if (!fill_conv(p, kind, (int)d[0], (int)d[1], (int)d[2], (int)d[3], (int)d[4], (int)d[5], (int)d[6], (int)d[7],
+                     stride))
         return 0;
       outs = (size_t)(p.gm * p.gn);
       extra = niti_tc_scratch_bytes(p);
@@ -368,20 +374,20 @@ static int conv_args_ok(int B, int H, int W, int Ci, int Co, int R, int S, int p
          (round_mode == 0 || round_mode == 1);
 }
 
-extern "C" int niti_conv_fwd(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x,
-                             const int8_t *w, const int32_t *s_w, int8_t *y, int32_t *s_y, int32_t *b_y,
-                             int B, int H, int W, int Cin, int Cout, int R, int S, int pad, int relu,
-                             int round_mode, void *ws, size_t ws_bytes) {
+extern "C" int niti_conv_fwd_strided(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x,
+                                     const int8_t *w, const int32_t *s_w, int8_t *y, int32_t *s_y, int32_t *b_y,
+                                     int B, int H, int W, int Cin, int Cout, int R, int S, int pad, int stride,
+                                     int relu, int round_mode, void *ws, size_t ws_bytes) {
   if (!ctx) return NITI_ERR_ARG;
   GemmProblem p;
   memset(&p, 0, sizeof(p));
   if (!x || !w || !y || !s_x || !s_w || !conv_args_ok(B, H, W, Cin, Cout, R, S, pad, round_mode) ||
       misaligned16(x) || misaligned16(w) || misaligned16(y) ||
-      !fill_conv(p, GK_CONV_FWD, B, H, W, Cin, Cout, R, S, pad))
+      !fill_conv(p, GK_CONV_FWD, B, H, W, Cin, Cout, R, S, pad, stride))
     return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_fwd: bad argument (pointers must be 16-byte aligned)");
   p.p0 = x; p.p1 = w;
-  int64_t dims[8] = {B, H, W, Cin, Cout, R, S, pad};
-  const size_t need = niti_workspace_bytes(NITI_OP_CONV_FWD, dims, 8);
+  int64_t dims[9] = {B, H, W, Cin, Cout, R, S, pad, stride};
+  const size_t need = niti_workspace_bytes(NITI_OP_CONV_FWD, dims, 9);
   if (few_channel_conv(Cin, R, S) && ctx->engine != 1) {
     if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
       return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
@@ -391,7 +397,7 @@ extern "C" int niti_conv_fwd(niti_ctx *ctx, void *stream, const int8_t *x, const
     char *base = (char *)ws + NITI_WS_HEADER + round_up(M * (size_t)Cout * 4, 256);
     int8_t *xcol = (int8_t *)base;
     int8_t *wcol = (int8_t *)(base + round_up(M * 32, 256));
-    int rc = niti_launch_im2col32(ctx, st, x, xcol, B, H, W, Cin, R, S, pad, p.Ho, p.Wo);
+    int rc = niti_launch_im2col32(ctx, st, x, xcol, B, H, W, Cin, R, S, pad, stride, p.Ho, p.Wo);
     if (rc == NITI_OK) rc = niti_launch_pad_rows32(ctx, st, w, wcol, Cout, R * S * Cin);
     if (rc != NITI_OK) return rc;
     GemmProblem q;
@@ -403,42 +409,58 @@ extern "C" int niti_conv_fwd(niti_ctx *ctx, void *stream, const int8_t *x, const
                         s_x, s_w, s_y, b_y);
 }
 
-extern "C" int niti_conv_dgrad(niti_ctx *ctx, void *stream, const int8_t *e, const int8_t *w,
-                               int8_t *e_prev, const int8_t *relu_mask_src, int32_t *b_e, int B, int H,
-                               int W, int Cin, int Cout, int R, int S, int pad, int round_mode, void *ws,
-                               size_t ws_bytes) {
+extern "C" int niti_conv_fwd(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x,
+                             const int8_t *w, const int32_t *s_w, int8_t *y, int32_t *s_y, int32_t *b_y,
+                             int B, int H, int W, int Cin, int Cout, int R, int S, int pad, int relu,
+                             int round_mode, void *ws, size_t ws_bytes) {
+  return niti_conv_fwd_strided(ctx, stream, x, s_x, w, s_w, y, s_y, b_y, B, H, W, Cin, Cout, R, S, pad, 1, relu,
+                               round_mode, ws, ws_bytes);
+}
+
+extern "C" int niti_conv_dgrad_strided(niti_ctx *ctx, void *stream, const int8_t *e, const int8_t *w,
+                                       int8_t *e_prev, const int8_t *relu_mask_src, int32_t *b_e, int B, int H,
+                                       int W, int Cin, int Cout, int R, int S, int pad, int stride, int round_mode,
+                                       void *ws, size_t ws_bytes) {
   if (!ctx) return NITI_ERR_ARG;
   GemmProblem p;
   memset(&p, 0, sizeof(p));
   if (!e || !w || !e_prev || !conv_args_ok(B, H, W, Cin, Cout, R, S, pad, round_mode) || misaligned16(e) ||
       misaligned16(w) || misaligned16(e_prev) || misaligned16(relu_mask_src) ||
-      !fill_conv(p, GK_CONV_DGRAD, B, H, W, Cin, Cout, R, S, pad))
+      !fill_conv(p, GK_CONV_DGRAD, B, H, W, Cin, Cout, R, S, pad, stride))
     return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_dgrad: bad argument (pointers must be 16-byte aligned)");
   p.p0 = e; p.p1 = w;
-  int64_t dims[8] = {B, H, W, Cin, Cout, R, S, pad};
+  int64_t dims[9] = {B, H, W, Cin, Cout, R, S, pad, stride};
   return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes,
-                        niti_workspace_bytes(NITI_OP_CONV_DGRAD, dims, 8), e_prev, 7, round_mode, 0,
+                        niti_workspace_bytes(NITI_OP_CONV_DGRAD, dims, 9), e_prev, 7, round_mode, 0,
                         relu_mask_src, nullptr, nullptr, nullptr, b_e);
+}
+
+extern "C" int niti_conv_dgrad(niti_ctx *ctx, void *stream, const int8_t *e, const int8_t *w,
+                               int8_t *e_prev, const int8_t *relu_mask_src, int32_t *b_e, int B, int H,
+                               int W, int Cin, int Cout, int R, int S, int pad, int round_mode, void *ws,
+                               size_t ws_bytes) {
+  return niti_conv_dgrad_strided(ctx, stream, e, w, e_prev, relu_mask_src, b_e, B, H, W, Cin, Cout, R, S, pad, 1,
+                                 round_mode, ws, ws_bytes);
 }
 
 // Weight gradient of a convolution; with update_w the rounded gradient is subtracted from the
 // weights in place instead of being returned.
 static int conv_wgrad_impl(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
                            int8_t *update_w, int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S,
-                           int pad, int m_u, int round_mode, void *ws, size_t ws_bytes, const char *who) {
+                           int pad, int stride, int m_u, int round_mode, void *ws, size_t ws_bytes, const char *who) {
   if (!ctx) return NITI_ERR_ARG;
   GemmProblem p;
   memset(&p, 0, sizeof(p));
   if (!x || !e || (!g && !update_w) || m_u < 1 || m_u > 7 || !conv_args_ok(B, H, W, Cin, Cout, R, S, pad, round_mode) ||
       misaligned16(x) || misaligned16(e) || misaligned16(g) || misaligned16(update_w) ||
-      !fill_conv(p, GK_CONV_WGRAD, B, H, W, Cin, Cout, R, S, pad)) {
+      !fill_conv(p, GK_CONV_WGRAD, B, H, W, Cin, Cout, R, S, pad, stride)) {
     snprintf(ctx->err, sizeof(ctx->err), "%s: bad argument (pointers must be 16-byte aligned)", who);
     return NITI_ERR_ARG;
   }
   p.p0 = e; p.p1 = x;
-  int64_t dims[8] = {B, H, W, Cin, Cout, R, S, pad};
-  const size_t need_base = niti_workspace_bytes(NITI_OP_CONV_WGRAD, dims, 8);
-  const size_t need = update_w ? niti_workspace_bytes(NITI_OP_CONV_WGRAD_UPDATE, dims, 8) : need_base;
+  int64_t dims[9] = {B, H, W, Cin, Cout, R, S, pad, stride};
+  const size_t need_base = niti_workspace_bytes(NITI_OP_CONV_WGRAD, dims, 9);
+  const size_t need = update_w ? niti_workspace_bytes(NITI_OP_CONV_WGRAD_UPDATE, dims, 9) : need_base;
   if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
     return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
   if (update_w) g = (int8_t *)((char *)ws + need_base);       // scratch, used only where the rounding stores int8
@@ -453,7 +475,7 @@ static int conv_wgrad_impl(niti_ctx *ctx, void *stream, const int8_t *x, const i
     int32_t *acc32 = (int32_t *)(base + round_up(M * 32, 256) + round_up((size_t)Cout * 32, 256));
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, NITI_WS_HEADER, st));
     ctx->launches++;
-    int rc = niti_launch_im2col32(ctx, st, x, xcol, B, H, W, Cin, R, S, pad, p.Ho, p.Wo);
+    int rc = niti_launch_im2col32(ctx, st, x, xcol, B, H, W, Cin, R, S, pad, stride, p.Ho, p.Wo);
     if (rc != NITI_OK) return rc;
     GemmProblem q;
     fill_fc(q, GK_FC_WGRAD, (int)M, Cout, 32);     // rows M are the contraction
@@ -477,18 +499,25 @@ static int conv_wgrad_impl(niti_ctx *ctx, void *stream, const int8_t *x, const i
                         nullptr, nullptr, nullptr, b_g, update_w);
 }
 
+extern "C" int niti_conv_wgrad_strided(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
+                                       int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
+                                       int stride, int m_u, int round_mode, void *ws, size_t ws_bytes) {
+  if (ctx && !g) return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_wgrad: bad argument (g is null)");
+  return conv_wgrad_impl(ctx, stream, x, e, g, nullptr, b_g, B, H, W, Cin, Cout, R, S, pad, stride, m_u, round_mode,
+                         ws, ws_bytes, "niti_conv_wgrad");
+}
+
 extern "C" int niti_conv_wgrad(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *g,
                                int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
                                int m_u, int round_mode, void *ws, size_t ws_bytes) {
-  if (ctx && !g) return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_wgrad: bad argument (g is null)");
-  return conv_wgrad_impl(ctx, stream, x, e, g, nullptr, b_g, B, H, W, Cin, Cout, R, S, pad, m_u, round_mode, ws,
-                         ws_bytes, "niti_conv_wgrad");
+  return niti_conv_wgrad_strided(ctx, stream, x, e, g, b_g, B, H, W, Cin, Cout, R, S, pad, 1, m_u, round_mode, ws,
+                                 ws_bytes);
 }
 
 extern "C" int niti_conv_wgrad_update(niti_ctx *ctx, void *stream, const int8_t *x, const int8_t *e, int8_t *w,
                                       int32_t *b_g, int B, int H, int W, int Cin, int Cout, int R, int S, int pad,
                                       int m_u, int round_mode, void *ws, size_t ws_bytes) {
   if (ctx && !w) return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_wgrad_update: bad argument (w is null)");
-  return conv_wgrad_impl(ctx, stream, x, e, nullptr, w, b_g, B, H, W, Cin, Cout, R, S, pad, m_u, round_mode, ws,
+  return conv_wgrad_impl(ctx, stream, x, e, nullptr, w, b_g, B, H, W, Cin, Cout, R, S, pad, 1, m_u, round_mode, ws,
                          ws_bytes, "niti_conv_wgrad_update");
 }

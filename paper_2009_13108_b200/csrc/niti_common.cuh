@@ -13,7 +13,9 @@ struct niti_ctx {
   int sm_count;
   int engine;               // niti_set_engine: 0 auto, 1 CUDA-core kernels only, 2 single-CTA tensor-core kernel,
                             // 3 paired-CTA only, 4 two-pass (int32 spill) epilogue, 5 no resident-weights mode
-  uint32_t *d_status;       // device status word
+  uint32_t *d_status;       // device status word (+ counter of recomputations)
+  int32_t *d_spec_tab;      // NITI_SPEC_SLOTS x {tag, error}: per call site, by how many bits the sample-based
+                            // estimate of the speculative epilogue missed the true bit-width last time
   uint64_t launches;
   uint64_t tc_launches;     // launches of the tensor-core matrix-multiply kernel
   uint64_t tc2_launches;    // of those, launches of the paired-CTA (cta_group::2) variant
@@ -38,6 +40,7 @@ struct niti_ctx {
 
 
 #define NITI_PROF_MAX 8192
+#define NITI_SPEC_SLOTS 4096
 #define NITI_WS_HEADER 4096 // bytes reserved at the start of every workspace: reduction scalars, then split maxima
 // A contraction that is split over CTAs adds int32 partial sums; split s records the largest magnitude
 // among its partial sums in split_max[s] (unsigned words from byte NITI_SPLIT_MAX_OFF of the header).
@@ -132,9 +135,9 @@ struct GemmProblem {
   int kind;
   const int8_t *p0;  // first operand  (a / e / x)
   const int8_t *p1;  // second operand (w / a / e)
-  // fully connected: M, N, K of the layer.  convolution: B,H,W (input), Ho,Wo (output), Ci, Co, R, S, pad
+  // fully connected: M, N, K of the layer.  convolution: B,H,W (input), Ho,Wo (output), Ci, Co, R, S, pad, stride
   int M, N, K;
-  int B, H, W, Ho, Wo, Ci, Co, R, S, pad;
+  int B, H, W, Ho, Wo, Ci, Co, R, S, pad, stride;
   // the matrix multiply actually run
   long long gm, gn, gk;
   // row pitch in bytes of p0 when its rows are padded (fully connected kinds; 0 = dense)

@@ -104,7 +104,7 @@ int niti_launch_round(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, const 
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 im2col32_kernel(const int8_t *__restrict__ x, int8_t *__restrict__ xcol, int B, int H, int W, int Ci, int R,
-                int S, int pad, int Ho, int Wo) {
+                int S, int pad, int stride, int Ho, int Wo) {
   const long long M = (long long)B * Ho * Wo;
   for (long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x; m < M;
        m += (long long)gridDim.x * blockDim.x) {
@@ -115,9 +115,9 @@ im2col32_kernel(const int8_t *__restrict__ x, int8_t *__restrict__ xcol, int B, 
     unsigned w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     int k = 0;
     for (int r = 0; r < R; ++r) {
-      const int ii = i + r - pad;
+      const int ii = i * stride + r - pad;
       for (int q = 0; q < S; ++q) {
-        const int jj = j + q - pad;
+        const int jj = j * stride + q - pad;
         const bool in = ii >= 0 && ii < H && jj >= 0 && jj < W;
         const int8_t *src = x + ((b * H + ii) * W + jj) * Ci;
         for (int c = 0; c < Ci; ++c, ++k) {
@@ -228,8 +228,8 @@ __global__ void round_compact32_kernel(const int32_t *__restrict__ acc, const Ws
 }
 
 int niti_launch_im2col32(niti_ctx *ctx, cudaStream_t st, const int8_t *x, int8_t *xcol, int B, int H, int W,
-                         int Ci, int R, int S, int pad, int Ho, int Wo) {
-  if (Ci == 3 && R == 3 && S == 3 && pad == 1 && (W % 4) == 0 && (long long)B * H < (1LL << 31) &&
+                         int Ci, int R, int S, int pad, int stride, int Ho, int Wo) {
+  if (Ci == 3 && R == 3 && S == 3 && pad == 1 && stride == 1 && (W % 4) == 0 && (long long)B * H < (1LL << 31) &&
       ((uintptr_t)xcol & 31) == 0) {
     const int threads = W / 4 >= 128 ? 128 : (W / 4 > 32 ? 64 : 32);
     const size_t smem = (size_t)3 * (W * 3 / 4 + 2) * sizeof(unsigned);
@@ -243,7 +243,7 @@ int niti_launch_im2col32(niti_ctx *ctx, cudaStream_t st, const int8_t *x, int8_t
   long long M = (long long)B * Ho * Wo;
   long long blocks = (M + 255) / 256;
   if (blocks > (long long)ctx->sm_count * 16) blocks = (long long)ctx->sm_count * 16;
-  im2col32_kernel<<<(unsigned)blocks, 256, 0, st>>>(x, xcol, B, H, W, Ci, R, S, pad, Ho, Wo);
+  im2col32_kernel<<<(unsigned)blocks, 256, 0, st>>>(x, xcol, B, H, W, Ci, R, S, pad, stride, Ho, Wo);
   ctx->launches++;
   NITI_CUDA_TRY(ctx, cudaGetLastError());
   return NITI_OK;

@@ -14,7 +14,7 @@ struct Addr {
   const int8_t *p0, *p1;
   int kind;
   int M, N, K;                                  // fully connected dims
-  int H, W, Ho, Wo, Ci, Co, R, S, pad;          // convolution dims
+  int H, W, Ho, Wo, Ci, Co, R, S, pad, stride;  // convolution dims
   long long gm, gn, gk;
   long long pitch0;                             // row pitch of p0 for the fully connected backward kinds
 };
@@ -34,7 +34,7 @@ __device__ __forceinline__ int8_t load_a(const Addr &q, long long m, long long k
       long long t = m / q.Wo;
       int i = (int)(t % q.Ho);
       long long b = t / q.Ho;
-      int ii = i + r - q.pad, jj = j + s - q.pad;
+      int ii = i * q.stride + r - q.pad, jj = j * q.stride + s - q.pad;
       if (ii < 0 || ii >= q.H || jj < 0 || jj >= q.W) return 0;
       return q.p0[((b * q.H + ii) * q.W + jj) * q.Ci + ci];
     }
@@ -46,8 +46,15 @@ __device__ __forceinline__ int8_t load_a(const Addr &q, long long m, long long k
       long long t = m / q.W;
       int ii = (int)(t % q.H);
       long long b = t / q.H;
-      int i = ii - r + q.pad, j = jj - s + q.pad;
-      if (i < 0 || i >= q.Ho || j < 0 || j >= q.Wo) return 0;
+      // the output pixel (i, j) whose window puts tap (r, s) on this input pixel, if there is one
+      int ti = ii - r + q.pad, tj = jj - s + q.pad;
+      if (ti < 0 || tj < 0) return 0;
+      int i = ti, j = tj;
+      if (q.stride > 1) {
+        i = ti / q.stride; j = tj / q.stride;
+        if (i * q.stride != ti || j * q.stride != tj) return 0;
+      }
+      if (i >= q.Ho || j >= q.Wo) return 0;
       return q.p0[((b * q.Ho + i) * q.Wo + j) * q.Co + co];
     }
     default: /* GK_CONV_WGRAD */ return q.p0[k * q.Co + m];   // e[pix][co]
@@ -75,7 +82,7 @@ __device__ __forceinline__ int8_t load_b(const Addr &q, long long n, long long k
       long long t = k / q.Wo;
       int i = (int)(t % q.Ho);
       long long b = t / q.Ho;
-      int ii = i + r - q.pad, jj = j + s - q.pad;
+      int ii = i * q.stride + r - q.pad, jj = j * q.stride + s - q.pad;
       if (ii < 0 || ii >= q.H || jj < 0 || jj >= q.W) return 0;
       return q.p1[((b * q.H + ii) * q.W + jj) * q.Ci + ci];
     }
@@ -228,6 +235,7 @@ int niti_simt_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t
   q.p0 = p.p0; q.p1 = p.p1; q.kind = p.kind;
   q.M = p.M; q.N = p.N; q.K = p.K;
   q.H = p.H; q.W = p.W; q.Ho = p.Ho; q.Wo = p.Wo; q.Ci = p.Ci; q.Co = p.Co; q.R = p.R; q.S = p.S; q.pad = p.pad;
+  q.stride = p.stride > 0 ? p.stride : 1;
   q.gm = p.gm; q.gn = p.gn; q.gk = p.gk;
   q.pitch0 = p.ld0 ? p.ld0 : p.N;
   long long gx = (p.gn + TN - 1) / TN, gy = (p.gm + TM - 1) / TM;

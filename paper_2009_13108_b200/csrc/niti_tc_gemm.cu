@@ -74,6 +74,8 @@ struct TcParams {
   int w_tiles, h_tiles, b_tiles;
   int PW, PH, PB;               // extent of the pixel grid the output rows (or k-blocks) run over
   int R, S, pad;
+  int stride;                   // convolution stride (forward and weight gradient; the shifted operand is then
+                                // copied with that element stride, so a box still lands as Wt x Ht pixels)
   int c_chunks;                 // channel chunks per tap along the contraction (fwd / dgrad)
   int Cn;                       // wgrad: input channels Ci (columns per tap)
   int n_chunks;                 // wgrad: column chunks per tap
@@ -102,6 +104,7 @@ struct TcParams {
   int epi_mode;                 // EPI_SPILL / EPI_ATOMIC / EPI_SPECULATE / EPI_KNOWN_B
   int mbits, round_mode, relu;
   unsigned spec_mul256;         // the sampled max is scaled by this / 256 before taking its bit length
+  int spec_tag;                 // identifies the call site (its b_out scalar) in the table of estimate errors
   int single_wave;              // every CTA has at most one tile: the sample is the whole tensor, the shift
                                 // is exact, and the last CTA to finish publishes b and the exponent
 };
@@ -171,12 +174,23 @@ __device__ __forceinline__ bool mbar_try_sleep(unsigned bar, unsigned parity, un
       : "memory");
   return ok != 0;
 }
+// A waiting warp that keeps polling competes with the working warps of its scheduler for issue slots
+// and for the integer pipe (measured: the hardware wait above returns after a few tens of cycles, so a
+// warp that waits through a whole epilogue-bound tile executes a poll loop every ~70 cycles, a fifth of
+// its scheduler's integer-pipe capacity).  After two failed polls the warp therefore sleeps between
+// polls, 128 ns at first and 256 ns from the eighth poll on: short waits (data about to land) are not
+// delayed, long waits (the pipeline is bound elsewhere) cost almost nothing.
+__device__ __forceinline__ void wait_backoff(unsigned &polls) {
+  ++polls;
+  if (polls > 2) __nanosleep(polls > 8 ? 256u : 128u);
+}
 // Bounded wait.  Returns false (and raises the abort flag) if the barrier did not flip in time or
 // another thread already gave up.
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int *abort_flag,
                                           uint32_t *status, long long limit_cycles = WAIT_LIMIT_CYCLES) {
   if (mbar_try(bar, parity)) return true;
   long long t0 = clock64();
+  unsigned polls = 0;
   while (true) {
     if (mbar_try_sleep(bar, parity, 20000u)) return true;
     if (*abort_flag) return false;
@@ -185,6 +199,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatil
       atomicOr(status, NITI_DEV_TIMEOUT);
       return false;
     }
+    wait_backoff(polls);
   }
 }
 // The same bounded wait for a whole converged warp: every lane polls, the votes make the outcome (and
@@ -194,6 +209,7 @@ __device__ __forceinline__ bool mbar_wait_warp(unsigned bar, unsigned parity, vo
                                                uint32_t *status, long long limit_cycles = WAIT_LIMIT_CYCLES) {
   if (__all_sync(0xffffffffu, mbar_try(bar, parity))) return true;
   const long long t0 = clock64();
+  unsigned polls = 0;
   while (true) {
     if (__all_sync(0xffffffffu, mbar_try_sleep(bar, parity, 20000u))) return true;
     if (__any_sync(0xffffffffu, *abort_flag != 0)) return false;
@@ -202,6 +218,7 @@ __device__ __forceinline__ bool mbar_wait_warp(unsigned bar, unsigned parity, vo
       atomicOr(status, NITI_DEV_TIMEOUT);
       return false;
     }
+    wait_backoff(polls);
   }
 }
 // One lane of a converged warp (the same one every time it is asked).
@@ -656,7 +673,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const TcParams p, int32_t *__restrict__ acc, WsHeader *hdr, uint32_t *status,
                int8_t *__restrict__ out8, const int8_t *__restrict__ mask8, const int32_t *s_a,
-               const int32_t *s_w, int32_t *s_out, int32_t *b_out) {
+               const int32_t *s_w, int32_t *s_out, int32_t *b_out, int32_t *spec_slot) {
   if (p.epi_mode == EPI_SPECULATE && !p.single_wave) {
     // the follow-up launch may be scheduled now (it is launched as a programmatic dependent): its CTAs
     // take the SMs as this grid's CTAs retire and wait there for the whole grid to finish
@@ -667,6 +684,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     asm volatile("griddepcontrol.wait;" ::: "memory");     // the first pass has completed and is visible
     const int b_true = niti_bitlen32(hdr->maxabs32), b_est = (int)hdr->spec_b - 1;   // (stored + 1)
     if (blockIdx.x == 0 && threadIdx.x == 0) {
+      if (spec_slot) {
+        // remember, for the next call from this call site, how far the sample-based estimate was off
+        // (b_est = raw estimate + the correction this call applied)
+        const int corr = spec_slot[0] == p.spec_tag ? spec_slot[1] : 0;
+        int err = b_true - (b_est - corr);
+        err = err < -2 ? -2 : (err > 2 ? 2 : err);
+        spec_slot[0] = p.spec_tag;
+        spec_slot[1] = err;
+      }
       const int bp = b_true > p.mbits ? b_true - p.mbits : 0;
       if (b_out) *b_out = b_true;
       if (s_out) {
@@ -864,6 +890,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           decode_item(p, item, mu, nt, split);
           if (p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) pixel_box(p, mu * CTAS + (int)rank, w0, h0, b0);
         }
+        if (p.kind == GK_CONV_FWD) { w0 *= p.stride; h0 *= p.stride; }     // output pixel -> window origin in x
         const int mt = mu * CTAS + (int)rank;     // this CTA's 128-row tile
         const int nb = nt * p.bn + (int)rank * bn_cta;
         const int kb0 = split * p.kb_per_split;
@@ -932,8 +959,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               for (int j = 0; j < p.a_boxes; ++j)
                 load4<CTAS>(sa + j * p.a_box_bytes, &map_a, full, mt * BM + j * p.a_box_step, kw0, kh0, kbb0);
               for (int j = 0; j < p.b_boxes; ++j)
-                load4<CTAS>(sb + j * p.b_box_bytes, &map_b, full, ci0 + j * p.b_box_step, kw0 + wg_s - p.pad,
-                            kh0 + wg_r - p.pad, kbb0);
+                load4<CTAS>(sb + j * p.b_box_bytes, &map_b, full, ci0 + j * p.b_box_step, kw0 * p.stride + wg_s - p.pad,
+                            kh0 * p.stride + wg_r - p.pad, kbb0);
               break;
             }
           }
@@ -1326,7 +1353,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   // to the whole tensor before taking the bit length (a wrong guess only costs the redo)
                   unsigned long long scaled = ((unsigned long long)v_max * p.spec_mul256) >> 8;
                   if (scaled > 0x7fffffffull) scaled = 0x7fffffffull;
-                  const unsigned mine = (unsigned)niti_bitlen32((unsigned)scaled) + 1u;
+                  // plus what the same estimate missed by at this call site last time (a systematic
+                  // error of the sample, e.g. a tensor whose extremes sit outside the first tiles); never
+                  // below the bit length of the sample's own maximum, which the tensor's cannot undercut
+                  int guess = niti_bitlen32((unsigned)scaled);
+                  if (spec_slot && p.spec_mul256 != 256 && *(volatile int *)&spec_slot[0] == p.spec_tag)
+                    guess += *(volatile int *)&spec_slot[1];
+                  const int floor_b = niti_bitlen32(v_max);
+                  guess = guess < floor_b ? floor_b : (guess > 31 ? 31 : guess);
+                  const unsigned mine = (unsigned)guess + 1u;
                   const unsigned old = atomicCAS(&hdr->spec_b, 0u, mine);
                   pub = old ? old : mine;
                   break;
@@ -1675,9 +1710,10 @@ struct MapSpec {
   int nd;
   cuuint64_t dims[4];
   cuuint64_t strides[3];   // bytes, dims 1..3
-  cuuint32_t box[4];
+  cuuint32_t box[4];       // extent of the box in tensor elements (before the element stride)
   int swizzle;
   const void *base;
+  cuuint32_t estr[4];      // element (traversal) stride per dimension; 0 = 1
 };
 
 static bool encode(niti_ctx *ctx, CUtensorMap *m, const MapSpec &s) {
@@ -1688,6 +1724,8 @@ static bool encode(niti_ctx *ctx, CUtensorMap *m, const MapSpec &s) {
   for (int i = 0; i < s.nd; ++i)
     if (s.box[i] == 0 || s.box[i] > 256) return false;
   cuuint32_t es[4] = {1, 1, 1, 1};
+  for (int i = 0; i < s.nd; ++i)
+    if (s.estr[i] > 1) es[i] = s.estr[i];
   CUresult r = ((EncodeTiledFn)ctx->encode_tiled)(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)s.nd,
                                                   const_cast<void *>(s.base), s.dims, s.strides, s.box, es,
                                                   CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_enum(s.swizzle),
@@ -1771,26 +1809,36 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
     }
     case GK_CONV_FWD:
     case GK_CONV_DGRAD: {
-      // rows run over the pixels of the OUTPUT tensor of this multiply; the shifted operand is the
-      // other activation tensor.  Only "same" geometry (odd taps, pad = (R-1)/2) is taken here.
-      if (g.Ho != g.H || g.Wo != g.W) return false;
+      // Rows run over the pixels of the OUTPUT tensor of this multiply (forward: the Ho x Wo output;
+      // error: the H x W input-shaped tensor); the shifted operand is the other activation tensor and
+      // may have another size (padding other than (R-1)/2, strides): its copies start at any
+      // coordinate and read zeros outside it.  A forward stride becomes the element stride of those
+      // copies.  The error of a strided convolution is left to the CUDA-core engine.
       const bool fwd = g.kind == GK_CONV_FWD;
+      const int st = g.stride > 1 ? g.stride : 1;
+      if (!fwd && st != 1) return false;
+      const int RW = fwd ? g.Wo : g.W, RH = fwd ? g.Ho : g.H;      // pixel grid of the rows
+      const int OW = fwd ? g.W : g.Wo, OH = fwd ? g.H : g.Ho;      // pixel grid of the shifted operand
+      const bool same = g.Ho == g.H && g.Wo == g.W && st == 1;
       const int Cc = fwd ? g.Ci : g.Co;        // contraction channels
       const int Cn = fwd ? g.Co : g.Ci;        // output channels of this multiply
       p.kdepth = pick_swizzle(Cc);
       if (!p.kdepth || Cc % p.kdepth) return false;
-      if (!pick_pixel_box(g.W, g.H, g.B, p.Wt, p.Ht, p.Bt)) return false;
-      p.w_tiles = (g.W + p.Wt - 1) / p.Wt;
-      p.h_tiles = (g.H + p.Ht - 1) / p.Ht;
+      if (!pick_pixel_box(RW, RH, g.B, p.Wt, p.Ht, p.Bt)) return false;
+      if (p.Wt * st > 256 || p.Ht * st > 256) return false;
+      p.w_tiles = (RW + p.Wt - 1) / p.Wt;
+      p.h_tiles = (RH + p.Ht - 1) / p.Ht;
       p.b_tiles = (g.B + p.Bt - 1) / p.Bt;
-      p.PW = g.W; p.PH = g.H; p.PB = g.B;
+      p.PW = RW; p.PH = RH; p.PB = g.B;
       p.R = g.R; p.S = g.S; p.pad = g.pad;
+      p.stride = st;
       p.c_chunks = Cc / p.kdepth;
       p.Cn = Cn;
       a_sw = p.kdepth;
-      sa = {4, {(cuuint64_t)Cc, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.B},
-            {(cuuint64_t)Cc, (cuuint64_t)Cc * g.W, (cuuint64_t)Cc * g.W * g.H},
-            {(cuuint32_t)p.kdepth, (cuuint32_t)p.Wt, (cuuint32_t)p.Ht, (cuuint32_t)p.Bt}, a_sw, g.p0};
+      sa = {4, {(cuuint64_t)Cc, (cuuint64_t)OW, (cuuint64_t)OH, (cuuint64_t)g.B},
+            {(cuuint64_t)Cc, (cuuint64_t)Cc * OW, (cuuint64_t)Cc * OW * OH},
+            {(cuuint32_t)p.kdepth, (cuuint32_t)(p.Wt * st), (cuuint32_t)(p.Ht * st), (cuuint32_t)p.Bt}, a_sw, g.p0,
+            {1, (cuuint32_t)st, (cuuint32_t)st, 1}};
       if (fwd) {
         p.bn = Cn >= 256 ? 256 : round_up32(Cn);
         if (ctas == 2 && Cn > 256) {
@@ -1818,7 +1866,7 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
       m_tiles = (long long)p.w_tiles * p.h_tiles * p.b_tiles;
       p.n_tiles_n = (Cn + p.bn - 1) / p.bn;
       // halo mode: one channel chunk, one column tile, weights of all taps fit beside >= 3 patches
-      if (want_halo && ctas == 1 && g.R == 3 && g.S == 3 && g.pad == 1 && p.c_chunks == 1 && p.n_tiles_n == 1 &&
+      if (want_halo && same && ctas == 1 && g.R == 3 && g.S == 3 && g.pad == 1 && p.c_chunks == 1 && p.n_tiles_n == 1 &&
           g.W >= 10 && g.H >= 18) {
         const int a_stage = (180 * p.kdepth + 1023) / 1024 * 1024;
         const int b_res = (9 * p.bn * p.kdepth + 1023) / 1024 * 1024;
@@ -1838,10 +1886,14 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
       break;
     }
     case GK_CONV_WGRAD: {
-      if (g.Ho != g.H || g.Wo != g.W) return false;
+      // the contraction runs over the pixels of the OUTPUT grid (Ho x Wo); the input tensor is copied
+      // shifted by the tap, with the stride as element stride
+      const int st = g.stride > 1 ? g.stride : 1;
+      const bool same = g.Ho == g.H && g.Wo == g.W && st == 1;
+      p.stride = st;
       // (64 x 64)-channel blocks re-read the activations once per block of the other operand, so this
       // mode is kept for layers with few blocks; wide layers use the per-tap tiles below
-      if (want_halo && ctas == 1 && g.R == 3 && g.S == 3 && g.pad == 1 && g.Ci % 64 == 0 && g.Co % 64 == 0 &&
+      if (want_halo && same && ctas == 1 && g.R == 3 && g.S == 3 && g.pad == 1 && g.Ci % 64 == 0 && g.Co % 64 == 0 &&
           g.W >= 10 && g.H >= 18 && (long long)g.Ci * g.Co <= 32768) {
         p.halo = 2;
         p.kdepth = 128;
@@ -1901,23 +1953,25 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
       a_sw = pick_swizzle(g.Co);
       b_sw = pick_swizzle(g.Ci);
       if (!a_sw || !b_sw || g.Co % a_sw || g.Ci % b_sw) return false;
-      if (!pick_pixel_box(g.W, g.H, g.B, p.Wt, p.Ht, p.Bt)) return false;
+      if (!pick_pixel_box(g.Wo, g.Ho, g.B, p.Wt, p.Ht, p.Bt)) return false;
+      if (p.Wt * st > 256 || p.Ht * st > 256) return false;
       p.kdepth = 128;
-      p.w_tiles = (g.W + p.Wt - 1) / p.Wt;
-      p.h_tiles = (g.H + p.Ht - 1) / p.Ht;
+      p.w_tiles = (g.Wo + p.Wt - 1) / p.Wt;
+      p.h_tiles = (g.Ho + p.Ht - 1) / p.Ht;
       p.b_tiles = (g.B + p.Bt - 1) / p.Bt;
-      p.PW = g.W; p.PH = g.H; p.PB = g.B;
+      p.PW = g.Wo; p.PH = g.Ho; p.PB = g.B;
       p.R = g.R; p.S = g.S; p.pad = g.pad;
       p.Cn = g.Ci;
       p.bn = g.Ci >= 256 ? 256 : g.Ci;
       if (p.bn % 32 || g.Ci % p.bn) return false;
       p.n_chunks = g.Ci / p.bn;
-      sa = {4, {(cuuint64_t)g.Co, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.B},
-            {(cuuint64_t)g.Co, (cuuint64_t)g.Co * g.W, (cuuint64_t)g.Co * g.W * g.H},
+      sa = {4, {(cuuint64_t)g.Co, (cuuint64_t)g.Wo, (cuuint64_t)g.Ho, (cuuint64_t)g.B},
+            {(cuuint64_t)g.Co, (cuuint64_t)g.Co * g.Wo, (cuuint64_t)g.Co * g.Wo * g.Ho},
             {(cuuint32_t)a_sw, (cuuint32_t)p.Wt, (cuuint32_t)p.Ht, (cuuint32_t)p.Bt}, a_sw, g.p0};
       sb = {4, {(cuuint64_t)g.Ci, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.B},
             {(cuuint64_t)g.Ci, (cuuint64_t)g.Ci * g.W, (cuuint64_t)g.Ci * g.W * g.H},
-            {(cuuint32_t)b_sw, (cuuint32_t)p.Wt, (cuuint32_t)p.Ht, (cuuint32_t)p.Bt}, b_sw, g.p1};
+            {(cuuint32_t)b_sw, (cuuint32_t)(p.Wt * st), (cuuint32_t)(p.Ht * st), (cuuint32_t)p.Bt}, b_sw, g.p1,
+            {1, (cuuint32_t)st, (cuuint32_t)st, 1}};
       p.kb_total = p.w_tiles * p.h_tiles * p.b_tiles;
       m_tiles = (g.Co + BM - 1) / BM;
       p.n_tiles_n = g.R * g.S * p.n_chunks;
@@ -2164,8 +2218,15 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
     q.magic_w = (p.w_tiles > 1 && n_max * p.w_tiles < (1ull << 32)) ? (unsigned)((1ull << 32) / p.w_tiles + 1) : 0u;
     q.magic_h = (p.h_tiles > 1 && n_max * p.h_tiles < (1ull << 32)) ? (unsigned)((1ull << 32) / p.h_tiles + 1) : 0u;
   }
+  // per call site (keyed by the address of its bit-width scalar): the error of the last speculative estimate
+  int32_t *slot = nullptr;
+  if (r.b_out && ctx->d_spec_tab) {
+    const uintptr_t key = (uintptr_t)r.b_out >> 2;
+    slot = ctx->d_spec_tab + 2 * (size_t)((key ^ (key >> 13)) % NITI_SPEC_SLOTS);
+    q.spec_tag = (int)(unsigned)(key | 1u);
+  }
   NITI_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, tc_gemm_kernel<CTAS>, ma, mb, q, acc, hdr, ctx->d_status, r.out, r.mask,
-                                        r.s_a, r.s_w, r.s_out, r.b_out));
+                                        r.s_a, r.s_w, r.s_out, r.b_out, slot));
   ctx->launches++;
   ctx->tc_launches++;
   if (CTAS == 2) ctx->tc2_launches++;

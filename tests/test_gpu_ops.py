@@ -271,6 +271,32 @@ def test_speculative_shift_is_corrected(niti, oref, engine):
     niti.check()
 
 
+def test_speculative_estimate_learns_what_it_missed_at_a_call_site(niti, oref):
+    """A call site (recognised by the address of its bit-width scalar) whose extremes sit outside the
+    sampled first tiles mispredicts once, then no more; when the data changes the estimate follows after
+    one more recomputation.  Every result is exact."""
+    M, N, K = 128 * 400, 64, 128
+    w = np.full((N, K), 100, np.int8)
+    base = np.where(np.arange(M) % 2 == 0, 5, 6).astype(np.int8)[:, None].repeat(K, 1)   # sums up to 76800: 17 bits
+    tail = base.copy()
+    tail[-5:] = 11                                                                       # 140800: 18 bits
+    wt = _T(niti, w)
+    s_a, s_w = niti.scalar(-7), niti.scalar(-10)
+    out = torch.empty((M, N), dtype=torch.int8, device=niti.device)
+    s_out, b_out = niti.scalar(), niti.scalar(-1)
+    redo = []
+    for a, bits in ((tail, 18), (tail, 18), (tail, 18), (base, 17), (base, 17)):
+        want, s, b = oref.linear_fwd(a, -7, w, -10, True)
+        assert b == bits
+        r0 = niti.redo_count()
+        niti.linear_fwd(_T(niti, a), s_a, wt, s_w, out=out, s_out=s_out, b_out=b_out, relu=True)
+        _eq(out, want)
+        assert (int(s_out), int(b_out)) == (s, b)
+        redo.append(niti.redo_count() - r0)
+    assert redo == [1, 0, 0, 1, 0], redo
+    niti.check()
+
+
 def test_speculative_shift_is_corrected_in_conv_and_row_batched_modes(niti, oref):
     """Same for the resident-weights convolution (small channel counts) and for the row-batched
     multiply of short contractions: only the end of the tensor is large."""
@@ -335,8 +361,8 @@ def test_general_taps_and_padding_use_the_fallback(niti, oref):
 
 @pytest.mark.parametrize("engine", [0, 2, 3])
 @pytest.mark.parametrize("R,pad", [(5, 2), (7, 3), (1, 0)])
-@pytest.mark.parametrize("B,H,W,Ci,Co", [(2, 16, 16, 32, 64), (2, 12, 20, 64, 128), (3, 8, 16, 128, 32),
-                                         (1, 24, 40, 64, 64)])
+@pytest.mark.parametrize("B,H,W,Ci,Co", [(2, 16, 16, 32, 64), (8, 12, 20, 64, 128), (3, 8, 16, 128, 32),
+                                         (2, 24, 40, 64, 64)])
 def test_large_and_pointwise_filters_on_the_tensor_cores(niti, oref, B, H, W, Ci, Co, R, pad, engine):
     """5x5, 7x7 (the paper's LeNet / AlexNet filter sizes, Section 4) and 1x1 convolutions with "same"
     geometry and at least 32 channels run on the tcgen05 kernel: forward, error and weight gradient
@@ -415,6 +441,58 @@ def test_accumulator_range_is_flagged_where_the_oracle_reports_an_overflow(niti,
                 assert int(b_g) == bg and niti.check() == 0
     finally:
         niti.set_engine(0)
+
+
+STRIDED_SHAPES = [
+    # B, H, W, Ci, Co, R, pad, stride
+    (2, 23, 23, 3, 16, 11, 2, 4),      # the geometry of the paper's AlexNet first layer (11 x 11, stride 4), RGB input
+    (4, 16, 16, 32, 64, 3, 1, 2),      # tensor cores: element stride 2
+    (2, 32, 32, 64, 128, 5, 2, 2),
+    (8, 24, 24, 128, 64, 3, 1, 3),
+    (8, 33, 31, 64, 64, 3, 0, 2),      # odd sizes, no padding: rows the windows never reach
+    (3, 28, 28, 1, 32, 5, 0, 1),       # LeNet's 5 x 5 first layer without padding (gathered taps)
+    (8, 20, 20, 32, 64, 5, 0, 1),      # "valid" convolution on the tensor cores: output smaller than input
+    (8, 12, 12, 64, 32, 3, 3, 1),      # padding larger than (R - 1) / 2: output larger than input
+]
+
+
+@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("B,H,W,Ci,Co,R,pad,stride", STRIDED_SHAPES)
+def test_strided_and_unpadded_convolutions(niti, oref, B, H, W, Ci, Co, R, pad, stride, engine):
+    """Strides other than 1 and paddings other than (R - 1) / 2, forward / error / weight gradient,
+    against the oracle; with at least 32 channels on both sides the forward pass and the weight gradient
+    must run on the tensor cores (the error of a strided layer is the CUDA-core engine's)."""
+    rng = np.random.default_rng(B + H * 3 + W * 5 + Ci * 7 + Co * 11 + R + 13 * stride)
+    x, w = _i8(rng, (B, H, W, Ci)), _i8(rng, (Co, R, R, Ci))
+    Ho, Wo = oref.conv_out_hw(H, W, R, R, pad, stride)
+    e = _i8(rng, (B, Ho, Wo, Co))
+    xm = np.maximum(x, 0)
+    niti.set_engine(engine)
+    try:
+        n0 = niti.tc_launch_count()
+        wy, s, b = oref.conv_fwd(x, -7, w, -9, pad, True, stride=stride)
+        y, s_y, b_y = niti.conv_fwd(_T(niti, x), niti.scalar(-7), _T(niti, w), niti.scalar(-9), pad=pad,
+                                    relu=True, stride=stride)
+        _eq(y, wy)
+        assert (int(s_y), int(b_y)) == (s, b)
+        n1 = niti.tc_launch_count()
+        wd, bd = oref.conv_dgrad(e, w, (H, W), pad, xm, stride=stride)
+        ep, b_e = niti.conv_dgrad(_T(niti, e), _T(niti, w), (H, W), relu_mask_src=_T(niti, xm), pad=pad,
+                                  stride=stride)
+        _eq(ep, wd)
+        assert int(b_e) == bd
+        n2 = niti.tc_launch_count()
+        wg, bg = oref.conv_wgrad(x, e, (R, R), pad, 5, stride=stride)
+        g, b_g = niti.conv_wgrad(_T(niti, x), _T(niti, e), (R, R), pad=pad, stride=stride)
+        _eq(g, wg)
+        assert int(b_g) == bg
+        n3 = niti.tc_launch_count()
+        if engine == 0 and Ci >= 32 and Co >= 32:
+            assert n1 > n0 and n3 > n2, "forward / weight gradient fell back to the CUDA-core engine"
+            assert (n2 > n1) == (stride == 1)
+    finally:
+        niti.set_engine(0)
+    niti.check()
 
 
 def test_saturation_and_zero_tensor(niti, oref):

@@ -62,6 +62,76 @@ def test_conv_against_float64_conv2d(oref, B, H, W, Ci, Co, R, pad):
     assert np.array_equal(oref.conv_wgrad_acc(x, e, (R, R), pad), gw.astype(np.int64))
 
 
+STRIDED = [(1, 7, 7, 1, 1, 3, 1, 2), (2, 9, 8, 3, 4, 3, 1, 2), (1, 23, 23, 3, 5, 11, 2, 4),
+           (2, 10, 10, 4, 3, 5, 2, 2), (1, 8, 9, 2, 2, 2, 0, 2), (2, 6, 7, 3, 2, 1, 0, 3)]
+
+
+@pytest.mark.parametrize("B,H,W,Ci,Co,R,pad,stride", STRIDED)
+def test_strided_conv_against_float64_conv2d(oref, B, H, W, Ci, Co, R, pad, stride):
+    """Strides other than 1 (the first layer of the paper's AlexNet is 11 x 11 with stride 4, Section 4)
+    against torch's float64 conv2d / conv_transpose2d / conv2d_weight (exact below 2^53)."""
+    rng = np.random.default_rng(B + 10 * H + 100 * Ci + 1000 * Co + R + 7 * stride)
+    x, w = _i8(rng, (B, H, W, Ci)), _i8(rng, (Co, R, R, Ci))
+    xt = torch.from_numpy(x.astype(np.float64)).permute(0, 3, 1, 2)
+    wt = torch.from_numpy(w.astype(np.float64)).permute(0, 3, 1, 2)
+    want = torch.nn.functional.conv2d(xt, wt, padding=pad, stride=stride).permute(0, 2, 3, 1).numpy()
+    y = oref.conv_fwd_acc(x, w, pad, stride)
+    assert y.shape == want.shape == (B,) + oref.conv_out_hw(H, W, R, R, pad, stride) + (Co,)
+    assert np.array_equal(y, want.astype(np.int64))
+    e = _i8(rng, y.shape)
+    et = torch.from_numpy(e.astype(np.float64)).permute(0, 3, 1, 2)
+    # input rows the strided windows never reach get no error: output_padding restores the input size
+    Ho, Wo = y.shape[1:3]
+    op = (H - ((Ho - 1) * stride - 2 * pad + R), W - ((Wo - 1) * stride - 2 * pad + R))
+    ex = torch.nn.functional.conv_transpose2d(et, wt, padding=pad, stride=stride, output_padding=op)
+    assert np.array_equal(oref.conv_dgrad_acc(e, w, (H, W), pad, stride),
+                          ex.permute(0, 2, 3, 1).numpy().astype(np.int64))
+    gw = torch.nn.grad.conv2d_weight(xt, wt.shape, et, padding=pad, stride=stride).permute(0, 2, 3, 1).numpy()
+    assert np.array_equal(oref.conv_wgrad_acc(x, e, (R, R), pad, stride), gw.astype(np.int64))
+    # exact adjoint identities in integers
+    lhs = int((y * e.astype(np.int64)).sum())
+    assert lhs == int((oref.conv_dgrad_acc(e, w, (H, W), pad, stride) * x.astype(np.int64)).sum())
+    assert lhs == int((oref.conv_wgrad_acc(x, e, (R, R), pad, stride) * w.astype(np.int64)).sum())
+
+
+def test_strided_conv_hand_case(oref):
+    """1-D in effect: x = [1..5] on a 1 x 5 image, taps [1, 10, 100] (1 x 3), pad 1, stride 2.
+    Windows are centred on x[0], x[2], x[4]: y = [10*1 + 100*2, 2 + 10*3 + 100*4, 4 + 10*5]."""
+    x = np.arange(1, 6, dtype=np.int8).reshape(1, 1, 5, 1)
+    w = np.zeros((1, 3, 3, 1), np.int8)
+    w[0, 1, :, 0] = [1, 10, 100]
+    y = oref.conv_fwd_acc(x, w, 1, 2)
+    assert y.shape == (1, 1, 3, 1) and y.reshape(-1).tolist() == [210, 432, 54]
+    e = np.array([1, 2, 3], np.int8).reshape(1, 1, 3, 1)
+    # ex[j] collects e[i] * w[t] with 2 i + t - 1 == j
+    assert oref.conv_dgrad_acc(e, w, (1, 5), 1, 2).reshape(-1).tolist() == [10, 100 + 2, 20, 200 + 3, 30]
+    g = oref.conv_wgrad_acc(x, e, (3, 3), 1, 2)
+    assert g[0, 1, :, 0].tolist() == [2 * 2 + 3 * 4, 1 + 2 * 3 + 3 * 5, 2 + 2 * 4]
+    assert int(np.abs(g[0, 0]).sum()) == 0 and int(np.abs(g[0, 2]).sum()) == 0
+
+
+def test_weight_gradient_loop_order_does_not_matter(oref):
+    """The oracle's weight gradient runs the pixels as outer loops; the same sums with the pixel loops
+    innermost (the formula read literally), in pure Python on a small case."""
+    rng = np.random.default_rng(21)
+    B, H, W, Ci, Co, R, pad, stride = 2, 5, 6, 3, 2, 3, 1, 1
+    x, e = _i8(rng, (B, H, W, Ci)), _i8(rng, (B, H, W, Co))
+    want = np.zeros((Co, R, R, Ci), np.int64)
+    for co in range(Co):
+        for r in range(R):
+            for t in range(R):
+                for ci in range(Ci):
+                    s = 0
+                    for b in range(B):
+                        for i in range(H):
+                            for j in range(W):
+                                ii, jj = i + r - pad, j + t - pad
+                                if 0 <= ii < H and 0 <= jj < W:
+                                    s += int(e[b, i, j, co]) * int(x[b, ii, jj, ci])
+                    want[co, r, t, ci] = s
+    assert np.array_equal(oref.conv_wgrad_acc(x, e, (R, R), pad, stride), want)
+
+
 def test_conv_adjoint_identities(oref):
     """<fwd(x,w), e> = <x, dgrad(e,w)> = <w, wgrad(x,e)>, exactly, in integers."""
     rng = np.random.default_rng(11)
