@@ -431,7 +431,8 @@ def run_ours(args):
     input_digests = {"x": hashlib.sha256(memoryview(x).cast("B")).hexdigest()[:16],
                      "labels": hashlib.sha256(memoryview(labels).cast("B")).hexdigest()[:16],
                      "weights": wh.hexdigest()[:16]}      # guards against drift of the seeded generator
-    tr = NitiTrainer(niti, net, weights, fused_update=args.fused_update, pool_codes=args.pool_codes)
+    tr = NitiTrainer(niti, net, weights, fused_update=args.fused_update, pool_codes=args.pool_codes,
+                     pool_fused=args.pool_fused)
     # Config 2 is "trained for 100 integer steps": consecutive steps on fresh mini-batches with the weights
     # carried over.  The other configs time ONE step K times: every iteration restores the seeded weights
     # (device-to-device copies inside the timed region) and repeats the same step; repeated steps on
@@ -608,6 +609,7 @@ def run_ours(args):
                              "weights restored to the seeded initial values before every step"),
                    "launch": "cuda-graph replay" if args.graph else "eager",
                    "weight_update": "fused with the weight gradient" if args.fused_update else "separate call",
+                   "max_pool_forward": "in the convolution's epilogue" if tr.pool_fused else "separate pass",
                    "parallelism": "replicas" if world > 1 else "single",
                    "inputs_sha256_16": input_digests},
         "outputs": out_digests,
@@ -684,6 +686,8 @@ def main():
     ap.add_argument("--per-launch", action="store_true",
                     help="one eager step with a CUDA event pair around every tensor-core multiply")
     ap.add_argument("--full-sweep", action="store_true", help="with --sweep: time the second operand set on every shape")
+    ap.add_argument("--no-pool-fused", dest="pool_fused", action="store_false",
+                    help="separate max-pool passes in the forward step instead of pooling in the convolution's epilogue")
     ap.add_argument("--sustain-seconds", type=float, default=3.0,
                     help="also replay the step for this many seconds and report the sustained rate (0: skip)")
     ap.add_argument("--cpu-baseline-json", action="store_true", help=argparse.SUPPRESS)

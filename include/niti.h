@@ -180,6 +180,19 @@ int niti_conv_fwd(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s
                   int H, int W, int Cin, int Cout, int R, int S, int pad, int relu, int round_mode,
                   void *ws, size_t ws_bytes);
 
+/* niti_conv_fwd followed by the 2 x 2 max-pool of its output, in one call
+ * (Sections 3.2-3.3 fuse what follows a multiply into it; the networks of
+ * Section 4 pool after a ReLU'd convolution): y as niti_conv_fwd, y_pool
+ * [B][Ho/2][Wo/2][Cout] = niti_maxpool2_fwd(y).  Ho and Wo must be even.  With
+ * relu != 0, Cout a multiple of 32 and 32-byte aligned y / y_pool the
+ * tensor-core kernel's epilogue writes the pooled tile itself (the four pixels
+ * of a window sit in one warp and are combined with shuffles); otherwise the
+ * pooling kernel runs after the convolution.  Same results either way. */
+int niti_conv_fwd_pool(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x, const int8_t *w,
+                       const int32_t *s_w, int8_t *y, int8_t *y_pool, int32_t *s_y, int32_t *b_y, int B, int H,
+                       int W, int Cin, int Cout, int R, int S, int pad, int relu, int round_mode, void *ws,
+                       size_t ws_bytes);
+
 /* Error back-propagation through the convolution (Algorithm 1, reverse loop):
  *   e32[b][i][j][ci] = sum_{r,s,co} e[b][i-r+pad][j-s+pad][co] * w[co][r][s][ci]
  * rounded to 7 bits.  H, W are the INPUT sizes of the forward convolution;

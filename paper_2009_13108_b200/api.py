@@ -25,7 +25,7 @@ EXPORTS = [
     "niti_set_engine", "niti_set_reduce_hook", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
     "niti_redo_count", "niti_selftest_timeout", "niti_profile_enable", "niti_profile_read_launches",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
-    "niti_conv_dgrad", "niti_conv_wgrad", "niti_conv_fwd_strided", "niti_conv_dgrad_strided", "niti_conv_wgrad_strided",
+    "niti_conv_dgrad", "niti_conv_wgrad", "niti_conv_fwd_pool", "niti_conv_fwd_strided", "niti_conv_dgrad_strided", "niti_conv_wgrad_strided",
     "niti_conv_wgrad_update", "niti_linear_bwd_update", "niti_int_xent", "niti_int_xent_noalloc", "niti_int_sgd_update",
     "niti_relu_fwd",
     "niti_relu_bwd", "niti_maxpool2_fwd", "niti_maxpool2_bwd", "niti_maxpool2_fwd_idx", "niti_maxpool2_bwd_idx",
@@ -76,6 +76,7 @@ def load_library():
     lib.niti_conv_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
     lib.niti_conv_dgrad.argtypes = [vp, vp, vp, vp, vp, vp, vp] + [i32] * 9 + [vp, sz]
     lib.niti_conv_wgrad.argtypes = [vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
+    lib.niti_conv_fwd_pool.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
     lib.niti_conv_fwd_strided.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp] + [i32] * 11 + [vp, sz]
     lib.niti_conv_dgrad_strided.argtypes = [vp, vp, vp, vp, vp, vp, vp] + [i32] * 10 + [vp, sz]
     lib.niti_conv_wgrad_strided.argtypes = [vp, vp, vp, vp, vp, vp] + [i32] * 11 + [vp, sz]
@@ -267,6 +268,23 @@ class Niti:
                                                     _ptr(s_w), _ptr(y), _ptr(s_y), _ptr(b_y), B, H, W, Ci, Co,
                                                     R, S, pad, stride, int(relu), round_mode, ws, wsb))
         return y, s_y, b_y
+
+    def conv_fwd_pool(self, x, s_x, w, s_w, y=None, y_pool=None, s_y=None, b_y=None, pad=1, relu=True,
+                      round_mode=ROUND_PSR):
+        """niti_conv_fwd_pool: the convolution's output and its 2 x 2 max-pool in one call."""
+        B, H, W, Ci = x.shape
+        Co, R, S, _ = w.shape
+        Ho, Wo = H + 2 * pad - R + 1, W + 2 * pad - S + 1
+        y = y if y is not None else torch.empty((B, Ho, Wo, Co), dtype=torch.int8, device=self.device)
+        y_pool = y_pool if y_pool is not None else torch.empty((B, Ho // 2, Wo // 2, Co), dtype=torch.int8,
+                                                               device=self.device)
+        s_y = s_y if s_y is not None else self.scalar()
+        b_y = b_y if b_y is not None else self.scalar()
+        ws, wsb = self._ws_for(OP_CONV_FWD, [B, H, W, Ci, Co, R, S, pad])
+        self._ck(self.lib.niti_conv_fwd_pool(self.h, self._stream(), _ptr(x), _ptr(s_x), _ptr(w), _ptr(s_w),
+                                             _ptr(y), _ptr(y_pool), _ptr(s_y), _ptr(b_y), B, H, W, Ci, Co, R, S,
+                                             pad, int(relu), round_mode, ws, wsb))
+        return y, y_pool, s_y, b_y
 
     def conv_dgrad(self, e, w, in_hw, e_prev=None, relu_mask_src=None, b_e=None, pad=1,
                    round_mode=ROUND_PSR, stride=1):

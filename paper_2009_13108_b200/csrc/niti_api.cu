@@ -169,6 +169,13 @@ static bool fill_conv(GemmProblem &p, int kind, int B, int H, int W, int Ci, int
   return true;
 }
 
+// int32 elements of the accumulator scratch of a fully connected backward call: the larger of the weight
+// gradient [N][K] and the error [M][K] (times its partial slices when the batch is small)
+static size_t linear_bwd_acc_elems(long long M, long long N, long long K) {
+  const size_t a = (size_t)(M * K) * (size_t)niti_partial_slices(GK_FC_DGRAD, M), b = (size_t)(N * K);
+  return a > b ? a : b;
+}
+
 static void fill_fc(GemmProblem &p, int kind, int M, int N, int K) {
   memset(&p, 0, sizeof(p));
   p.kind = kind; p.M = M; p.N = N; p.K = K;
@@ -187,14 +194,14 @@ extern "C" size_t niti_workspace_bytes(int op, const int64_t *d, int nd) {
     case NITI_OP_LINEAR_FWD:
       if (nd != 3 || d[0] <= 0 || d[1] <= 0 || d[2] <= 0) return 0;
       fill_fc(p, GK_FC_FWD, (int)d[0], (int)d[1], (int)d[2]);
-      outs = (size_t)(d[0] * d[1]);
+      outs = (size_t)(d[0] * d[1]) * (size_t)niti_partial_slices(GK_FC_FWD, d[0]);
       extra = niti_tc_scratch_bytes(p);
       break;
     case NITI_OP_LINEAR_BWD_UPDATE:
     case NITI_OP_LINEAR_BWD: {
       if (nd != 3 || d[0] <= 0 || d[1] <= 0 || d[2] <= 0) return 0;
-      size_t a = (size_t)(d[0] * d[2]), b = (size_t)(d[1] * d[2]);
-      outs = a > b ? a : b;
+      size_t b = (size_t)(d[1] * d[2]);
+      outs = linear_bwd_acc_elems(d[0], d[1], d[2]);
       fill_fc(p, GK_FC_DGRAD, (int)d[0], (int)d[1], (int)d[2]);
       fill_fc(p2, GK_FC_WGRAD, (int)d[0], (int)d[1], (int)d[2]);
       size_t e1 = niti_tc_scratch_bytes(p), e2 = niti_tc_scratch_bytes(p2);
@@ -259,10 +266,12 @@ int niti_reduce_after_gemm(niti_ctx *ctx, cudaStream_t st, int kind, int32_t *ac
 // weights in place.  When the int32 accumulators exist (split contractions) the rounding pass does
 // that itself and the int8 gradient is never stored; when the multiply rounds in its own epilogue,
 // `out` is a scratch tensor and the plain update kernel follows.
+int niti_launch_maxpool2_fwd(niti_ctx *ctx, cudaStream_t st, const int8_t *x, int8_t *y, int B, int H, int W, int C);
+
 static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, void *ws, size_t ws_bytes,
                           size_t need, int8_t *out, int mbits, int round_mode, int relu,
                           const int8_t *mask, const int32_t *s_a, const int32_t *s_w, int32_t *s_out,
-                          int32_t *b_out, int8_t *update_w = nullptr) {
+                          int32_t *b_out, int8_t *update_w = nullptr, int8_t *pool_out = nullptr) {
   if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
     return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
   WsHeader *hdr = (WsHeader *)ws;
@@ -271,16 +280,24 @@ static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, 
   ctx->launches++;
   int rc = NITI_ERR_SHAPE;
   bool fused = false;
-  RoundSpec rs = {out, mask, mbits, round_mode, relu, s_a, s_w, s_out, b_out};
-  if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, rs, acc, hdr, &fused);
+  bool pooled = false;
+  RoundSpec rs = {out, mask, mbits, round_mode, relu, s_a, s_w, s_out, b_out, pool_out};
+  if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, rs, acc, hdr, &fused, &pooled);
   if (rc == NITI_ERR_SHAPE) {
     rc = niti_simt_gemm(ctx, st, p, acc, hdr);
     if (rc == NITI_OK) rc = niti_reduce_after_gemm(ctx, st, p.kind, acc, p.gm * p.gn, hdr);
   }
   if (rc != NITI_OK) return rc;
-  if (fused) return update_w ? niti_launch_sgd_update(ctx, st, update_w, out, p.gm * p.gn) : NITI_OK;
-  return niti_launch_round(ctx, st, acc, hdr, out, p.gm * p.gn, mbits, round_mode, relu, mask, s_a, s_w,
+  if (fused) {
+    if (update_w) return niti_launch_sgd_update(ctx, st, update_w, out, p.gm * p.gn);
+  } else {
+    rc = niti_launch_round(ctx, st, acc, hdr, out, p.gm * p.gn, mbits, round_mode, relu, mask, s_a, s_w,
                            s_out, b_out, update_w);
+    if (rc != NITI_OK) return rc;
+  }
+  // the pooled copy of a forward convolution, where the multiply's own epilogue did not write it
+  if (pool_out && !pooled) return niti_launch_maxpool2_fwd(ctx, st, out, pool_out, p.B, p.Ho, p.Wo, p.Co);
+  return NITI_OK;
 }
 
 extern "C" int niti_linear_fwd(niti_ctx *ctx, void *stream, const int8_t *a, const int32_t *s_a,
@@ -326,8 +343,7 @@ static int linear_bwd_impl(niti_ctx *ctx, void *stream, const int8_t *a, const i
   long long e_ld = 0;
   if ((N % 16) != 0 && N >= 32 && ctx->engine != 1) {
     const int pitch = (N + 15) / 16 * 16;
-    size_t a_out = (size_t)M * K, b_out = (size_t)N * K;
-    int8_t *epad = (int8_t *)((char *)ws + NITI_WS_HEADER + round_up((a_out > b_out ? a_out : b_out) * 4, 256));
+    int8_t *epad = (int8_t *)((char *)ws + NITI_WS_HEADER + round_up(linear_bwd_acc_elems(M, N, K) * 4, 256));
     int rcp = niti_launch_pad_pitch(ctx, (cudaStream_t)stream, e, epad, M, N, pitch);
     if (rcp != NITI_OK) return rcp;
     e_tc = epad;
@@ -374,10 +390,10 @@ static int conv_args_ok(int B, int H, int W, int Ci, int Co, int R, int S, int p
          (round_mode == 0 || round_mode == 1);
 }
 
-extern "C" int niti_conv_fwd_strided(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x,
-                                     const int8_t *w, const int32_t *s_w, int8_t *y, int32_t *s_y, int32_t *b_y,
-                                     int B, int H, int W, int Cin, int Cout, int R, int S, int pad, int stride,
-                                     int relu, int round_mode, void *ws, size_t ws_bytes) {
+static int conv_fwd_impl(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x, const int8_t *w,
+                         const int32_t *s_w, int8_t *y, int8_t *y_pool, int32_t *s_y, int32_t *b_y, int B, int H,
+                         int W, int Cin, int Cout, int R, int S, int pad, int stride, int relu, int round_mode,
+                         void *ws, size_t ws_bytes) {
   if (!ctx) return NITI_ERR_ARG;
   GemmProblem p;
   memset(&p, 0, sizeof(p));
@@ -403,10 +419,32 @@ extern "C" int niti_conv_fwd_strided(niti_ctx *ctx, void *stream, const int8_t *
     GemmProblem q;
     fill_fc(q, GK_FC_FWD, (int)M, Cout, 32);
     q.p0 = xcol; q.p1 = wcol;
-    return run_gemm_round(ctx, st, q, ws, ws_bytes, need, y, 7, round_mode, relu, nullptr, s_x, s_w, s_y, b_y);
+    rc = run_gemm_round(ctx, st, q, ws, ws_bytes, need, y, 7, round_mode, relu, nullptr, s_x, s_w, s_y, b_y);
+    if (rc != NITI_OK || !y_pool) return rc;
+    return niti_launch_maxpool2_fwd(ctx, st, y, y_pool, B, p.Ho, p.Wo, Cout);
   }
   return run_gemm_round(ctx, (cudaStream_t)stream, p, ws, ws_bytes, need, y, 7, round_mode, relu, nullptr,
-                        s_x, s_w, s_y, b_y);
+                        s_x, s_w, s_y, b_y, nullptr, y_pool);
+}
+
+extern "C" int niti_conv_fwd_strided(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x,
+                                     const int8_t *w, const int32_t *s_w, int8_t *y, int32_t *s_y, int32_t *b_y,
+                                     int B, int H, int W, int Cin, int Cout, int R, int S, int pad, int stride,
+                                     int relu, int round_mode, void *ws, size_t ws_bytes) {
+  return conv_fwd_impl(ctx, stream, x, s_x, w, s_w, y, nullptr, s_y, b_y, B, H, W, Cin, Cout, R, S, pad, stride, relu,
+                       round_mode, ws, ws_bytes);
+}
+
+extern "C" int niti_conv_fwd_pool(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x, const int8_t *w,
+                                  const int32_t *s_w, int8_t *y, int8_t *y_pool, int32_t *s_y, int32_t *b_y, int B,
+                                  int H, int W, int Cin, int Cout, int R, int S, int pad, int relu, int round_mode,
+                                  void *ws, size_t ws_bytes) {
+  if (!ctx) return NITI_ERR_ARG;
+  const int Ho = H + 2 * pad - R + 1, Wo = W + 2 * pad - S + 1;
+  if (!y_pool || Ho <= 0 || Wo <= 0 || (Ho & 1) || (Wo & 1) || misaligned16(y_pool))
+    return niti_fail(ctx, NITI_ERR_ARG, "niti_conv_fwd_pool: bad argument (output height and width must be even)");
+  return conv_fwd_impl(ctx, stream, x, s_x, w, s_w, y, y_pool, s_y, b_y, B, H, W, Cin, Cout, R, S, pad, 1, relu,
+                       round_mode, ws, ws_bytes);
 }
 
 extern "C" int niti_conv_fwd(niti_ctx *ctx, void *stream, const int8_t *x, const int32_t *s_x,
@@ -481,7 +519,7 @@ static int conv_wgrad_impl(niti_ctx *ctx, void *stream, const int8_t *x, const i
     fill_fc(q, GK_FC_WGRAD, (int)M, Cout, 32);     // rows M are the contraction
     q.p0 = e; q.p1 = xcol;
     bool fused = false;
-    RoundSpec none = {nullptr, nullptr, m_u, round_mode, 0, nullptr, nullptr, nullptr, nullptr};
+    RoundSpec none = {nullptr, nullptr, m_u, round_mode, 0, nullptr, nullptr, nullptr, nullptr, nullptr};
     const int saved = ctx->engine;
     if (saved == 0) ctx->engine = 4;               // int32 accumulators are needed here, not a fused store
     rc = niti_tc_gemm(ctx, st, q, none, acc32, hdr, &fused);

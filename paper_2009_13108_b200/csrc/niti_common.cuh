@@ -144,6 +144,16 @@ struct GemmProblem {
   long long ld0;
 };
 
+// Fully connected forward / error multiplies with at most 128 output rows (weight streaming: the
+// contraction is split over the SMs) keep up to this many int32 partial tensors in the scratch, one
+// per split; 1 for every other multiply.  The workspace query reserves room accordingly.
+#define NITI_PARTIAL_SLICES 16
+static inline int niti_partial_slices(int kind, long long gm) {
+  return ((kind == 0 || kind == 1) && gm <= 128) ? NITI_PARTIAL_SLICES : 1;   // GK_FC_FWD, GK_FC_DGRAD
+}
+// acc holds `splits` partial tensors of n int32 each: adds them into the first, takes max |sum| into
+// hdr->maxabs32 and raises NITI_DEV_ACC_RANGE when the magnitudes of an element's partial sums add up to 2^31
+int niti_launch_sum_partials(niti_ctx *ctx, cudaStream_t st, int32_t *acc, int splits, long long n, WsHeader *hdr);
 int niti_reduce_after_gemm(niti_ctx *ctx, cudaStream_t st, int kind, int32_t *acc, long long n, WsHeader *hdr);
 // max |acc| into hdr->maxabs32; splits > 1: also adds up the split maxima of the header and raises
 // NITI_DEV_ACC_RANGE when an accumulator may have left the int32 range
@@ -157,12 +167,14 @@ struct RoundSpec {
   int mbits, round_mode, relu;
   const int32_t *s_a, *s_w;
   int32_t *s_out, *b_out;
+  int8_t *pool_out;        // optional (may be null): 2 x 2 max-pool of `out`, forward convolutions with ReLU
 };
 // Tensor-core engine (tcgen05); returns NITI_ERR_SHAPE if the shape is not eligible.  *fused is set
 // when the kernel also did the bit-width / shift / round / store (nothing is left to do); otherwise
 // acc holds the int32 accumulators and hdr->maxabs32 their max magnitude.
+// *pooled (may be null) is set when the kernel's epilogue also wrote r.pool_out.
 int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, const RoundSpec &r, int32_t *acc,
-                 WsHeader *hdr, bool *fused);
+                 WsHeader *hdr, bool *fused, bool *pooled = nullptr);
 size_t niti_tc_scratch_bytes(const GemmProblem &p);
 
 // Epilogue pass: b from hdr->maxabs32, bp = max(0, b - mbits), out = Round(acc) with optional ReLU

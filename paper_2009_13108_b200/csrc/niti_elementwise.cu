@@ -1055,20 +1055,24 @@ extern "C" int niti_relu_bwd(niti_ctx *ctx, void *stream, const int8_t *y, const
   return NITI_OK;
 }
 
+int niti_launch_maxpool2_fwd(niti_ctx *ctx, cudaStream_t st, const int8_t *x, int8_t *y, int B, int H, int W, int C) {
+  bool vec = (C % 16 == 0) && !(((uintptr_t)x | (uintptr_t)y) & 15);
+  long long items = (long long)B * (H / 2) * (W / 2) * (vec ? C / 16 : C);
+  if (vec)
+    maxpool2_fwd_kernel<16><<<ew_blocks(ctx, items), 256, 0, st>>>(x, y, B, H, W, C);
+  else
+    maxpool2_fwd_kernel<1><<<ew_blocks(ctx, items), 256, 0, st>>>(x, y, B, H, W, C);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
 extern "C" int niti_maxpool2_fwd(niti_ctx *ctx, void *stream, const int8_t *x, int8_t *y, int B, int H,
                                  int W, int C) {
   if (!ctx) return NITI_ERR_ARG;
   if (!x || !y || B <= 0 || H <= 0 || W <= 0 || C <= 0 || (H & 1) || (W & 1))
     return niti_fail(ctx, NITI_ERR_ARG, "niti_maxpool2_fwd: bad argument (H and W must be even)");
-  bool vec = (C % 16 == 0) && !(((uintptr_t)x | (uintptr_t)y) & 15);
-  long long items = (long long)B * (H / 2) * (W / 2) * (vec ? C / 16 : C);
-  if (vec)
-    maxpool2_fwd_kernel<16><<<ew_blocks(ctx, items), 256, 0, (cudaStream_t)stream>>>(x, y, B, H, W, C);
-  else
-    maxpool2_fwd_kernel<1><<<ew_blocks(ctx, items), 256, 0, (cudaStream_t)stream>>>(x, y, B, H, W, C);
-  ctx->launches++;
-  NITI_CUDA_TRY(ctx, cudaGetLastError());
-  return NITI_OK;
+  return niti_launch_maxpool2_fwd(ctx, (cudaStream_t)stream, x, y, B, H, W, C);
 }
 
 extern "C" int niti_maxpool2_fwd_idx(niti_ctx *ctx, void *stream, const int8_t *x, int8_t *y, uint8_t *idx, int B,

@@ -230,6 +230,48 @@ int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long 
   return NITI_OK;
 }
 
+// Sum of the partial tensors of a split contraction (one slice of n int32 per split) into the first
+// slice, the max magnitude of the sums, and the int32 range check: the magnitudes of an element's
+// partial sums bound its total, and every partial sum is exact (a split is at most NITI_SPLIT_MAX_K long).
+__global__ void __launch_bounds__(256)
+sum_partials_kernel(int32_t *__restrict__ acc, int splits, long long n, WsHeader *hdr, uint32_t *status) {
+  unsigned mx = 0;
+  unsigned long long worst = 0;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    int s = acc[i];
+    unsigned long long bound = (unsigned)abs(s);
+    for (int k = 1; k < splits; ++k) {
+      const int v = acc[(long long)k * n + i];
+      s += v;
+      bound += (unsigned)abs(v);
+    }
+    acc[i] = s;
+    const unsigned a = (unsigned)abs(s);
+    mx = a > mx ? a : mx;
+    worst = bound > worst ? bound : worst;
+  }
+  if (worst >= 0x80000000ull) atomicOr(status, NITI_DEV_ACC_RANGE);
+  mx = __reduce_max_sync(0xffffffffu, mx);
+  __shared__ unsigned smax[8];
+  if ((threadIdx.x & 31) == 0) smax[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < 8; ++i) mx = smax[i] > mx ? smax[i] : mx;
+    if (mx) atomicMax(&hdr->maxabs32, mx);
+  }
+}
+
+int niti_launch_sum_partials(niti_ctx *ctx, cudaStream_t st, int32_t *acc, int splits, long long n, WsHeader *hdr) {
+  long long blocks = (n + 255) / 256;
+  if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+  if (blocks < 1) blocks = 1;
+  sum_partials_kernel<<<(unsigned)blocks, 256, 0, st>>>(acc, splits, n, hdr, ctx->d_status);
+  ctx->launches++;
+  NITI_CUDA_TRY(ctx, cudaGetLastError());
+  return NITI_OK;
+}
+
 int niti_simt_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, int32_t *acc, WsHeader *hdr) {
   Addr q;
   q.p0 = p.p0; q.p1 = p.p1; q.kind = p.kind;

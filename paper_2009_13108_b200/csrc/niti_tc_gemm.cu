@@ -105,6 +105,8 @@ struct TcParams {
   int mbits, round_mode, relu;
   unsigned spec_mul256;         // the sampled max is scaled by this / 256 before taking its bit length
   int spec_tag;                 // identifies the call site (its b_out scalar) in the table of estimate errors
+  int pool;                     // 1: the epilogue also stores the 2 x 2 max-pool of the (ReLU'd) output tile
+  int pool_xh;                  // lane distance of the pixel one image row below (the pixel to the right is lane ^ 1)
   int single_wave;              // every CTA has at most one tile: the sample is the whole tensor, the shift
                                 // is exact, and the last CTA to finish publishes b and the exponent
 };
@@ -120,7 +122,13 @@ struct TcParams {
 //                 the common case costs one multiply and no int32 traffic)
 //  EPI_KNOWN_B    bit-width known (hdr->maxabs32): round and store directly.  The kernel returns at
 //                 once when the speculative pass was right.
-enum { EPI_SPILL = 0, EPI_ATOMIC = 1, EPI_SPECULATE = 2, EPI_KNOWN_B = 3 };
+//  EPI_PARTIAL    split contraction of a multiply with few output rows (fully connected layers at batch
+//                 <= 128): every split stores its int32 partial tile to its own slice of the scratch
+//                 (plain 16-byte stores) and a small kernel adds the slices and takes the max.  An SM
+//                 retires only about 1.6 atomic additions per cycle, so the 64 x 256 partial tile of a
+//                 weight-streaming multiply took 5 us to add atomically, as long as a 4 MB layer takes
+//                 to stream.
+enum { EPI_SPILL = 0, EPI_ATOMIC = 1, EPI_SPECULATE = 2, EPI_KNOWN_B = 3, EPI_PARTIAL = 4 };
 
 
 // ------------------------------------------------------------------------------------------
@@ -454,6 +462,31 @@ __device__ __forceinline__ unsigned bytes_gt0(unsigned b) {
   return r;
 }
 
+// Byte-wise maximum of two words whose bytes are all in [0, 127] (ReLU outputs): bit 7 of
+// (a | 0x80..) - b is set per byte exactly where a >= b, and no byte borrows from its neighbour.
+__device__ __forceinline__ unsigned bytes_max_u7(unsigned a, unsigned b) {
+  const unsigned t = (a | 0x80808080u) - b;
+  unsigned m;
+  asm("prmt.b32 %0, %1, %1, 0xba98;" : "=r"(m) : "r"(t));   // 0xff where a >= b
+  return (a & m) | (b & ~m);
+}
+// 2 x 2 max-pool of a 32-channel chunk held one pixel per lane: the window's other pixels are the lanes
+// lane ^ 1 (next column) and lane ^ xh (next image row); every lane ends up with its window's maximum.
+__device__ __forceinline__ void pool_chunk32(unsigned (&w8)[8], int xh) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    unsigned a = w8[j];
+    a = bytes_max_u7(a, __shfl_xor_sync(0xffffffffu, a, 1));
+    a = bytes_max_u7(a, __shfl_xor_sync(0xffffffffu, a, xh));
+    w8[j] = a;
+  }
+}
+__device__ __forceinline__ void store32(int8_t *dst, const unsigned (&w8)[8]) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"l"(dst), "r"(w8[0]), "r"(w8[1]), "r"(w8[2]), "r"(w8[3]), "r"(w8[4]), "r"(w8[5]), "r"(w8[6]), "r"(w8[7])
+               : "memory");
+}
+
 // n / d with the host's reciprocal (exact while n * d < 2^32, which the host checked), else a division
 __device__ __forceinline__ int div_tiles(int n, int d, unsigned magic) {
   return magic ? (int)__umulhi((unsigned)n, magic) : n / d;
@@ -673,7 +706,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const TcParams p, int32_t *__restrict__ acc, WsHeader *hdr, uint32_t *status,
                int8_t *__restrict__ out8, const int8_t *__restrict__ mask8, const int32_t *s_a,
-               const int32_t *s_w, int32_t *s_out, int32_t *b_out, int32_t *spec_slot) {
+               const int32_t *s_w, int32_t *s_out, int32_t *b_out, int32_t *spec_slot, int8_t *__restrict__ pool8) {
   if (p.epi_mode == EPI_SPECULATE && !p.single_wave) {
     // the follow-up launch may be scheduled now (it is launched as a programmatic dependent): its CTAs
     // take the SMs as this grid's CTAs retire and wait there for the whole grid to finish
@@ -1201,6 +1234,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         long long rem = p.gn - col0;
         ncols_valid = rem < p.bn ? (int)rem : p.bn;
       }
+      // fused 2 x 2 max-pool (convolutions only): this lane's pixel and the row of its window in the pooled tensor
+      long long pool_row = 0;
+      if (p.pool) {
+        const long long pw = out_row % p.PW, t2 = out_row / p.PW;
+        const long long ph = t2 % p.PH, pb = t2 / p.PH;
+        pool_row = (pb * (p.PH >> 1) + (ph >> 1)) * (p.PW >> 1) + (pw >> 1);
+      }
       if (!mbar_wait(tfull0 + 8 * buf, tpar, &abort_flag, status)) { ok = false; break; }
       tc_fence_after();
       const unsigned tm_row = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * (unsigned)p.bn;
@@ -1233,8 +1273,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         pmx = __reduce_max_sync(0xffffffffu, pmx);
         if (lane == 0 && pmx) atomicMax(niti_split_max(hdr) + split, pmx);
-      } else if (p.epi_mode <= EPI_ATOMIC) {
+      } else if (p.epi_mode <= EPI_ATOMIC || p.epi_mode == EPI_PARTIAL) {
         int32_t *dst = acc + out_row * p.gn + col0;
+        if (p.epi_mode == EPI_PARTIAL) dst += (long long)split * p.gm * p.gn;      // this split's slice
         const bool vec_ok = ((p.gn & 3) == 0) && ((col0 & 3) == 0);
         unsigned pmx = 0;                                      // largest partial-sum magnitude of this item
         for (int c = 32 * chunk_phase; c < p.bn; c += 32 * wpq) {
@@ -1416,6 +1457,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int v[32];
             const bool rok = row_ok && orow < p.gm;
             unsigned m[8];
+            unsigned pw8[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};     // pooling input of lanes outside the tensor
             if (mrow && rok)
               asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                            : "=r"(m[0]), "=r"(m[1]), "=r"(m[2]), "=r"(m[3]), "=r"(m[4]), "=r"(m[5]), "=r"(m[6]), "=r"(m[7])
@@ -1434,6 +1476,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                            ::"l"(drow + cc), "r"(w8[0]), "r"(w8[1]), "r"(w8[2]), "r"(w8[3]), "r"(w8[4]), "r"(w8[5]),
                              "r"(w8[6]), "r"(w8[7])
                            : "memory");
+              if (p.pool) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) pw8[j] = w8[j];
+              }
+            }
+            if (p.pool) {                          // (warp-uniform: every lane takes part in the exchange)
+              pool_chunk32(pw8, p.pool_xh);
+              if (rok && (lane & (1 | p.pool_xh)) == 0) store32(pool8 + pool_row * p.gn + col0 + cc, pw8);
             }
             cc += cstep;
             while (cc >= bn_mma) { cc -= bn_mma; orow += BM; drow += sub_stride; if (mrow) mrow += sub_stride; }
@@ -1521,8 +1571,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // executes only what changes (measured on the first layer: the general loop above spends a third
     // of its integer instructions on tests whose outcome is the same for every tile).
     if (ok && lean_item >= 0) {
-      auto lean = [&](auto relu_c, auto mask_c, auto batched_c) {
+      auto lean = [&](auto relu_c, auto mask_c, auto batched_c, auto pool_c) {
         constexpr bool RELU = decltype(relu_c)::value, MASK = decltype(mask_c)::value, BATCHED = decltype(batched_c)::value;
+        constexpr bool POOL = decltype(pool_c)::value;       // fused 2 x 2 max-pool of the ReLU'd tile
+        const int pool_xh = p.pool_xh;
+        const bool pool_lane = (lane & (1 | pool_xh)) == 0;  // the window's top-left pixel stores the maximum
         const int kind = p.halo ? 0 : ((p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) ? 1 : 2);
         const int istep = item_step * egroups, nbuf = p.nbuf, bn = p.bn, n_tiles_n = p.n_tiles_n;
         const int cstep = 32 * wpq, c_first = 32 * chunk_phase;
@@ -1538,10 +1591,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (ebuf >= (unsigned)nbuf) { ebuf -= (unsigned)nbuf; epar ^= 1u; }
           long long out_row;
           bool row_ok;
+          long long pool_row = 0;
           if (kind == 0) {
             const int w = h_wt * 8 + (row_in_tile & 7), h = h_ht * 16 + (row_in_tile >> 3);
             row_ok = w < p.PW && h < p.PH;
             out_row = ((long long)h_bt * p.PH + h) * p.PW + w;
+            if (POOL) pool_row = ((long long)h_bt * (p.PH >> 1) + (h >> 1)) * (p.PW >> 1) + (w >> 1);
             h_wt += egroups;
             while (h_wt >= p.w_tiles) { h_wt -= p.w_tiles; if (++h_ht == p.h_tiles) { h_ht = 0; ++h_bt; } }
           } else if (kind == 1) {
@@ -1550,6 +1605,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int w = w0 + r_ww, h = h0 + r_hh, b = b0 + r_bb;
             row_ok = w < p.PW && h < p.PH && b < p.PB;
             out_row = ((long long)b * p.PH + h) * p.PW + w;
+            if (POOL) pool_row = ((long long)b * (p.PH >> 1) + (h >> 1)) * (p.PW >> 1) + (w >> 1);
           } else {
             out_row = (long long)(mu * CTAS + (int)rank) * (BM * p.mrep) + row_in_tile;
             row_ok = out_row < gm;
@@ -1567,6 +1623,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const long long row_off = out_row * gn + col0;
           int8_t *drow = out8 + row_off;
           const int8_t *mrow = MASK ? mask8 + row_off : nullptr;
+          int8_t *prow = POOL ? pool8 + pool_row * gn + col0 : nullptr;
           long long orow = out_row;
           int cc = c_first;
           if (BATCHED) while (cc >= bn_mma) { cc -= bn_mma; orow += BM; drow += sub_stride; if (MASK) mrow += sub_stride; }
@@ -1579,17 +1636,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                            : "=r"(m[0]), "=r"(m[1]), "=r"(m[2]), "=r"(m[3]), "=r"(m[4]), "=r"(m[5]), "=r"(m[6]), "=r"(m[7])
                            : "l"(mrow + cc));
             tc_ld32(tm_row + (unsigned)c, v);
+            unsigned w8[8];
+            if (POOL) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) w8[j] = 0u;          // lanes outside the tensor pool zeros
+            }
             if (rok) {
-              unsigned w8[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 w8[j] = round_pack4_aligned<RELU>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, ex_all);
                 if (MASK) w8[j] &= bytes_gt0(m[j]);
               }
-              asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                           ::"l"(drow + cc), "r"(w8[0]), "r"(w8[1]), "r"(w8[2]), "r"(w8[3]), "r"(w8[4]), "r"(w8[5]),
-                             "r"(w8[6]), "r"(w8[7])
-                           : "memory");
+              store32(drow + cc, w8);
+            }
+            if (POOL) {                                        // (warp-uniform: all lanes exchange)
+              pool_chunk32(w8, pool_xh);
+              if (rok && pool_lane) store32(prow + cc, w8);
             }
             cc += cstep;
             if (BATCHED) while (cc >= bn_mma) { cc -= bn_mma; orow += BM; drow += sub_stride; if (MASK) mrow += sub_stride; }
@@ -1605,9 +1667,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       using T = std::true_type;
       using F = std::false_type;
       const bool relu = p.relu != 0, masked = mask8 != nullptr, batched = p.mrep > 1;
-      if (batched) { if (relu) lean(T{}, F{}, T{}); else lean(F{}, F{}, T{}); }      // (row-batched: forward only)
-      else if (relu) { if (masked) lean(T{}, T{}, F{}); else lean(T{}, F{}, F{}); }
-      else { if (masked) lean(F{}, T{}, F{}); else lean(F{}, F{}, F{}); }
+      if (batched) { if (relu) lean(T{}, F{}, T{}, F{}); else lean(F{}, F{}, T{}, F{}); }      // (row-batched: forward only)
+      else if (p.pool) lean(T{}, F{}, F{}, T{});                                               // (pooling: ReLU, no mask)
+      else if (relu) { if (masked) lean(T{}, T{}, F{}, F{}); else lean(T{}, F{}, F{}, F{}); }
+      else { if (masked) lean(F{}, T{}, F{}, F{}); else lean(F{}, F{}, F{}, F{}); }
       mx |= ex_all.magnitude_bits();
     }
     if (p.epi_mode == EPI_SPILL || p.epi_mode == EPI_SPECULATE) {
@@ -2060,7 +2123,10 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
     // four k-blocks
     double best = 1e30;
     int best_s = 1;
-    const int max_s = p.kb_total / 4;
+    int max_s = p.kb_total / 4;
+    // (multiplies with few output rows keep their splits' partial tiles in separate slices of the scratch)
+    const int slices = niti_partial_slices(g.kind, g.gm);
+    if (slices > 1 && max_s > slices) max_s = slices;
     for (int sp = 1; sp <= max_s && sp <= 4 * units; ++sp) {
       const long long it = tiles * sp;
       const long long waves = (it + units - 1) / units;
@@ -2226,7 +2292,7 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
     q.spec_tag = (int)(unsigned)(key | 1u);
   }
   NITI_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, tc_gemm_kernel<CTAS>, ma, mb, q, acc, hdr, ctx->d_status, r.out, r.mask,
-                                        r.s_a, r.s_w, r.s_out, r.b_out, slot));
+                                        r.s_a, r.s_w, r.s_out, r.b_out, slot, r.pool_out));
   ctx->launches++;
   ctx->tc_launches++;
   if (CTAS == 2) ctx->tc2_launches++;
@@ -2234,10 +2300,11 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
 }
 
 int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const RoundSpec &r, int32_t *acc,
-                 WsHeader *hdr, bool *fused) {
+                 WsHeader *hdr, bool *fused, bool *pooled) {
   TcParams p;
   CUtensorMap ma, mb;
   *fused = false;
+  if (pooled) *pooled = false;
   // engine 0: pairs of CTAs (cta_group::2) when there are enough 256-row tiles to fill the GPU.
   // Test switches: 2 / 3 force the single-CTA / paired kernel, 4 keeps the int32 spill epilogue.
   // Test switches: 5 disables the halo mode of small-channel convolutions.
@@ -2282,9 +2349,24 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
   p.round_mode = r.round_mode;
   p.relu = r.relu;
   p.epi_mode = (p.splits > 1 || p.halo == 2) ? EPI_ATOMIC : ((ctx->engine == 4 || dp_sum) ? EPI_SPILL : EPI_SPECULATE);
+  if (p.epi_mode == EPI_ATOMIC && niti_partial_slices(g.kind, g.gm) > 1 && p.splits <= niti_partial_slices(g.kind, g.gm) &&
+      !p.halo && p.mrep == 1)
+    p.epi_mode = EPI_PARTIAL;
   if (p.epi_mode == EPI_ATOMIC) {
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(acc, 0, sizeof(int32_t) * (size_t)(g.gm * g.gn), st));
     ctx->launches++;
+  }
+  // Fused 2 x 2 max-pool: the fused epilogue of a forward convolution with ReLU also stores the pooled
+  // tile when every pooling window lies inside one warp's 32 pixels (8 x 16 pixel tiles of the
+  // resident-weights mode, or pixel boxes at most 16 wide and at least 2 high) and the rows are whole,
+  // 32-byte aligned chunks.  Otherwise the caller runs the pooling kernel.
+  p.pool = 0;
+  if (pooled && r.pool_out && g.kind == GK_CONV_FWD && r.relu && !r.mask && p.epi_mode == EPI_SPECULATE &&
+      p.mrep == 1 && (p.PW % 2) == 0 && (p.PH % 2) == 0 && (g.gn % 32) == 0 && ((uintptr_t)r.out & 31) == 0 &&
+      ((uintptr_t)r.pool_out & 31) == 0 && r.mbits == 7) {
+    if (p.halo == 1) { p.pool = 1; p.pool_xh = 8; }
+    else if (!p.halo && p.Wt >= 2 && p.Wt <= 16 && p.Ht >= 2) { p.pool = 1; p.pool_xh = p.Wt; }
+    *pooled = p.pool != 0;
   }
   const bool prof = ctx->profile_on && ctx->prof_ev && ctx->prof_used < NITI_PROF_MAX;
   if (prof) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st);
@@ -2307,6 +2389,11 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
     cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st);
     ctx->prof_ops[ctx->prof_used] = 2.0 * (double)g.gm * (double)g.gn * (double)g.gk;
     ctx->prof_used++;
+  }
+  if (p.epi_mode == EPI_PARTIAL) {     // adds the splits' slices into the first one and takes the max magnitude
+    rc = niti_launch_sum_partials(ctx, st, acc, p.splits, g.gm * g.gn, hdr);
+    if (rc != NITI_OK || !dp) return rc;
+    return niti_reduce(ctx, st, &hdr->maxabs32, 1, NITI_REDUCE_MAX_U32);
   }
   if (p.epi_mode == EPI_ATOMIC) {
     if (dp_sum) {                      // sums over the ranks first, then their max

@@ -13,7 +13,7 @@ from .api import Niti, ROUND_PSR
 
 class NitiTrainer:
     def __init__(self, niti: Niti, net, weights, round_mode: int = ROUND_PSR, fused_update: bool = False,
-                 pool_codes: bool = False, dist_group=None, data_parallel: bool = False):
+                 pool_codes: bool = False, dist_group=None, data_parallel: bool = False, pool_fused: bool = True):
         """``net``: an object with ``batch``, ``in_shape``, ``s_in``, ``m_u`` and ``layers`` (dicts
         with op in {"conv", "pool", "fc"}); ``weights``: int8 host arrays / tensors per weight
         layer ([Cout,3,3,Cin] or [N,K]).  ``fused_update``: weight gradient and weight update in one
@@ -29,6 +29,9 @@ class NitiTrainer:
         self.net = net
         self.round_mode = round_mode
         self.fused_update = fused_update
+        # ``pool_fused``: a convolution that is followed by a max-pool writes the pooled tensor from its own
+        # epilogue (niti_conv_fwd_pool) and the separate pooling pass of the forward step is dropped
+        self.pool_fused = pool_fused and not pool_codes
         # exact data parallelism: ``net.batch`` is this rank's share of the batch; bit-widths and
         # weight-gradient sums are combined over the ranks of ``dist_group`` (None = the default group),
         # so every rank holds the weights one process with the whole batch would have
@@ -154,11 +157,19 @@ class NitiTrainer:
         n, net = self.n, self.net
         a, s = self.x, self.s_in
         wi = 0
+        pooled_by_conv = -1
         for li, L in enumerate(net.layers):
             out = self.acts[li]
             if L["op"] == "conv":
-                n.conv_fwd(a, s, self.weights[wi], self.s_w[li], y=out, s_y=self.s_act[li],
-                           b_y=self.b_fwd[li], pad=1, relu=L["relu"], round_mode=self.round_mode)
+                nxt_is_pool = li + 1 < len(net.layers) and net.layers[li + 1]["op"] == "pool"
+                if self.pool_fused and nxt_is_pool and L["relu"] and a.shape[1] % 2 == 0 and a.shape[2] % 2 == 0:
+                    n.conv_fwd_pool(a, s, self.weights[wi], self.s_w[li], y=out, y_pool=self.acts[li + 1],
+                                    s_y=self.s_act[li], b_y=self.b_fwd[li], pad=1, relu=True,
+                                    round_mode=self.round_mode)
+                    pooled_by_conv = li + 1
+                else:
+                    n.conv_fwd(a, s, self.weights[wi], self.s_w[li], y=out, s_y=self.s_act[li],
+                               b_y=self.b_fwd[li], pad=1, relu=L["relu"], round_mode=self.round_mode)
                 s = self.s_act[li]
                 wi += 1
             elif L["op"] == "fc":
@@ -167,6 +178,8 @@ class NitiTrainer:
                              round_mode=self.round_mode)
                 s = self.s_act[li]
                 wi += 1
+            elif pooled_by_conv == li:
+                pass                                  # written by the convolution before it
             else:
                 if self.pool_idx[li] is not None:
                     n.maxpool2_fwd_idx(a, y=out, idx=self.pool_idx[li])

@@ -495,6 +495,51 @@ def test_strided_and_unpadded_convolutions(niti, oref, B, H, W, Ci, Co, R, pad, 
     niti.check()
 
 
+POOL_SHAPES = [(2, 32, 32, 64, 64), (3, 28, 36, 64, 128), (2, 16, 16, 256, 256), (8, 8, 8, 128, 512),
+               (16, 4, 4, 512, 512), (32, 2, 2, 512, 512), (1, 64, 64, 256, 64), (2, 12, 20, 96, 160),
+               (2, 6, 10, 32, 48), (3, 20, 36, 3, 32), (2, 16, 64, 128, 128), (1, 18, 26, 64, 64),
+               (2, 34, 22, 128, 128)]
+
+
+@pytest.mark.parametrize("engine", [0, 1, 2, 3, 4, 5])
+@pytest.mark.parametrize("B,H,W,Ci,Co", POOL_SHAPES)
+def test_conv_fwd_pool(niti, oref, B, H, W, Ci, Co, engine):
+    """Convolution + ReLU + 2 x 2 max-pool in one call: both outputs equal the oracle's convolution
+    followed by its pooling, whether the tensor-core epilogue pools (windows inside a warp: 8 x 16 pixel
+    tiles, narrow pixel boxes, ragged tiles) or the pooling kernel runs afterwards (wide pixel boxes, 48
+    output channels, the gathered RGB layer, the other engines)."""
+    rng = np.random.default_rng(B + H * 3 + W * 5 + Ci * 7 + Co * 11)
+    x, w = _i8(rng, (B, H, W, Ci)), _i8(rng, (Co, 3, 3, Ci))
+    wy, s, b = oref.conv_fwd(x, -7, w, -9, 1, True)
+    wp = oref.maxpool2_fwd(wy)
+    niti.set_engine(engine)
+    try:
+        y, yp, s_y, b_y = niti.conv_fwd_pool(_T(niti, x), niti.scalar(-7), _T(niti, w), niti.scalar(-9))
+        _eq(y, wy)
+        _eq(yp, wp)
+        assert (int(s_y), int(b_y)) == (s, b)
+    finally:
+        niti.set_engine(0)
+    niti.check()
+
+
+def test_conv_fwd_pool_after_a_wrong_speculative_shift(niti, oref):
+    """The pooled tensor is rewritten with the full-resolution one when the first pass rounded with too
+    small a shift (only the end of the tensor is large)."""
+    rng = np.random.default_rng(79)
+    B, H, W, C = 40, 32, 32, 64
+    x = rng.integers(-3, 4, size=(B, H, W, C), dtype=np.int8)
+    x[-1, -4:, -8:] = rng.integers(100, 128, size=(4, 8, C), dtype=np.int8)
+    w = rng.integers(64, 128, size=(C, 3, 3, C), dtype=np.int8)
+    wy, s, b = oref.conv_fwd(x, -7, w, -9, 1, True)
+    redo0 = niti.redo_count()
+    y, yp, s_y, b_y = niti.conv_fwd_pool(_T(niti, x), niti.scalar(-7), _T(niti, w), niti.scalar(-9))
+    _eq(y, wy)
+    _eq(yp, oref.maxpool2_fwd(wy))
+    assert (int(s_y), int(b_y)) == (s, b) and niti.redo_count() > redo0
+    niti.check()
+
+
 def test_saturation_and_zero_tensor(niti, oref):
     # all-zero accumulators: b = 0, output zero, exponent = s_a + s_w
     a = np.zeros((32, 64), np.int8)

@@ -18,12 +18,12 @@ def niti():
     n.close()
 
 
-def _run_both(niti, net, steps, fused_update=False, pool_codes=False):
+def _run_both(niti, net, steps, fused_update=False, pool_codes=False, pool_fused=True):
     from oracle import OracleNetState, oracle_train_step
     from paper_2009_13108_b200 import NitiTrainer
     x, labels, weights = make_net_inputs(net)
     st = OracleNetState([w.copy() for w in weights])
-    tr = NitiTrainer(niti, net, weights, fused_update=fused_update, pool_codes=pool_codes)
+    tr = NitiTrainer(niti, net, weights, fused_update=fused_update, pool_codes=pool_codes, pool_fused=pool_fused)
     tr.load_batch(x, labels)
     for step in range(steps):
         rec = oracle_train_step(net, x, labels, st)
@@ -165,3 +165,10 @@ def test_config1_sweep_full_size_sampled(niti, oref, M, N, K):
         acc = oref.fc_fwd_acc(a, w[c:c + 1])[:, 0]
         want = np.array([oref.psr(int(v), bp, 7) for v in acc], dtype=np.int8)
         assert np.array_equal(got[:, c], want)
+
+
+def test_steps_with_separate_pooling_passes(niti):
+    """The default forward step pools in the convolution's epilogue; the separate pooling pass gives the
+    same steps."""
+    _run_both(niti, config_net(3, batch=8), steps=2, pool_fused=False)
+    _run_both(niti, config_net(2, batch=16), steps=2, pool_fused=False)
