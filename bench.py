@@ -253,6 +253,46 @@ def run_paper_table(args):
     niti.check()
 
 
+def run_conv_shape(args):
+    """One 3x3 / pad 1 convolution layer at BxHxWxCinxCout: forward (with ReLU), error (with the ReLU gate)
+    and weight gradient, each timed with CUDA events; a small case for profiler captures."""
+    import numpy as np
+    import torch
+    from paper_2009_13108_b200 import Niti
+    niti = Niti(0)
+    dev = niti.device
+    B, H, W, Ci, Co = (int(v) for v in args.conv_shape.lower().split("x"))
+    rng = np.random.Generator(np.random.PCG64(12))
+    x = torch.from_numpy(np.maximum(rng.integers(-127, 128, size=(B, H, W, Ci), dtype=np.int8), 0)).to(dev)
+    w = torch.from_numpy(rng.integers(-127, 128, size=(Co, 3, 3, Ci), dtype=np.int8)).to(dev)
+    e = torch.from_numpy(rng.integers(-127, 128, size=(B, H, W, Co), dtype=np.int8)).to(dev)
+    y, ep, g = torch.empty_like(e), torch.empty_like(x), torch.empty_like(w)
+    sx, sw, sy = niti.scalar(-7), niti.scalar(-10), niti.scalar()
+    b_y, b_e, b_g = niti.scalar(), niti.scalar(), niti.scalar()
+    ops = 2.0 * B * H * W * Ci * Co * 9
+    row = {"conv": [B, H, W, Ci, Co], "int8_ops": ops}
+    for name, fn, nbytes in (
+            ("fwd", lambda: niti.conv_fwd(x, sx, w, sw, y=y, s_y=sy, b_y=b_y, relu=True), x.numel() + w.numel() + y.numel()),
+            ("dgrad", lambda: niti.conv_dgrad(e, w, (H, W), e_prev=ep, relu_mask_src=x, b_e=b_e),
+             e.numel() + w.numel() + 2 * x.numel()),
+            ("wgrad", lambda: niti.conv_wgrad(x, e, g=g, b_g=b_g), x.numel() + e.numel() + w.numel())):
+        if args.only and name != args.only:
+            continue
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(True), torch.cuda.Event(True)
+        e0.record()
+        for _ in range(args.iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.iters
+        row[name] = {"ms": ms, "tops": ops / ms / 1e9, "algorithmic_bytes": nbytes}
+    print(json.dumps(row), flush=True)
+    niti.check()
+
+
 def run_elementwise(args):
     """HBM-bound kernels at sizes well beyond the 126 MB L2: achieved GB/s = algorithmic bytes / time."""
     import numpy as np
@@ -678,6 +718,9 @@ def main():
                     help="weight gradient and weight update in one library call (default: two calls)")
     ap.add_argument("--gemm-shape", default=None,
                     help="MxNxK: time only the fused GEMM at this shape (for profiling a small case)")
+    ap.add_argument("--conv-shape", default=None,
+                    help="BxHxWxCinxCout: time one 3x3 convolution layer (forward, error, weight gradient)")
+    ap.add_argument("--only", default=None, choices=["fwd", "dgrad", "wgrad"], help="with --conv-shape: one of the three")
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--sweep", action="store_true", help="run the fused-GEMM sweep (config 1), one JSON line per point")
     ap.add_argument("--paper-table", action="store_true",
@@ -706,6 +749,9 @@ def main():
         return
     if args.per_launch:
         run_per_launch(args)
+        return
+    if args.conv_shape:
+        run_conv_shape(args)
         return
     if args.gemm_shape:
         from paper_2009_13108_b200 import Niti

@@ -126,8 +126,8 @@ uint64_t niti_tc_pair_launch_count(niti_ctx *ctx);
  * tile of every CTA and recomputes the multiply when the whole tensor turns out to need a larger
  * shift (results are exact either way).  A call that passes a bit-width scalar (b_out / b_e / b_g)
  * is recognised by that scalar's address when it comes again (the same layer in the next training
- * step): the estimate is then corrected by what it missed last time, which removes the recomputations
- * of tensors whose extremes the sample systematically misses.  Returns how many recomputations this
+ * step): an estimate that missed by the same amount twice in a row is corrected by that amount, which
+ * removes the recomputations of tensors whose extremes the sample systematically misses.  Returns how many recomputations this
  * context has run so far (synchronises `stream`; -1 on error). */
 int64_t niti_redo_count(niti_ctx *ctx, void *stream);
 
@@ -274,8 +274,23 @@ int niti_linear_bwd_update(niti_ctx *ctx, void *stream, const int8_t *a, const i
 #define NITI_REDUCE_MAX_U32 0
 #define NITI_REDUCE_MAX_U64 1
 #define NITI_REDUCE_SUM_I32 2
+/* Only after niti_set_dp_shard(ctx, rank, world) with world > 1 (count is a multiple of world):
+ *   NITI_REDUCE_SCATTER_SUM_I32: dev_ptr -> count int32; on return the rank's own slice
+ *     [rank * count / world, (rank + 1) * count / world) holds the sums over the ranks of that slice
+ *     (the other slices are unspecified): a reduce-scatter in place;
+ *   NITI_ALLGATHER_I8: dev_ptr -> count bytes; every rank's own slice (same split) is distributed to all
+ *     ranks: an all-gather in place. */
+#define NITI_REDUCE_SCATTER_SUM_I32 3
+#define NITI_ALLGATHER_I8 4
 typedef int (*niti_reduce_fn)(void *user, void *stream, void *dev_ptr, int64_t count, int kind);
 int niti_set_reduce_hook(niti_ctx *ctx, niti_reduce_fn fn, void *user);
+/* Tells the library this process' place among the data-parallel ranks.  With world > 1 a weight
+ * gradient is no longer all-reduced as a whole int32 tensor (8 bytes per weight on the wire): its
+ * sums are reduce-scattered (4 bytes per weight), every rank takes the max over its shard and the
+ * maxima are combined, every rank rounds its shard (or updates its shard of the weights, in the
+ * fused-update calls) and the int8 result is all-gathered (1 byte per weight).  Results are the same
+ * bit for bit.  world = 1 (the default) keeps the all-reduce. */
+int niti_set_dp_shard(niti_ctx *ctx, int rank, int world);
 
 /* Integer cross-entropy gradient (Section 3.5, Eq. 1-4).  Per sample r:
  *   e32[r][i] = T_i - [i == labels[r]] * sum_j T_j

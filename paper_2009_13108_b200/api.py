@@ -17,12 +17,12 @@ OK, ERR_ARG, ERR_SHAPE, ERR_WORKSPACE, ERR_RANGE, ERR_CUDA, ERR_DEVICE = range(7
 ROUND_PSR, ROUND_NEAREST = 0, 1
 OP_LINEAR_FWD, OP_LINEAR_BWD, OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_INT_XENT = range(6)
 OP_LINEAR_BWD_UPDATE, OP_CONV_WGRAD_UPDATE = 6, 7
-REDUCE_MAX_U32, REDUCE_MAX_U64, REDUCE_SUM_I32 = 0, 1, 2
+REDUCE_MAX_U32, REDUCE_MAX_U64, REDUCE_SUM_I32, REDUCE_SCATTER_SUM_I32, ALLGATHER_I8 = 0, 1, 2, 3, 4
 _REDUCE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int)
 
 EXPORTS = [
     "niti_create", "niti_destroy", "niti_last_error", "niti_check", "niti_workspace_bytes",
-    "niti_set_engine", "niti_set_reduce_hook", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
+    "niti_set_engine", "niti_set_reduce_hook", "niti_set_dp_shard", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
     "niti_redo_count", "niti_selftest_timeout", "niti_profile_enable", "niti_profile_read_launches",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
     "niti_conv_dgrad", "niti_conv_wgrad", "niti_conv_fwd_pool", "niti_conv_fwd_strided", "niti_conv_dgrad_strided", "niti_conv_wgrad_strided",
@@ -57,6 +57,7 @@ def load_library():
     lib.niti_workspace_bytes.restype = sz
     lib.niti_set_engine.argtypes = [vp, i32]
     lib.niti_set_reduce_hook.argtypes = [vp, _REDUCE_FN, vp]
+    lib.niti_set_dp_shard.argtypes = [vp, i32, i32]
     lib.niti_launch_count.argtypes = [vp]
     lib.niti_launch_count.restype = C.c_uint64
     lib.niti_tc_launch_count.argtypes = [vp]
@@ -149,7 +150,12 @@ class Niti:
         def cb(user, stream, ptr, count, kind):
             try:
                 dtype, size = {REDUCE_MAX_U32: (torch.int32, 4), REDUCE_MAX_U64: (torch.int64, 8),
-                               REDUCE_SUM_I32: (torch.int32, 4)}[kind]
+                               REDUCE_SUM_I32: (torch.int32, 4), REDUCE_SCATTER_SUM_I32: (torch.int32, 4),
+                               ALLGATHER_I8: (torch.int8, 1)}[kind]
+                if kind == ALLGATHER_I8 and not (0 <= ptr - self._ws.data_ptr() < self._ws.numel()):
+                    # the gathered tensor is the caller's gradient or weight tensor, not the workspace
+                    fn(_device_view(ptr, count, self.device), kind)
+                    return 0
                 off = ptr - self._ws.data_ptr()
                 if off < 0 or off + count * size > self._ws.numel():
                     return 2
@@ -161,6 +167,11 @@ class Niti:
 
         self._reduce_cb = _REDUCE_FN(cb)      # keep the callback object alive
         self._ck(self.lib.niti_set_reduce_hook(self.h, self._reduce_cb, None))
+
+    def set_dp_shard(self, rank: int, world: int):
+        """niti_set_dp_shard: with world > 1 weight gradients are reduce-scattered, rounded per shard and
+        all-gathered as int8; the reduction hook must handle REDUCE_SCATTER_SUM_I32 and ALLGATHER_I8."""
+        self._ck(self.lib.niti_set_dp_shard(self.h, rank, world))
 
     def reserve_workspace(self, nbytes: int):
         if self._ws.numel() < nbytes:
@@ -417,13 +428,40 @@ class Niti:
         return e_in
 
 
+def _device_view(ptr: int, nbytes: int, device):
+    """An int8 tensor over ``nbytes`` of device memory at ``ptr`` (memory owned by someone else)."""
+    class _Mem:
+        __cuda_array_interface__ = {"shape": (nbytes,), "typestr": "|i1", "data": (ptr, False), "version": 3}
+    return torch.as_tensor(_Mem(), device=device)
+
+
 def dist_reducer(group=None):
     """A reduction hook for ``Niti.set_reduce_hook`` over a torch.distributed process group (NCCL: the
-    all-reduce is ordered on the current stream; gloo: through the host)."""
+    collectives are ordered on the current stream; gloo: through the host).  Reduce-scatter and
+    all-gather run in place on the tensor the library hands over; backends without a reduce-scatter
+    (gloo) all-reduce instead, which leaves the same sums in the rank's slice."""
     import torch.distributed as dist
 
     def reduce(view, kind):
-        op = dist.ReduceOp.SUM if kind == REDUCE_SUM_I32 else dist.ReduceOp.MAX
-        dist.all_reduce(view, op=op, group=group)
+        if kind == REDUCE_SCATTER_SUM_I32:
+            world, rank = dist.get_world_size(group), dist.get_rank(group)
+            n = view.numel() // world
+            if dist.get_backend(group) == "nccl":
+                dist.reduce_scatter_tensor(view[rank * n:(rank + 1) * n], view, op=dist.ReduceOp.SUM, group=group)
+            else:
+                dist.all_reduce(view, op=dist.ReduceOp.SUM, group=group)
+        elif kind == ALLGATHER_I8:
+            world, rank = dist.get_world_size(group), dist.get_rank(group)
+            n = view.numel() // world
+            if dist.get_backend(group) == "nccl":
+                dist.all_gather_into_tensor(view, view[rank * n:(rank + 1) * n], group=group)
+            else:
+                parts = [torch.empty(n, dtype=view.dtype, device=view.device) for _ in range(world)]
+                dist.all_gather(parts, view[rank * n:(rank + 1) * n].clone(), group=group)
+                for r, part in enumerate(parts):
+                    view[r * n:(r + 1) * n].copy_(part)
+        else:
+            op = dist.ReduceOp.SUM if kind == REDUCE_SUM_I32 else dist.ReduceOp.MAX
+            dist.all_reduce(view, op=op, group=group)
 
     return reduce

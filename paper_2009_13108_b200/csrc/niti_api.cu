@@ -78,6 +78,13 @@ extern "C" int niti_set_reduce_hook(niti_ctx *ctx, niti_reduce_fn fn, void *user
   return NITI_OK;
 }
 
+extern "C" int niti_set_dp_shard(niti_ctx *ctx, int rank, int world) {
+  if (!ctx || world < 1 || rank < 0 || rank >= world) return NITI_ERR_ARG;
+  ctx->dp_rank = rank;
+  ctx->dp_world = world;
+  return NITI_OK;
+}
+
 extern "C" uint64_t niti_launch_count(niti_ctx *ctx) { return ctx ? ctx->launches : 0; }
 extern "C" uint64_t niti_tc_launch_count(niti_ctx *ctx) { return ctx ? ctx->tc_launches : 0; }
 extern "C" uint64_t niti_tc_pair_launch_count(niti_ctx *ctx) { return ctx ? ctx->tc2_launches : 0; }
@@ -251,9 +258,27 @@ int niti_launch_sgd_update(niti_ctx *ctx, cudaStream_t st, int8_t *w, const int8
 // Data parallelism (niti_set_reduce_hook), after a multiply has left its int32 accumulators in acc and
 // their max magnitude in the header: a weight gradient is summed over the ranks and its max taken
 // again from the sums; any other tensor only shares the max.
-int niti_reduce_after_gemm(niti_ctx *ctx, cudaStream_t st, int kind, int32_t *acc, long long n, WsHeader *hdr) {
+int niti_reduce_after_gemm(niti_ctx *ctx, cudaStream_t st, int kind, int32_t *acc, long long n, WsHeader *hdr,
+                           bool shard_ok) {
   if (!ctx->reduce_fn) return NITI_OK;
   if (!niti_is_wgrad(kind)) return niti_reduce(ctx, st, &hdr->maxabs32, 1, NITI_REDUCE_MAX_U32);
+  if (shard_ok && niti_dp_sharded(ctx, kind)) {
+    // Sharded (Section 3.3's update distributed over the ranks): every rank receives the sums of its own
+    // shard only (reduce-scatter, 4 bytes per weight on the wire), the few elements that do not divide
+    // evenly are all-reduced, each rank takes the max over what it holds and the maxima are combined.
+    // The caller then rounds its shard and all-gathers the int8 result (1 byte per weight).
+    const NitiDpShard sh = niti_dp_shard(ctx, n);
+    int rc = NITI_OK;
+    if (sh.main > 0) rc = niti_reduce(ctx, st, acc, sh.main, NITI_REDUCE_SCATTER_SUM_I32);
+    if (rc == NITI_OK && n > sh.main) rc = niti_reduce(ctx, st, acc + sh.main, n - sh.main, NITI_REDUCE_SUM_I32);
+    if (rc != NITI_OK) return rc;
+    NITI_CUDA_TRY(ctx, cudaMemsetAsync(&hdr->maxabs32, 0, sizeof(unsigned int), st));
+    ctx->launches++;
+    if (sh.shard > 0) rc = niti_launch_maxabs(ctx, st, acc + sh.off, sh.shard, hdr);
+    if (rc == NITI_OK && n > sh.main) rc = niti_launch_maxabs(ctx, st, acc + sh.main, n - sh.main, hdr);
+    if (rc != NITI_OK) return rc;
+    return niti_reduce(ctx, st, &hdr->maxabs32, 1, NITI_REDUCE_MAX_U32);
+  }
   int rc = niti_reduce(ctx, st, acc, n, NITI_REDUCE_SUM_I32);
   if (rc != NITI_OK) return rc;
   NITI_CUDA_TRY(ctx, cudaMemsetAsync(&hdr->maxabs32, 0, sizeof(unsigned int), st));
@@ -282,14 +307,29 @@ static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, 
   bool fused = false;
   bool pooled = false;
   RoundSpec rs = {out, mask, mbits, round_mode, relu, s_a, s_w, s_out, b_out, pool_out};
-  if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, rs, acc, hdr, &fused, &pooled);
+  if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, rs, acc, hdr, &fused, &pooled, true);
   if (rc == NITI_ERR_SHAPE) {
     rc = niti_simt_gemm(ctx, st, p, acc, hdr);
-    if (rc == NITI_OK) rc = niti_reduce_after_gemm(ctx, st, p.kind, acc, p.gm * p.gn, hdr);
+    if (rc == NITI_OK) rc = niti_reduce_after_gemm(ctx, st, p.kind, acc, p.gm * p.gn, hdr, true);
   }
   if (rc != NITI_OK) return rc;
   if (fused) {
     if (update_w) return niti_launch_sgd_update(ctx, st, update_w, out, p.gm * p.gn);
+  } else if (niti_dp_sharded(ctx, p.kind)) {
+    // sharded weight gradient: acc holds the sums over the ranks for this rank's shard (and the
+    // remainder): round those (into the gradient, or straight into the weights), then every rank
+    // collects the other shards' int8 results
+    const long long n = p.gm * p.gn;
+    const NitiDpShard sh = niti_dp_shard(ctx, n);
+    int8_t *dst = update_w ? update_w : out;
+    if (sh.shard > 0)
+      rc = niti_launch_round(ctx, st, acc + sh.off, hdr, out + sh.off, sh.shard, mbits, round_mode, relu, nullptr,
+                             s_a, s_w, s_out, b_out, update_w ? update_w + sh.off : nullptr);
+    if (rc == NITI_OK && n > sh.main)
+      rc = niti_launch_round(ctx, st, acc + sh.main, hdr, out + sh.main, n - sh.main, mbits, round_mode, relu, nullptr,
+                             s_a, s_w, s_out, b_out, update_w ? update_w + sh.main : nullptr);
+    if (rc == NITI_OK && sh.main > 0) rc = niti_reduce(ctx, st, dst, sh.main, NITI_ALLGATHER_I8);
+    if (rc != NITI_OK) return rc;
   } else {
     rc = niti_launch_round(ctx, st, acc, hdr, out, p.gm * p.gn, mbits, round_mode, relu, mask, s_a, s_w,
                            s_out, b_out, update_w);

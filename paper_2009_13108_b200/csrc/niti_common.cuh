@@ -31,6 +31,8 @@ struct niti_ctx {
   // combined over the ranks before the rounding may use it
   niti_reduce_fn reduce_fn;
   void *reduce_user;
+  int dp_rank, dp_world;    // niti_set_dp_shard: > 1 ranks = weight gradients are reduce-scattered, rounded per
+                            // shard and all-gathered as int8 (5 bytes per weight on the wire instead of 8)
   // per-device facts of the tensor-core kernel, indexed by CTAs per tile (1 or 2): co-resident CTAs /
   // CTA pairs (0 = not asked yet) and the dynamic shared-memory limit already set on the kernel
   int tc_units[3];
@@ -154,7 +156,24 @@ static inline int niti_partial_slices(int kind, long long gm) {
 // acc holds `splits` partial tensors of n int32 each: adds them into the first, takes max |sum| into
 // hdr->maxabs32 and raises NITI_DEV_ACC_RANGE when the magnitudes of an element's partial sums add up to 2^31
 int niti_launch_sum_partials(niti_ctx *ctx, cudaStream_t st, int32_t *acc, int splits, long long n, WsHeader *hdr);
-int niti_reduce_after_gemm(niti_ctx *ctx, cudaStream_t st, int kind, int32_t *acc, long long n, WsHeader *hdr);
+// shard_ok: the caller rounds only this rank's shard afterwards (niti_dp_shard) and all-gathers the result
+int niti_reduce_after_gemm(niti_ctx *ctx, cudaStream_t st, int kind, int32_t *acc, long long n, WsHeader *hdr,
+                           bool shard_ok = false);
+// Sharding of a weight-gradient tensor of n elements over the data-parallel ranks: `main` elements are
+// split evenly (every shard a multiple of 16 elements, so that vector accesses stay aligned), the
+// remaining `n - main` are combined with an all-reduce and handled by every rank.
+struct NitiDpShard { long long main, shard, off; };
+static inline NitiDpShard niti_dp_shard(const niti_ctx *ctx, long long n) {
+  NitiDpShard s;
+  const long long unit = 16LL * ctx->dp_world;
+  s.main = n / unit * unit;
+  s.shard = s.main / ctx->dp_world;
+  s.off = s.shard * ctx->dp_rank;
+  return s;
+}
+static inline bool niti_dp_sharded(const niti_ctx *ctx, int kind) {
+  return ctx->reduce_fn && ctx->dp_world > 1 && (kind == 2 || kind == 5);   // weight gradients only
+}
 // max |acc| into hdr->maxabs32; splits > 1: also adds up the split maxima of the header and raises
 // NITI_DEV_ACC_RANGE when an accumulator may have left the int32 range
 int niti_launch_maxabs(niti_ctx *ctx, cudaStream_t st, const int32_t *acc, long long n, WsHeader *hdr, int splits = 0);
@@ -174,7 +193,7 @@ struct RoundSpec {
 // acc holds the int32 accumulators and hdr->maxabs32 their max magnitude.
 // *pooled (may be null) is set when the kernel's epilogue also wrote r.pool_out.
 int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, const RoundSpec &r, int32_t *acc,
-                 WsHeader *hdr, bool *fused, bool *pooled = nullptr);
+                 WsHeader *hdr, bool *fused, bool *pooled = nullptr, bool shard_ok = false);
 size_t niti_tc_scratch_bytes(const GemmProblem &p);
 
 // Epilogue pass: b from hdr->maxabs32, bp = max(0, b - mbits), out = Round(acc) with optional ReLU

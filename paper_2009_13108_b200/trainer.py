@@ -37,8 +37,11 @@ class NitiTrainer:
         # so every rank holds the weights one process with the whole batch would have
         self.data_parallel = data_parallel
         if data_parallel:
+            import torch.distributed as dist
             from .api import dist_reducer
             niti.set_reduce_hook(dist_reducer(dist_group))
+            # weight gradients: reduce-scatter of the int32 sums, per-shard rounding, all-gather of int8
+            niti.set_dp_shard(dist.get_rank(dist_group), dist.get_world_size(dist_group))
             self._dist_group = dist_group
         dev = niti.device
         i8 = dict(dtype=torch.int8, device=dev)

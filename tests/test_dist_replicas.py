@@ -72,7 +72,16 @@ def _reducer_worker(rank, world, port, q):
     reduce(m32, REDUCE_MAX_U32)
     reduce(m64, REDUCE_MAX_U64)
     reduce(acc, REDUCE_SUM_I32)
-    q.put((rank, int(m32[0]), int(m64[0]), acc.tolist()))
+    # the sharded weight-gradient path: reduce-scatter of int32 sums (each rank only needs its own
+    # slice afterwards), then all-gather of the int8 slices every rank produced from them
+    from paper_2009_13108_b200.api import ALLGATHER_I8, REDUCE_SCATTER_SUM_I32
+    g32 = torch.arange(8, dtype=torch.int32) * (rank + 1)
+    reduce(g32, REDUCE_SCATTER_SUM_I32)
+    mine = g32[rank * 4:(rank + 1) * 4].tolist()
+    g8 = torch.full((8,), -1, dtype=torch.int8)
+    g8[rank * 4:(rank + 1) * 4] = torch.tensor([10 * rank + i for i in range(4)], dtype=torch.int8)
+    reduce(g8, ALLGATHER_I8)
+    q.put((rank, int(m32[0]), int(m64[0]), acc.tolist(), mine, g8.tolist()))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -88,10 +97,12 @@ def test_the_data_parallel_reducer_combines_max_and_sum_over_two_gloo_ranks():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    for rank, m32, m64, acc in res:                       # the same on every rank
+    for rank, m32, m64, acc, mine, g8 in res:             # the same on every rank
         assert m32 == 1007
         assert m64 == (1 << 40) + 3
         assert acc == [10, -12, 21, -2147483000]
+        assert mine == [3 * i for i in range(rank * 4, rank * 4 + 4)]      # sums over ranks 1x + 2x
+        assert g8 == [0, 1, 2, 3, 10, 11, 12, 13]
 
 
 def test_launch_ranks_starts_one_process_per_rank_on_localhost(tmp_path):
