@@ -22,7 +22,7 @@ _REDUCE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
 
 EXPORTS = [
     "niti_create", "niti_destroy", "niti_last_error", "niti_check", "niti_workspace_bytes",
-    "niti_set_engine", "niti_set_reduce_hook", "niti_set_dp_shard", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
+    "niti_set_engine", "niti_set_reduce_hook", "niti_set_dp_shard", "niti_set_tap_cache", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
     "niti_redo_count", "niti_selftest_timeout", "niti_profile_enable", "niti_profile_read_launches",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
     "niti_conv_dgrad", "niti_conv_wgrad", "niti_conv_fwd_pool", "niti_conv_fwd_strided", "niti_conv_dgrad_strided", "niti_conv_wgrad_strided",
@@ -58,6 +58,7 @@ def load_library():
     lib.niti_set_engine.argtypes = [vp, i32]
     lib.niti_set_reduce_hook.argtypes = [vp, _REDUCE_FN, vp]
     lib.niti_set_dp_shard.argtypes = [vp, i32, i32]
+    lib.niti_set_tap_cache.argtypes = [vp, vp, sz]
     lib.niti_launch_count.argtypes = [vp]
     lib.niti_launch_count.restype = C.c_uint64
     lib.niti_tc_launch_count.argtypes = [vp]
@@ -172,6 +173,12 @@ class Niti:
         """niti_set_dp_shard: with world > 1 weight gradients are reduce-scattered, rounded per shard and
         all-gathered as int8; the reduction hook must handle REDUCE_SCATTER_SUM_I32 and ALLGATHER_I8."""
         self._ck(self.lib.niti_set_dp_shard(self.h, rank, world))
+
+    def set_tap_cache(self, nbytes: int):
+        """niti_set_tap_cache with a buffer of ``nbytes`` owned by this object (0 removes it): the gathered
+        taps of a few-channel first layer are kept between its forward and its weight-gradient call."""
+        self._tap = torch.empty(nbytes, dtype=torch.uint8, device=self.device) if nbytes else None
+        self._ck(self.lib.niti_set_tap_cache(self.h, _ptr(self._tap), nbytes))
 
     def reserve_workspace(self, nbytes: int):
         if self._ws.numel() < nbytes:

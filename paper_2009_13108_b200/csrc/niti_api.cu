@@ -78,6 +78,25 @@ extern "C" int niti_set_reduce_hook(niti_ctx *ctx, niti_reduce_fn fn, void *user
   return NITI_OK;
 }
 
+extern "C" int niti_set_tap_cache(niti_ctx *ctx, void *buf, size_t bytes) {
+  if (!ctx || (buf && (((uintptr_t)buf & 255) || bytes == 0))) return NITI_ERR_ARG;
+  ctx->tap_buf = (int8_t *)buf;
+  ctx->tap_bytes = buf ? bytes : 0;
+  ctx->tap_x = nullptr;
+  ctx->tap_dims[8] = 0;
+  return NITI_OK;
+}
+
+// Does the tap cache hold the gathered rows of exactly this input tensor and geometry?
+static bool tap_cache_hit(const niti_ctx *ctx, const void *x, int B, int H, int W, int Ci, int R, int S, int pad,
+                          int stride) {
+  const int want[8] = {B, H, W, Ci, R, S, pad, stride};
+  if (!ctx->tap_buf || !ctx->tap_dims[8] || ctx->tap_x != x) return false;
+  for (int i = 0; i < 8; ++i)
+    if (ctx->tap_dims[i] != want[i]) return false;
+  return true;
+}
+
 extern "C" int niti_set_dp_shard(niti_ctx *ctx, int rank, int world) {
   if (!ctx || world < 1 || rank < 0 || rank >= world) return NITI_ERR_ARG;
   ctx->dp_rank = rank;
@@ -453,6 +472,13 @@ static int conv_fwd_impl(niti_ctx *ctx, void *stream, const int8_t *x, const int
     char *base = (char *)ws + NITI_WS_HEADER + round_up(M * (size_t)Cout * 4, 256);
     int8_t *xcol = (int8_t *)base;
     int8_t *wcol = (int8_t *)(base + round_up(M * 32, 256));
+    if (ctx->tap_buf && M * 32 <= ctx->tap_bytes) {
+      // gathered into the caller's tap cache: the weight-gradient call of this layer finds the rows there
+      xcol = ctx->tap_buf;
+      ctx->tap_x = x;
+      const int dims[9] = {B, H, W, Cin, R, S, pad, stride, 1};
+      memcpy(ctx->tap_dims, dims, sizeof(dims));
+    }
     int rc = niti_launch_im2col32(ctx, st, x, xcol, B, H, W, Cin, R, S, pad, stride, p.Ho, p.Wo);
     if (rc == NITI_OK) rc = niti_launch_pad_rows32(ctx, st, w, wcol, Cout, R * S * Cin);
     if (rc != NITI_OK) return rc;
@@ -553,7 +579,11 @@ static int conv_wgrad_impl(niti_ctx *ctx, void *stream, const int8_t *x, const i
     int32_t *acc32 = (int32_t *)(base + round_up(M * 32, 256) + round_up((size_t)Cout * 32, 256));
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, NITI_WS_HEADER, st));
     ctx->launches++;
-    int rc = niti_launch_im2col32(ctx, st, x, xcol, B, H, W, Cin, R, S, pad, stride, p.Ho, p.Wo);
+    int rc = NITI_OK;
+    if (tap_cache_hit(ctx, x, B, H, W, Cin, R, S, pad, stride)) {
+      xcol = ctx->tap_buf;                 // gathered by the forward call
+      ctx->tap_dims[8] = 0;                // (used once: the next forward call fills the cache again)
+    } else rc = niti_launch_im2col32(ctx, st, x, xcol, B, H, W, Cin, R, S, pad, stride, p.Ho, p.Wo);
     if (rc != NITI_OK) return rc;
     GemmProblem q;
     fill_fc(q, GK_FC_WGRAD, (int)M, Cout, 32);     // rows M are the contraction

@@ -31,6 +31,12 @@ struct niti_ctx {
   // combined over the ranks before the rounding may use it
   niti_reduce_fn reduce_fn;
   void *reduce_user;
+  // niti_set_tap_cache: caller-owned buffer that keeps the gathered taps of a few-channel convolution
+  // between its forward call and its weight-gradient call, and what it currently holds
+  int8_t *tap_buf;
+  size_t tap_bytes;
+  const void *tap_x;
+  int tap_dims[9];          // B, H, W, Cin, R, S, pad, stride, valid
   int dp_rank, dp_world;    // niti_set_dp_shard: > 1 ranks = weight gradients are reduce-scattered, rounded per
                             // shard and all-gathered as int8 (5 bytes per weight on the wire instead of 8)
   // per-device facts of the tensor-core kernel, indexed by CTAs per tile (1 or 2): co-resident CTAs /

@@ -85,6 +85,11 @@ class NitiTrainer:
         self.b_loss = niti.scalar()
         self.n_correct = niti.scalar()
         self.first_weight_layer = next(i for i, L in enumerate(net.layers) if L["op"] != "pool")
+        # an image network's first convolution (1 or 3 input channels) gathers its taps once per step: the
+        # weight gradient at the end of the step reads the rows the forward pass gathered
+        L0 = net.layers[self.first_weight_layer]
+        if L0["op"] == "conv" and 9 * L0["cin"] <= 32 and L0["cin"] % 16 != 0:
+            niti.set_tap_cache(32 * self.acts[self.first_weight_layer].numel() // L0["cout"])
 
     def global_hits(self):
         """Hit count of the last step over all ranks (data parallel), as a device tensor."""
