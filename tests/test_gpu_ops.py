@@ -109,7 +109,9 @@ CONV_SHAPES = [(2, 8, 8, 3, 16), (2, 16, 16, 64, 64), (4, 8, 8, 128, 256), (8, 4
                (4, 8, 8, 64, 320),
                # RGB first layers: staged gather (W % 4 == 0; one with more pixel groups than threads)
                # and the generic gather (W % 4 != 0)
-               (3, 20, 36, 3, 32), (1, 6, 520, 3, 16), (2, 9, 10, 3, 16)]
+               (3, 20, 36, 3, 32), (1, 6, 520, 3, 16), (2, 9, 10, 3, 16),
+               # more few-channel first layers (gathered taps): RGB and single-channel, several widths
+               (2, 32, 32, 3, 64), (4, 32, 16, 1, 32), (8, 64, 48, 3, 16), (3, 16, 48, 3, 32), (2, 32, 16, 1, 32)]
 
 
 @pytest.mark.parametrize("engine", [0, 1, 2, 3, 4, 5])
@@ -498,7 +500,7 @@ def test_strided_and_unpadded_convolutions(niti, oref, B, H, W, Ci, Co, R, pad, 
 POOL_SHAPES = [(2, 32, 32, 64, 64), (3, 28, 36, 64, 128), (2, 16, 16, 256, 256), (8, 8, 8, 128, 512),
                (16, 4, 4, 512, 512), (32, 2, 2, 512, 512), (1, 64, 64, 256, 64), (2, 12, 20, 96, 160),
                (2, 6, 10, 32, 48), (3, 20, 36, 3, 32), (2, 16, 64, 128, 128), (1, 18, 26, 64, 64),
-               (2, 34, 22, 128, 128)]
+               (2, 34, 22, 128, 128), (2, 32, 32, 3, 64), (4, 32, 16, 1, 32)]
 
 
 @pytest.mark.parametrize("engine", [0, 1, 2, 3, 4, 5])
