@@ -6,7 +6,8 @@
  * Every tensor pointer below is a DEVICE pointer owned by the caller unless a
  * function says otherwise.  The library allocates no device memory after
  * niti_create(); scratch comes from the caller's workspace `ws` (size from
- * niti_workspace_bytes(), 256-byte aligned).  All work is enqueued on the
+ * niti_workspace_bytes(), 256-byte aligned; its first 256 KB hold 64 small
+ * headers of reduction scalars, see niti_begin_step()).  All work is enqueued on the
  * caller's stream (`stream` is a cudaStream_t passed as void*) and the calls
  * return without synchronising; one workspace must not be used by two calls
  * that can overlap on the GPU.
@@ -284,6 +285,16 @@ int niti_linear_bwd_update(niti_ctx *ctx, void *stream, const int8_t *a, const i
 #define NITI_ALLGATHER_I8 4
 typedef int (*niti_reduce_fn)(void *user, void *stream, void *dev_ptr, int64_t count, int kind);
 int niti_set_reduce_hook(niti_ctx *ctx, niti_reduce_fn fn, void *user);
+/* Optional, once per training step (or per group of at most 64 calls): clears every header of the
+ * workspace `ws` with one memset on `stream`.  The calls that follow on that workspace (in stream
+ * order, from this context) then take one zeroed header each instead of clearing their own, which
+ * removes a memset node from in front of every multiply of the step.  After 64 calls, or for any other
+ * workspace, calls clear their header themselves as they do without this call.  The caller must not
+ * use that workspace from two streams at once (as for any workspace) and must call niti_begin_step
+ * again before the pattern repeats (each training step; a captured CUDA graph holds it as its first
+ * node).  ws = NULL ends the arrangement.  Results do not change. */
+int niti_begin_step(niti_ctx *ctx, void *stream, void *ws, size_t ws_bytes);
+
 /* Convolutions with very few input channels (R * S * Cin <= 32: the first layer of an image network)
  * are run as a matrix multiply over rows of gathered taps, 32 bytes per output pixel.  Forward and
  * weight gradient of such a layer read the same rows.  With a tap cache installed (a caller-owned

@@ -22,7 +22,7 @@ _REDUCE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
 
 EXPORTS = [
     "niti_create", "niti_destroy", "niti_last_error", "niti_check", "niti_workspace_bytes",
-    "niti_set_engine", "niti_set_reduce_hook", "niti_set_dp_shard", "niti_set_tap_cache", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
+    "niti_set_engine", "niti_set_reduce_hook", "niti_set_dp_shard", "niti_set_tap_cache", "niti_begin_step", "niti_launch_count", "niti_tc_launch_count", "niti_tc_pair_launch_count",
     "niti_redo_count", "niti_selftest_timeout", "niti_profile_enable", "niti_profile_read_launches",
     "niti_profile_read", "niti_linear_fwd", "niti_linear_bwd", "niti_conv_fwd",
     "niti_conv_dgrad", "niti_conv_wgrad", "niti_conv_fwd_pool", "niti_conv_fwd_strided", "niti_conv_dgrad_strided", "niti_conv_wgrad_strided",
@@ -59,6 +59,7 @@ def load_library():
     lib.niti_set_reduce_hook.argtypes = [vp, _REDUCE_FN, vp]
     lib.niti_set_dp_shard.argtypes = [vp, i32, i32]
     lib.niti_set_tap_cache.argtypes = [vp, vp, sz]
+    lib.niti_begin_step.argtypes = [vp, vp, vp, sz]
     lib.niti_launch_count.argtypes = [vp]
     lib.niti_launch_count.restype = C.c_uint64
     lib.niti_tc_launch_count.argtypes = [vp]
@@ -182,7 +183,13 @@ class Niti:
 
     def reserve_workspace(self, nbytes: int):
         if self._ws.numel() < nbytes:
+            self._ck(self.lib.niti_begin_step(self.h, None, None, 0))      # the old buffer's headers are gone
             self._ws = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+
+    def begin_step(self):
+        """niti_begin_step on this object's workspace: one memset clears the headers that the next 64
+        calls would otherwise clear one by one."""
+        self._ck(self.lib.niti_begin_step(self.h, self._stream(), self._ws.data_ptr(), self._ws.numel()))
 
     def _ws_for(self, op, dims):
         need = self.workspace_bytes(op, dims)

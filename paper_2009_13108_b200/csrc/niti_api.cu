@@ -78,6 +78,22 @@ extern "C" int niti_set_reduce_hook(niti_ctx *ctx, niti_reduce_fn fn, void *user
   return NITI_OK;
 }
 
+extern "C" int niti_begin_step(niti_ctx *ctx, void *stream, void *ws, size_t ws_bytes) {
+  if (!ctx) return NITI_ERR_ARG;
+  if (!ws) {                                     // forget the prepared workspace: calls clear their header again
+    ctx->step_ws = nullptr;
+    ctx->step_slot = 0;
+    return NITI_OK;
+  }
+  if (((uintptr_t)ws & 255) || ws_bytes < NITI_WS_HEADER)
+    return niti_fail(ctx, NITI_ERR_WORKSPACE, "niti_begin_step: workspace misaligned or too small");
+  NITI_CUDA_TRY(ctx, cudaMemsetAsync(ws, 0, NITI_WS_HEADER, (cudaStream_t)stream));
+  ctx->launches++;
+  ctx->step_ws = ws;
+  ctx->step_slot = 0;
+  return NITI_OK;
+}
+
 extern "C" int niti_set_tap_cache(niti_ctx *ctx, void *buf, size_t bytes) {
   if (!ctx || (buf && (((uintptr_t)buf & 255) || bytes == 0))) return NITI_ERR_ARG;
   ctx->tap_buf = (int8_t *)buf;
@@ -318,11 +334,11 @@ static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, 
                           int32_t *b_out, int8_t *update_w = nullptr, int8_t *pool_out = nullptr) {
   if (!ws || ((uintptr_t)ws & 255) || ws_bytes < need)
     return niti_fail(ctx, NITI_ERR_WORKSPACE, "workspace missing, misaligned or too small");
-  WsHeader *hdr = (WsHeader *)ws;
+  WsHeader *hdr = nullptr;
   int32_t *acc = (int32_t *)((char *)ws + NITI_WS_HEADER);
-  NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, NITI_WS_HEADER, st));        // reduction scalars and split maxima
-  ctx->launches++;
-  int rc = NITI_ERR_SHAPE;
+  int rc = niti_take_header(ctx, st, ws, &hdr);                            // zeroed reduction scalars and split maxima
+  if (rc != NITI_OK) return rc;
+  rc = NITI_ERR_SHAPE;
   bool fused = false;
   bool pooled = false;
   RoundSpec rs = {out, mask, mbits, round_mode, relu, s_a, s_w, s_out, b_out, pool_out};
@@ -573,13 +589,12 @@ static int conv_wgrad_impl(niti_ctx *ctx, void *stream, const int8_t *x, const i
     // R*S*Cin columns are rounded into g
     cudaStream_t st = (cudaStream_t)stream;
     const size_t M = (size_t)B * p.Ho * p.Wo;
-    WsHeader *hdr = (WsHeader *)ws;
+    WsHeader *hdr = nullptr;
     char *base = (char *)ws + NITI_WS_HEADER + round_up((size_t)(p.gm * p.gn) * 4, 256);
     int8_t *xcol = (int8_t *)base;
     int32_t *acc32 = (int32_t *)(base + round_up(M * 32, 256) + round_up((size_t)Cout * 32, 256));
-    NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, NITI_WS_HEADER, st));
-    ctx->launches++;
-    int rc = NITI_OK;
+    int rc = niti_take_header(ctx, st, ws, &hdr);
+    if (rc != NITI_OK) return rc;
     if (tap_cache_hit(ctx, x, B, H, W, Cin, R, S, pad, stride)) {
       xcol = ctx->tap_buf;                 // gathered by the forward call
       ctx->tap_dims[8] = 0;                // (used once: the next forward call fills the cache again)

@@ -37,6 +37,9 @@ struct niti_ctx {
   size_t tap_bytes;
   const void *tap_x;
   int tap_dims[9];          // B, H, W, Cin, R, S, pad, stride, valid
+  // niti_begin_step: workspace whose headers were cleared in one go, and how many of them are used up
+  void *step_ws;
+  int step_slot;
   int dp_rank, dp_world;    // niti_set_dp_shard: > 1 ranks = weight gradients are reduce-scattered, rounded per
                             // shard and all-gathered as int8 (5 bytes per weight on the wire instead of 8)
   // per-device facts of the tensor-core kernel, indexed by CTAs per tile (1 or 2): co-resident CTAs /
@@ -49,7 +52,14 @@ struct niti_ctx {
 
 #define NITI_PROF_MAX 8192
 #define NITI_SPEC_SLOTS 4096
-#define NITI_WS_HEADER 4096 // bytes reserved at the start of every workspace: reduction scalars, then split maxima
+// Every workspace starts with NITI_HDR_SLOTS headers of NITI_HDR_SLOT_BYTES each (reduction scalars, the
+// words of the speculative agreement, split maxima).  A call needs a zeroed header.  Without further
+// notice it clears and uses the first one.  After niti_begin_step() has cleared all of them with one
+// memset, the following calls on that workspace take one header each, in order, without clearing (a
+// cleared-per-call header costs a memset node of about 2 us in front of every multiply of a step).
+#define NITI_HDR_SLOTS 64
+#define NITI_HDR_SLOT_BYTES 4096
+#define NITI_WS_HEADER (NITI_HDR_SLOTS * NITI_HDR_SLOT_BYTES)   // bytes in front of the accumulator scratch
 // A contraction that is split over CTAs adds int32 partial sums; split s records the largest magnitude
 // among its partial sums in split_max[s] (unsigned words from byte NITI_SPLIT_MAX_OFF of the header).
 // The sum of those maxima bounds every accumulator of the tensor: when it reaches 2^31 the int32
@@ -71,7 +81,7 @@ struct WsHeader {
   unsigned int pad1[1];
 };
 static_assert(sizeof(WsHeader) == 32, "workspace header layout");
-static_assert(NITI_SPLIT_MAX_OFF + 4 * NITI_MAX_SPLITS <= NITI_WS_HEADER, "split maxima fit the header");
+static_assert(NITI_SPLIT_MAX_OFF + 4 * NITI_MAX_SPLITS <= NITI_HDR_SLOT_BYTES, "split maxima fit the header");
 __host__ __device__ __forceinline__ unsigned int *niti_split_max(WsHeader *hdr) {
   return reinterpret_cast<unsigned int *>(reinterpret_cast<char *>(hdr) + NITI_SPLIT_MAX_OFF);
 }
@@ -85,6 +95,22 @@ __host__ __device__ __forceinline__ unsigned int *niti_split_max(WsHeader *hdr) 
       return NITI_ERR_CUDA;                                                             \
     }                                                                                   \
   } while (0)
+
+// A zeroed header for the call that is being enqueued: the next unused one of a workspace prepared by
+// niti_begin_step(), else the first one, cleared here.
+static inline int niti_take_header(niti_ctx *ctx, cudaStream_t st, void *ws, WsHeader **hdr) {
+  if (ws == ctx->step_ws && ctx->step_slot < NITI_HDR_SLOTS) {
+    *hdr = reinterpret_cast<WsHeader *>(reinterpret_cast<char *>(ws) + (size_t)NITI_HDR_SLOT_BYTES * ctx->step_slot++);
+    return NITI_OK;
+  }
+  *hdr = reinterpret_cast<WsHeader *>(ws);
+  ctx->launches++;
+  if (cudaMemsetAsync(ws, 0, NITI_HDR_SLOT_BYTES, st) != cudaSuccess) {
+    snprintf(ctx->err, sizeof(ctx->err), "clearing the workspace header failed");
+    return NITI_ERR_CUDA;
+  }
+  return NITI_OK;
+}
 
 static inline int niti_fail(niti_ctx *ctx, int code, const char *msg) {
   if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s", msg);

@@ -701,10 +701,10 @@ extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const
   if (!ws || ((uintptr_t)ws & 255) || ws_bytes < niti_workspace_bytes(NITI_OP_INT_XENT, dims, 2))
     return niti_fail(ctx, NITI_ERR_WORKSPACE, "niti_int_xent: workspace missing, misaligned or too small");
   cudaStream_t st = (cudaStream_t)stream;
-  WsHeader *hdr = (WsHeader *)ws;
+  WsHeader *hdr = nullptr;
   long long *rowinfo = (long long *)((char *)ws + NITI_WS_HEADER);
-  NITI_CUDA_TRY(ctx, cudaMemsetAsync(hdr, 0, sizeof(WsHeader), st));
-  ctx->launches++;
+  const int rch = niti_take_header(ctx, st, ws, &hdr);
+  if (rch != NITI_OK) return rch;
   if (n_correct) {
     NITI_CUDA_TRY(ctx, cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st));
     ctx->launches++;

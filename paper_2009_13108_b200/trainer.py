@@ -199,6 +199,7 @@ class NitiTrainer:
     def step(self):
         """Forward, integer loss gradient, backward with in-place weight update."""
         n, net = self.n, self.net
+        n.begin_step()                     # one memset instead of one per multiply (the workspace is sized by then)
         logits, s_out = self.forward()
         cur = 0
         e = self._view(self.e_buf[cur], logits.shape)
