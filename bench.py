@@ -714,8 +714,9 @@ def main():
                     help="issue every launch from Python instead of replaying a CUDA graph of the step")
     ap.add_argument("--pool-codes", dest="pool_codes", action="store_true",
                     help="max-pool forward records its routing; backward reads the codes instead of the pooled tensor")
-    ap.add_argument("--fused-update", dest="fused_update", action="store_true",
-                    help="weight gradient and weight update in one library call (default: two calls)")
+    ap.add_argument("--separate-update", dest="fused_update", action="store_false",
+                    help="weight gradient and weight update as two library calls (niti_int_sgd_update after "
+                         "niti_conv_wgrad / niti_linear_bwd) instead of the fused *_update calls")
     ap.add_argument("--gemm-shape", default=None,
                     help="MxNxK: time only the fused GEMM at this shape (for profiling a small case)")
     ap.add_argument("--conv-shape", default=None,

@@ -341,15 +341,16 @@ static int run_gemm_round(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, 
   rc = NITI_ERR_SHAPE;
   bool fused = false;
   bool pooled = false;
-  RoundSpec rs = {out, mask, mbits, round_mode, relu, s_a, s_w, s_out, b_out, pool_out};
-  if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, rs, acc, hdr, &fused, &pooled, true);
+  bool updated = false;
+  RoundSpec rs = {out, mask, mbits, round_mode, relu, s_a, s_w, s_out, b_out, pool_out, update_w};
+  if (ctx->engine != 1) rc = niti_tc_gemm(ctx, st, p, rs, acc, hdr, &fused, &pooled, true, &updated);
   if (rc == NITI_ERR_SHAPE) {
     rc = niti_simt_gemm(ctx, st, p, acc, hdr);
     if (rc == NITI_OK) rc = niti_reduce_after_gemm(ctx, st, p.kind, acc, p.gm * p.gn, hdr, true);
   }
   if (rc != NITI_OK) return rc;
   if (fused) {
-    if (update_w) return niti_launch_sgd_update(ctx, st, update_w, out, p.gm * p.gn);
+    if (update_w && !updated) return niti_launch_sgd_update(ctx, st, update_w, out, p.gm * p.gn);
   } else if (niti_dp_sharded(ctx, p.kind)) {
     // sharded weight gradient: acc holds the sums over the ranks for this rank's shard (and the
     // remainder): round those (into the gradient, or straight into the weights), then every rank

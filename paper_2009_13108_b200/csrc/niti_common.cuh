@@ -78,7 +78,7 @@ struct WsHeader {
   unsigned int est_max;             // max |acc| over the first tile of the CTAs that have reported
   unsigned int tile_counter;        // CTAs that have reported
   unsigned int spec_b;              // 0, or 1 + the bit-width the speculative epilogue rounds with
-  unsigned int pad1[1];
+  unsigned int hits;               // integer cross-entropy: rows whose first arg-max is the label
 };
 static_assert(sizeof(WsHeader) == 32, "workspace header layout");
 static_assert(NITI_SPLIT_MAX_OFF + 4 * NITI_MAX_SPLITS <= NITI_HDR_SLOT_BYTES, "split maxima fit the header");
@@ -219,13 +219,16 @@ struct RoundSpec {
   const int32_t *s_a, *s_w;
   int32_t *s_out, *b_out;
   int8_t *pool_out;        // optional (may be null): 2 x 2 max-pool of `out`, forward convolutions with ReLU
+  int8_t *update_w;        // optional (may be null): weight gradients; the caller will subtract `out` from these weights
 };
 // Tensor-core engine (tcgen05); returns NITI_ERR_SHAPE if the shape is not eligible.  *fused is set
 // when the kernel also did the bit-width / shift / round / store (nothing is left to do); otherwise
 // acc holds the int32 accumulators and hdr->maxabs32 their max magnitude.
 // *pooled (may be null) is set when the kernel's epilogue also wrote r.pool_out.
+// *updated (may be null) is set when the epilogue subtracted the rounded gradient from r.update_w itself
+// (`out` is then not written).
 int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &p, const RoundSpec &r, int32_t *acc,
-                 WsHeader *hdr, bool *fused, bool *pooled = nullptr, bool shard_ok = false);
+                 WsHeader *hdr, bool *fused, bool *pooled = nullptr, bool shard_ok = false, bool *updated = nullptr);
 size_t niti_tc_scratch_bytes(const GemmProblem &p);
 
 // Epilogue pass: b from hdr->maxabs32, bp = max(0, b - mbits), out = Round(acc) with optional ReLU

@@ -299,7 +299,7 @@ constexpr int XENT_WARPS = 8;
 __global__ void __launch_bounds__(32 * XENT_WARPS)
 xent_row_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
                 const int32_t *__restrict__ labels, long long *__restrict__ rowinfo, WsHeader *hdr,
-                int32_t *__restrict__ n_correct, int B, int N, uint32_t *__restrict__ status) {
+                int B, int N, uint32_t *__restrict__ status) {
   __shared__ unsigned long long sh_max[XENT_WARPS];
   __shared__ int sh_hit[XENT_WARPS];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -366,7 +366,7 @@ xent_row_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_pt
     int h = 0;
     for (int w = 0; w < XENT_WARPS; ++w) { m = sh_max[w] > m ? sh_max[w] : m; h += sh_hit[w]; }
     if (m > *(volatile unsigned long long *)&hdr->maxabs64) atomicMax(&hdr->maxabs64, m);
-    if (n_correct && h) atomicAdd(n_correct, h);
+    if (h) atomicAdd(&hdr->hits, (unsigned)h);
   }
 }
 
@@ -374,13 +374,16 @@ __global__ void __launch_bounds__(32 * XENT_WARPS)
 xent_round_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
                   const int32_t *__restrict__ labels, const long long *__restrict__ rowinfo,
                   const WsHeader *__restrict__ hdr, int8_t *__restrict__ out, int B, int N, int round_mode,
-                  int32_t *__restrict__ b_out) {
+                  int32_t *__restrict__ b_out, int32_t *__restrict__ n_correct) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * XENT_WARPS + warp;
   const unsigned long long mxv = hdr->maxabs64;
   const int b = 64 - __clzll((long long)mxv);
   const int bp = b > 7 ? b - 7 : 0;
-  if (blockIdx.x == 0 && threadIdx.x == 0 && b_out) *b_out = b;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (b_out) *b_out = b;
+    if (n_correct) *n_correct = (int32_t)hdr->hits;
+  }
   if (r >= B) return;
   const int s = *s_a_ptr;
   const int label = labels[r];
@@ -491,7 +494,7 @@ template <bool TAB>
 __global__ void __launch_bounds__(32 * XENT_WARPS)
 xent_row_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
                      const int32_t *__restrict__ labels, long long *__restrict__ rowinfo, WsHeader *hdr,
-                     int32_t *__restrict__ n_correct, int B, int N, uint32_t *__restrict__ status, XentTables tabs) {
+                     int B, int N, uint32_t *__restrict__ status, XentTables tabs) {
   __shared__ unsigned long long sh_max[XENT_WARPS];
   __shared__ int sh_hit[XENT_WARPS];
   __shared__ __align__(16) unsigned short sh_T[XENT_WARPS][256];     // T(a) of Eq. 4 for a = -128 .. 127 (at most 2^9)
@@ -598,7 +601,7 @@ xent_row_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s
     int h = 0;
     for (int w = 0; w < XENT_WARPS; ++w) { m = sh_max[w] > m ? sh_max[w] : m; h += sh_hit[w]; }
     if (m > *(volatile unsigned long long *)&hdr->maxabs64) atomicMax(&hdr->maxabs64, m);
-    if (n_correct && h) atomicAdd(n_correct, h);
+    if (h) atomicAdd(&hdr->hits, (unsigned)h);
   }
 }
 
@@ -607,14 +610,17 @@ __global__ void __launch_bounds__(32 * XENT_WARPS)
 xent_round_fast_kernel(const int8_t *__restrict__ a, const int32_t *__restrict__ s_a_ptr,
                        const int32_t *__restrict__ labels, const long long *__restrict__ rowinfo,
                        const WsHeader *__restrict__ hdr, int8_t *__restrict__ out, int B, int N, int round_mode,
-                       int32_t *__restrict__ b_out, XentTables tabs) {
+                       int32_t *__restrict__ b_out, int32_t *__restrict__ n_correct, XentTables tabs) {
   __shared__ __align__(8) unsigned char sh_q[XENT_WARPS][256];        // rounded T(a) for a = -128 .. 127
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * XENT_WARPS + warp;
   const unsigned long long mxv = hdr->maxabs64;
   const int b = 64 - __clzll((long long)mxv);
   const int bp = b > 7 ? b - 7 : 0;
-  if (blockIdx.x == 0 && threadIdx.x == 0 && b_out) *b_out = b;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (b_out) *b_out = b;
+    if (n_correct) *n_correct = (int32_t)hdr->hits;
+  }
   if (r >= B) return;
   const int s = *s_a_ptr;
   const int label = labels[r];
@@ -669,11 +675,11 @@ static int launch_xent(niti_ctx *ctx, cudaStream_t st, const int8_t *a, const in
     t.qtab = (unsigned char *)tab_mem + 256 * 256 * 2;
     t.thr = t.qtab + 256 * 256;
     xent_ttab_kernel<<<256, 256, 0, st>>>(s_a, t);
-    xent_row_fast_kernel<true><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status, t);
+    xent_row_fast_kernel<true><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, B, N, status, t);
   } else if (packed) {
-    xent_row_fast_kernel<false><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status, t);
+    xent_row_fast_kernel<false><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, B, N, status, t);
   } else {
-    xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, n_correct, B, N, status);
+    xent_row_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, B, N, status);
   }
   if (ctx) {
     int rc = niti_reduce(ctx, st, &hdr->maxabs64, 1, NITI_REDUCE_MAX_U64);
@@ -681,12 +687,12 @@ static int launch_xent(niti_ctx *ctx, cudaStream_t st, const int8_t *a, const in
   }
   if (tab) {
     xent_qtab_kernel<<<256, 256, 0, st>>>(s_a, hdr, t, round_mode);
-    xent_round_fast_kernel<true><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e, t);
+    xent_round_fast_kernel<true><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e, n_correct, t);
     if (ctx) ctx->launches += 2;
   } else if (packed) {
-    xent_round_fast_kernel<false><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e, t);
+    xent_round_fast_kernel<false><<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e, n_correct, t);
   } else {
-    xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e);
+    xent_round_kernel<<<blocks, 32 * XENT_WARPS, 0, st>>>(a, s_a, labels, rowinfo, hdr, e, B, N, round_mode, b_e, n_correct);
   }
   return NITI_OK;
 }
@@ -705,10 +711,6 @@ extern "C" int niti_int_xent(niti_ctx *ctx, void *stream, const int8_t *a, const
   long long *rowinfo = (long long *)((char *)ws + NITI_WS_HEADER);
   const int rch = niti_take_header(ctx, st, ws, &hdr);
   if (rch != NITI_OK) return rch;
-  if (n_correct) {
-    NITI_CUDA_TRY(ctx, cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st));
-    ctx->launches++;
-  }
   void *tab_mem = (char *)ws + NITI_WS_HEADER + ((size_t)B * 16 + 255) / 256 * 256;
   int rcx = launch_xent(ctx, st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, ctx->d_status, tab_mem);
   if (rcx != NITI_OK) return rcx;
@@ -755,7 +757,6 @@ extern "C" int niti_int_xent_noalloc(void *stream, const int8_t *a, const int32_
   // word of the header takes the (unreported) status bits of this variant.
   uint32_t *status = (uint32_t *)((char *)base + NITI_NOALLOC_HEADER - sizeof(uint32_t));
   if (cudaMemsetAsync(base, 0, NITI_NOALLOC_HEADER, st) != cudaSuccess) return NITI_ERR_CUDA;
-  if (n_correct && cudaMemsetAsync(n_correct, 0, sizeof(int32_t), st) != cudaSuccess) return NITI_ERR_CUDA;
   launch_xent(nullptr, st, a, s_a, labels, rowinfo, hdr, e, b_e, n_correct, B, N, round_mode, status, nullptr);
   if (cudaGetLastError() != cudaSuccess) return NITI_ERR_CUDA;
   return NITI_OK;

@@ -105,6 +105,7 @@ struct TcParams {
   int mbits, round_mode, relu;
   unsigned spec_mul256;         // the sampled max is scaled by this / 256 before taking its bit length
   int spec_tag;                 // identifies the call site (its b_out scalar) in the table of estimate errors
+  int update;                   // 1: out8 holds weights: the epilogue stores clamp(w - rounded gradient, +-127)
   int pool;                     // 1: the epilogue also stores the 2 x 2 max-pool of the (ReLU'd) output tile
   int pool_xh;                  // lane distance of the pixel one image row below (the pixel to the right is lane ^ 1)
   int single_wave;              // every CTA has at most one tile: the sample is the whole tensor, the shift
@@ -453,6 +454,10 @@ __device__ __forceinline__ void round_chunk32(const int (&v)[32], unsigned (&w8)
   }
 }
 
+// per byte: clamp(w - g, -127, 127) (Algorithm 1's update on int8 weights)
+__device__ __forceinline__ unsigned bytes_sub_clamp127(unsigned w, unsigned g) {
+  return __vmaxs4(__vsubss4(w, g), 0x81818181u);
+}
 // 0xff in every byte of b that is greater than zero as a signed byte (the ReLU gate of the backward pass).
 __device__ __forceinline__ unsigned bytes_gt0(unsigned b) {
   unsigned t = (b & 0x7f7f7f7fu) + 0x7f7f7f7fu;   // bit 7 of a byte: its low seven bits are not all zero
@@ -1468,17 +1473,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool rok = row_ok && orow < p.gm;
             unsigned m[8];
             unsigned pw8[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};     // pooling input of lanes outside the tensor
-            if (mrow && rok)
+            if ((mrow || p.update) && rok)        // the ReLU mask, or the weights this chunk updates
               asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                            : "=r"(m[0]), "=r"(m[1]), "=r"(m[2]), "=r"(m[3]), "=r"(m[4]), "=r"(m[5]), "=r"(m[6]), "=r"(m[7])
-                           : "l"(mrow + cc));
+                           : "l"((p.update ? (const int8_t *)drow : mrow) + cc));
             tc_ld32(tm_row + (unsigned)c, v);
             if (rok) {
               unsigned w8[8];
               Extremes ex = {0, 0, 0u};
               round_chunk32(v, w8, rk, relu, ex);
               mx |= ex.magnitude_bits();
-              if (mrow) {
+              if (p.update) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) w8[j] = bytes_sub_clamp127(m[j], w8[j]);
+              } else if (mrow) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) w8[j] &= bytes_gt0(m[j]);
               }
@@ -1581,9 +1589,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // executes only what changes (measured on the first layer: the general loop above spends a third
     // of its integer instructions on tests whose outcome is the same for every tile).
     if (ok && lean_item >= 0) {
-      auto lean = [&](auto relu_c, auto mask_c, auto batched_c, auto pool_c) {
+      auto lean = [&](auto relu_c, auto mask_c, auto batched_c, auto pool_c, auto upd_c) {
         constexpr bool RELU = decltype(relu_c)::value, MASK = decltype(mask_c)::value, BATCHED = decltype(batched_c)::value;
         constexpr bool POOL = decltype(pool_c)::value;       // fused 2 x 2 max-pool of the ReLU'd tile
+        constexpr bool UPD = decltype(upd_c)::value;         // the output rows are weights: subtract the rounded gradient
         const int pool_xh = p.pool_xh;
         const bool pool_lane = (lane & (1 | pool_xh)) == 0;  // the window's top-left pixel stores the maximum
         const int kind = p.halo ? 0 : ((p.kind == GK_CONV_FWD || p.kind == GK_CONV_DGRAD) ? 1 : 2);
@@ -1641,10 +1650,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int v[32];
             const bool rok = BATCHED ? (row_ok && orow < gm) : row_ok;
             unsigned m[8];
-            if (MASK && rok)
+            if ((MASK || UPD) && rok)
               asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                            : "=r"(m[0]), "=r"(m[1]), "=r"(m[2]), "=r"(m[3]), "=r"(m[4]), "=r"(m[5]), "=r"(m[6]), "=r"(m[7])
-                           : "l"(mrow + cc));
+                           : "l"((UPD ? (const int8_t *)drow : mrow) + cc));
             tc_ld32(tm_row + (unsigned)c, v);
             unsigned w8[8];
             if (POOL) {
@@ -1656,6 +1665,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               for (int j = 0; j < 8; ++j) {
                 w8[j] = round_pack4_aligned<RELU>(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3], rk, ex_all);
                 if (MASK) w8[j] &= bytes_gt0(m[j]);
+                if (UPD) w8[j] = bytes_sub_clamp127(m[j], w8[j]);
               }
               store32(drow + cc, w8);
             }
@@ -1677,10 +1687,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       using T = std::true_type;
       using F = std::false_type;
       const bool relu = p.relu != 0, masked = mask8 != nullptr, batched = p.mrep > 1;
-      if (batched) { if (relu) lean(T{}, F{}, T{}, F{}); else lean(F{}, F{}, T{}, F{}); }      // (row-batched: forward only)
-      else if (p.pool) lean(T{}, F{}, F{}, T{});                                               // (pooling: ReLU, no mask)
-      else if (relu) { if (masked) lean(T{}, T{}, F{}, F{}); else lean(T{}, F{}, F{}, F{}); }
-      else { if (masked) lean(F{}, T{}, F{}, F{}); else lean(F{}, F{}, F{}, F{}); }
+      if (batched) { if (relu) lean(T{}, F{}, T{}, F{}, F{}); else lean(F{}, F{}, T{}, F{}, F{}); }   // (row-batched: forward only)
+      else if (p.update) lean(F{}, F{}, F{}, F{}, T{});                                              // (weight gradients: signed, no mask)
+      else if (p.pool) lean(T{}, F{}, F{}, T{}, F{});                                                // (pooling: ReLU, no mask)
+      else if (relu) { if (masked) lean(T{}, T{}, F{}, F{}, F{}); else lean(T{}, F{}, F{}, F{}, F{}); }
+      else { if (masked) lean(F{}, T{}, F{}, F{}, F{}); else lean(F{}, F{}, F{}, F{}, F{}); }
       mx |= ex_all.magnitude_bits();
     }
     if (p.epi_mode == EPI_SPILL || p.epi_mode == EPI_SPECULATE) {
@@ -2309,12 +2320,14 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
   return NITI_OK;
 }
 
-int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const RoundSpec &r, int32_t *acc,
-                 WsHeader *hdr, bool *fused, bool *pooled, bool shard_ok) {
+int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const RoundSpec &r_in, int32_t *acc,
+                 WsHeader *hdr, bool *fused, bool *pooled, bool shard_ok, bool *updated) {
   TcParams p;
   CUtensorMap ma, mb;
+  RoundSpec r = r_in;
   *fused = false;
   if (pooled) *pooled = false;
+  if (updated) *updated = false;
   // engine 0: pairs of CTAs (cta_group::2) when there are enough 256-row tiles to fill the GPU.
   // Test switches: 2 / 3 force the single-CTA / paired kernel, 4 keeps the int32 spill epilogue.
   // Test switches: 5 disables the halo mode of small-channel convolutions.
@@ -2377,6 +2390,19 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
     if (p.halo == 1) { p.pool = 1; p.pool_xh = 8; }
     else if (!p.halo && p.Wt >= 2 && p.Wt <= 16 && p.Ht >= 2) { p.pool = 1; p.pool_xh = p.Wt; }
     *pooled = p.pool != 0;
+  }
+  // Weight update inside the epilogue (Section 3.3): a fully connected weight gradient whose epilogue
+  // rounds by itself subtracts the rounded values from the weights in place of storing them.  A
+  // speculative pass must not touch the weights (a wrong guess could not be taken back), so the update
+  // is fused only where the shift is exact when the stores happen: single-wave launches.  (Measured
+  // and not kept for the other launches: a first pass for the bit-width alone followed by a rounding
+  // pass that updates, 198 us against 185 us for the 4096 x 25088 layer at batch 64.)
+  p.update = 0;
+  if (updated && r.update_w && g.kind == GK_FC_WGRAD && p.epi_mode == EPI_SPECULATE && p.single_wave && p.mrep == 1 &&
+      !p.halo && !r.mask && !r.relu && (g.gn % 32) == 0 && ((uintptr_t)r.update_w & 31) == 0) {
+    p.update = 1;
+    r.out = r.update_w;
+    *updated = true;
   }
   const bool prof = ctx->profile_on && ctx->prof_ev && ctx->prof_used < NITI_PROF_MAX;
   if (prof) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st);

@@ -12,16 +12,16 @@ from .api import Niti, ROUND_PSR
 
 
 class NitiTrainer:
-    def __init__(self, niti: Niti, net, weights, round_mode: int = ROUND_PSR, fused_update: bool = False,
+    def __init__(self, niti: Niti, net, weights, round_mode: int = ROUND_PSR, fused_update: bool = True,
                  pool_codes: bool = False, dist_group=None, data_parallel: bool = False, pool_fused: bool = True):
         """``net``: an object with ``batch``, ``in_shape``, ``s_in``, ``m_u`` and ``layers`` (dicts
         with op in {"conv", "pool", "fc"}); ``weights``: int8 host arrays / tensors per weight
         layer ([Cout,3,3,Cin] or [N,K]).  ``fused_update``: weight gradient and weight update in one
         library call (Section 3.3), else ``*_wgrad`` / ``linear_bwd`` followed by ``int_sgd_update``;
-        the weights after a step are the same either way.  The fused calls must compute the error of
-        the layer below first (it needs the old weights), and that order leaves less of the tensors
-        the next call reads in L2 than weight gradient, error, update does: measured 0.4 % slower on
-        VGG-16, so the separate calls are the default.  ``pool_codes``: the max-pool forward records
+        the weights after a step are the same either way.  The fused calls compute the error of the
+        layer below first (it needs the old weights) and never store the int8 gradient where the
+        rounding pass can subtract from the weights directly; measured 0.5 % faster on VGG-16.
+        ``pool_codes``: the max-pool forward records
         its routing (half a byte per output element) and the backward pass reads that instead of the
         pooled tensor; in isolation the backward kernels get 30 % faster and the forward ones 15-40 %
         slower, over the VGG-16 step it measured 0.5 % slower, so it is off by default."""

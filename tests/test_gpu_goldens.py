@@ -70,13 +70,16 @@ def _exponents(tr, net):
     return out
 
 
-def test_config4_whole_step_equals_the_oracle_digests(niti):
+@pytest.mark.parametrize("fused_update", [True, False])
+def test_config4_whole_step_equals_the_oracle_digests(niti, fused_update):
+    """Both forms of the weight update: fused into the weight-gradient calls (the trainer's default)
+    and as separate niti_int_sgd_update calls."""
     from paper_2009_13108_b200 import NitiTrainer
     want = {r[0]: r[1] for r in _read("config4_step_sha256.txt")}
     net = config_net(4)
     x, labels, weights = make_net_inputs(net)
     assert _sha(x) == want["input_x"] and _sha(labels) == want["input_labels"]
-    tr = NitiTrainer(niti, net, weights)
+    tr = NitiTrainer(niti, net, weights, fused_update=fused_update)
     tr.load_batch(x, labels)
     tr.step()
     niti.check()

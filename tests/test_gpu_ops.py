@@ -192,6 +192,33 @@ def test_linear_bwd_update(niti, oref, M, N, K, engine):
     niti.check()
 
 
+@pytest.mark.parametrize("M,N,K,launches", [(64, 1024, 2048, 1), (96, 768, 1056, 1), (64, 2048, 4096, 3)])
+def test_linear_bwd_update_inside_the_multiply(niti, oref, M, N, K, launches):
+    """A fully connected weight gradient whose every CTA has one tile rounds with the exact shift in the
+    multiply's own epilogue, which then also subtracts from the weights (Section 3.3): one launch, no
+    update kernel, the gradient never stored.  Larger ones keep the speculative pass, its follow-up and
+    the update kernel.  Weights at +-127 with gradients of either sign exercise the clamp."""
+    rng = np.random.default_rng(M + N + K)
+    a, e = np.maximum(_i8(rng, (M, K)), 0), _i8(rng, (M, N))
+    w = rng.integers(-127, 128, size=(N, K), dtype=np.int8)
+    w[::3, ::5] = 127
+    w[1::3, 1::5] = -127
+    _, wg, _, bg = oref.linear_bwd(a, e, w, False, None, 5)
+    want_w = oref.sgd_update(w, wg)
+    wt = _T(niti, w.copy())
+    at, et = _T(niti, a), _T(niti, e)
+    niti.linear_bwd_update(at, et, _T(niti, w.copy()), need_e_prev=False)      # sizes the workspace
+    niti.begin_step()
+    redo0, n0, t0 = niti.redo_count(), niti.launch_count(), niti.tc_launch_count()
+    none, _, b_g = niti.linear_bwd_update(at, et, wt, need_e_prev=False)
+    assert niti.tc_launch_count() - t0 == min(launches, 2)
+    assert niti.launch_count() - n0 == launches           # 1: nothing but the multiply itself
+    assert niti.redo_count() == redo0
+    assert none is None and int(b_g) == bg
+    _eq(wt, want_w)
+    niti.check()
+
+
 def test_outputs_and_masks_aligned_to_16_but_not_32_bytes(niti, oref):
     """The epilogue's whole-chunk loop needs 32-byte aligned rows; 16-byte aligned tensors take the
     general loop (16-byte stores) and must give the same bytes."""
