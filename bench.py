@@ -458,6 +458,7 @@ def run_ours(args):
     import numpy as np
     from paper_2009_13108_b200 import Niti, NitiTrainer
     from paper_2009_13108_b200.build import CSRC
+    from paper_2009_13108_b200 import build as _lib_build
     from synth import config_net, make_net_inputs, make_step_batch
 
     niti = Niti(local)
@@ -653,6 +654,8 @@ def run_ours(args):
                    "parallelism": "replicas" if world > 1 else "single",
                    "inputs_sha256_16": input_digests},
         "outputs": out_digests,
+        "library": {"sources_sha256_16": _lib_build.source_digest()[:16],
+                    "built_from_these_sources": _lib_build.built_from_current_sources()},
         "step_tops": ops_step / (ms / args.steps) / 1e9,
         "clocks": clocks,
         "e2e": {"value": images / (ms_e2e / 1e3), "unit": UNIT, "h2d_bytes_per_step": int(xh.numel() + lh.numel() * 4),

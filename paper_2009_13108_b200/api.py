@@ -46,6 +46,13 @@ def load_library():
     """Loads the built shared library; raises if it has not been built (no fallback exists)."""
     if not os.path.exists(_LIB_PATH):
         raise NitiError(ERR_CUDA, "%s is missing: run paper_2009_13108_b200/build.py" % _LIB_PATH)
+    if os.path.dirname(_LIB_PATH) == _HERE:
+        from .build import built_from_current_sources
+        if built_from_current_sources() is False:
+            import warnings
+            warnings.warn("libniti_b200.so was built from other sources than the ones in csrc/: "
+                          "run `python __graft_entry__.py` (or paper_2009_13108_b200/build.py) to rebuild it",
+                          RuntimeWarning, stacklevel=2)
     lib = C.CDLL(_LIB_PATH)
     vp, i32, i64, sz = C.c_void_p, C.c_int, C.c_int64, C.c_size_t
     lib.niti_create.argtypes = [C.POINTER(vp), i32]

@@ -34,6 +34,14 @@ def test_library_exports_every_declared_symbol(lib_path):
         assert hasattr(lib, name), name
 
 
+def test_library_is_built_from_the_sources_in_the_tree(lib_path):
+    """build() records the digest of the sources next to the binary and rebuilds when they differ; the
+    binding warns when it loads a library built from other sources."""
+    from paper_2009_13108_b200 import build
+    assert build.built_from_current_sources() is True
+    assert len(build.source_digest()) == 64
+
+
 def test_binding_lists_the_same_names(lib_path):
     from paper_2009_13108_b200 import api
     assert sorted(api.EXPORTS) == _declared()
