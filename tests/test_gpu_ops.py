@@ -219,6 +219,42 @@ def test_linear_bwd_update_inside_the_multiply(niti, oref, M, N, K, launches):
     niti.check()
 
 
+def test_header_slots_of_a_step(oref):
+    """niti_begin_step clears 64 header slots at once and the following calls take one each; the 65th
+    and later calls, and calls after the workspace has been replaced by a larger one, clear their own
+    header again.  The results never change, and no call of the first 64 enqueues a memset."""
+    from paper_2009_13108_b200 import Niti
+    niti = Niti(0)                                               # (its own, small workspace)
+    rng = np.random.default_rng(64)
+    M, N, K = 48, 96, 160
+    a, w = _i8(rng, (M, K)), _i8(rng, (N, K))
+    want, s_want, b_want = oref.linear_fwd(a, -7, w, -9, True)
+    at, wt = _T(niti, a), _T(niti, w)
+    sa, sw = niti.scalar(-7), niti.scalar(-9)
+    niti.linear_fwd(at, sa, wt, sw, relu=True)                   # sizes the workspace
+    niti.begin_step()
+    per_call = []
+    for i in range(70):
+        n0 = niti.launch_count()
+        out, s_out, b_out = niti.linear_fwd(at, sa, wt, sw, relu=True)
+        per_call.append(niti.launch_count() - n0)
+        _eq(out, want)
+        assert (int(s_out), int(b_out)) == (s_want, b_want), i
+    assert len(set(per_call[:64])) == 1 and per_call[64] == per_call[0] + 1 and per_call[69] == per_call[64]
+    # a larger workspace replaces the prepared one: its headers were never cleared by begin_step
+    niti.begin_step()
+    M2, N2, K2 = 256, 512, 384
+    a2, w2 = _i8(rng, (M2, K2)), _i8(rng, (N2, K2))
+    want2, s2, b2 = oref.linear_fwd(a2, -7, w2, -9, False)
+    out2, s_out2, b_out2 = niti.linear_fwd(_T(niti, a2), sa, _T(niti, w2), sw)
+    _eq(out2, want2)
+    assert (int(s_out2), int(b_out2)) == (s2, b2)
+    out, s_out, b_out = niti.linear_fwd(at, sa, wt, sw, relu=True)
+    _eq(out, want)
+    niti.check()
+    niti.close()
+
+
 def test_outputs_and_masks_aligned_to_16_but_not_32_bytes(niti, oref):
     """The epilogue's whole-chunk loop needs 32-byte aligned rows; 16-byte aligned tensors take the
     general loop (16-byte stores) and must give the same bytes."""
