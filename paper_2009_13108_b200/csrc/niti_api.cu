@@ -32,6 +32,7 @@ extern "C" int niti_create(niti_ctx **out, int device) {
     return NITI_ERR_SHAPE;
   }
   ctx->sm_count = prop.multiProcessorCount;
+  ctx->smem_optin = prop.sharedMemPerBlockOptin;
   // one allocation: the status words, then the table of speculative-estimate errors
   const size_t dev_bytes = 256 + sizeof(int32_t) * 2 * NITI_SPEC_SLOTS;
   e = cudaMalloc(&ctx->d_status, dev_bytes);

@@ -46,6 +46,10 @@ struct niti_ctx {
   // CTA pairs (0 = not asked yet) and the dynamic shared-memory limit already set on the kernel
   int tc_units[3];
   size_t tc_attr_smem[3];
+  // the device's opt-in limit of dynamic shared memory per CTA.  The limit set on a kernel belongs to the
+  // device, not to a context: every context therefore sets this same value (a context that set only what it
+  // needed would lower the limit under another context of the process)
+  size_t smem_optin;
 };
 
 

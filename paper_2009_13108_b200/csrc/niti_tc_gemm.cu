@@ -1927,8 +1927,10 @@ static bool plan(niti_ctx *ctx, const GemmProblem &g, int ctas, bool want_halo, 
         p.bn = Cn >= 256 ? 256 : round_up32(Cn);
         if (ctas == 2 && Cn > 256) {
           // Whole waves: with 256-wide tiles the 14 x 14 layers are 98 tile pairs on 74 pairs of SMs, two
-          // waves of which the second is a third full; 192-wide tiles make 147 items, two full waves
-          // of items that each take three quarters of the time.
+          // waves of which the second is a third full; 192-wide tiles make 147 items, two full waves.
+          // (A 192-wide MMA takes as long as a 256-wide one, so an item is not shorter; it moves three
+          // quarters of the weights.  Measured 31.0 against 31.5 us; 128-wide tiles, three waves of
+          // half the math each, are bound by the shared-memory traffic of their operands: 38.4 us.)
           const long long mu = ((long long)p.w_tiles * p.h_tiles * p.b_tiles + 1) / 2, units = ctx->sm_count / 2;
           const long long w256 = (mu * ((Cn + 255) / 256) + units - 1) / units;
           const long long w192 = (mu * ((Cn + 191) / 192) + units - 1) / units;
@@ -2226,6 +2228,18 @@ int niti_tc_timeout_probe(niti_ctx *ctx, cudaStream_t st) {
 // CTAs (CTAS = 1) or CTA pairs (CTAS = 2) that can be resident at the same time.  SMs pair up inside a
 // GPC, so the number of pairs can be below sm_count / 2; a persistent grid larger than that would run
 // a second, short wave.
+// Dynamic shared-memory limit of the kernel: once per context, and always the most the device allows
+// beside the kernel's static shared memory (see niti_ctx::smem_optin for why not "what this launch needs").
+template <int CTAS>
+static int tc_set_smem_limit(niti_ctx *ctx) {
+  cudaFuncAttributes fa;
+  NITI_CUDA_TRY(ctx, cudaFuncGetAttributes(&fa, tc_gemm_kernel<CTAS>));
+  const size_t limit = ctx->smem_optin > fa.sharedSizeBytes ? ctx->smem_optin - fa.sharedSizeBytes : 0;
+  NITI_CUDA_TRY(ctx, cudaFuncSetAttribute(tc_gemm_kernel<CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit));
+  ctx->tc_attr_smem[CTAS] = limit;
+  return NITI_OK;
+}
+
 template <int CTAS>
 static int tc_units(niti_ctx *ctx) {
   int &cached = ctx->tc_units[CTAS];
@@ -2244,9 +2258,7 @@ static int tc_units(niti_ctx *ctx) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaFuncSetAttribute(tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 201 * 1024) == cudaSuccess &&
-        ctx->tc_attr_smem[2] < 201 * 1024)
-      ctx->tc_attr_smem[2] = 201 * 1024;
+    (void)tc_set_smem_limit<2>(ctx);
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, tc_gemm_kernel<2>, &cfg) == cudaSuccess && n > 0 && n < cached) cached = n;
     else (void)cudaGetLastError();
@@ -2260,10 +2272,11 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
   size_t smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + (size_t)p.b_res_bytes + 1024;
   if (p.stg_off > 0) smem = (size_t)p.stg_off + (size_t)EPI_WARPS * 32 * 33 * 4 + 1024;
   size_t &attr_smem = ctx->tc_attr_smem[CTAS];
-  if (smem > attr_smem) {
-    NITI_CUDA_TRY(ctx, cudaFuncSetAttribute(tc_gemm_kernel<CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_smem = smem;
+  if (!attr_smem) {
+    const int rcs = tc_set_smem_limit<CTAS>(ctx);
+    if (rcs != NITI_OK) return rcs;
   }
+  if (smem > attr_smem) return niti_fail(ctx, NITI_ERR_SHAPE, "tensor-core kernel: stage buffers exceed the shared memory of an SM");
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3((unsigned)(ctx->sm_count / CTAS * CTAS), 1, 1);

@@ -219,6 +219,26 @@ def test_linear_bwd_update_inside_the_multiply(niti, oref, M, N, K, launches):
     niti.check()
 
 
+def test_two_contexts_on_one_device(niti, oref):
+    """The shared-memory limit of a kernel belongs to the device: a second context whose first launch
+    needs little must not lower it under a context that launches with more."""
+    from paper_2009_13108_b200 import Niti
+    rng = np.random.default_rng(5)
+    big = (_i8(rng, (512, 1024)), _i8(rng, (512, 1024)))             # 8 stages of 32 KB
+    small = (_i8(rng, (16, 32)), _i8(rng, (32, 32)))                 # two small stages
+    want_big = oref.linear_fwd(big[0], -7, big[1], -9, False)
+    want_small = oref.linear_fwd(small[0], -7, small[1], -9, False)
+    sa, sw = niti.scalar(-7), niti.scalar(-9)
+    _eq(niti.linear_fwd(_T(niti, big[0]), sa, _T(niti, big[1]), sw)[0], want_big[0])
+    other = Niti(0)
+    _eq(other.linear_fwd(_T(other, small[0]), other.scalar(-7), _T(other, small[1]), other.scalar(-9))[0], want_small[0])
+    _eq(niti.linear_fwd(_T(niti, big[0]), sa, _T(niti, big[1]), sw)[0], want_big[0])
+    _eq(other.linear_fwd(_T(other, big[0]), other.scalar(-7), _T(other, big[1]), other.scalar(-9))[0], want_big[0])
+    other.check()
+    other.close()
+    niti.check()
+
+
 def test_header_slots_of_a_step(oref):
     """niti_begin_step clears 64 header slots at once and the following calls take one each; the 65th
     and later calls, and calls after the workspace has been replaced by a larger one, clear their own
