@@ -2333,6 +2333,17 @@ static int launch_tc(niti_ctx *ctx, cudaStream_t st, const TcParams &p, const CU
   return NITI_OK;
 }
 
+// Profiling event of a launch.  On a stream that is being captured the record becomes an event-record
+// node of the graph (cudaEventRecordExternal), so that every replay of the graph times its launches
+// where they run; a plain record there would only add a dependency.
+static void prof_record(cudaEvent_t ev, cudaStream_t st) {
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusActive)
+    cudaEventRecordWithFlags(ev, st, cudaEventRecordExternal);
+  else
+    cudaEventRecord(ev, st);
+}
+
 int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const RoundSpec &r_in, int32_t *acc,
                  WsHeader *hdr, bool *fused, bool *pooled, bool shard_ok, bool *updated) {
   TcParams p;
@@ -2418,7 +2429,7 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
     *updated = true;
   }
   const bool prof = ctx->profile_on && ctx->prof_ev && ctx->prof_used < NITI_PROF_MAX;
-  if (prof) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st);
+  if (prof) prof_record(ctx->prof_ev[2 * ctx->prof_used], st);
   int rc = p.ctas == 2 ? launch_tc<2>(ctx, st, p, ma, mb, acc, hdr, r) : launch_tc<1>(ctx, st, p, ma, mb, acc, hdr, r);
   if (rc != NITI_OK) return rc;
   if (p.epi_mode == EPI_SPECULATE && p.single_wave) {
@@ -2435,7 +2446,7 @@ int niti_tc_gemm(niti_ctx *ctx, cudaStream_t st, const GemmProblem &g, const Rou
     *fused = true;
   }
   if (prof) {
-    cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st);
+    prof_record(ctx->prof_ev[2 * ctx->prof_used + 1], st);
     ctx->prof_ops[ctx->prof_used] = 2.0 * (double)g.gm * (double)g.gn * (double)g.gk;
     ctx->prof_used++;
   }
