@@ -117,3 +117,36 @@ def test_random_convolutions(niti, oref, seed):
         finally:
             niti.set_engine(0)
     niti.check()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_multi_wave_convolutions(niti, oref, seed):
+    """Medium 3 x 3 layers with more tiles than SMs (speculative shift over several waves, CTA pairs or
+    the resident-weights mode, the fused pooling, the fused update), drawn like the ones above."""
+    rng = np.random.default_rng(3000 + seed)
+    Ci = int(rng.choice([64, 128, 192, 256]))
+    Co = int(rng.choice([64, 128, 256, 320]))
+    H = int(rng.choice([20, 28, 36, 44])) + 2 * int(rng.integers(0, 4))
+    W = int(rng.choice([24, 32, 40, 56])) + 2 * int(rng.integers(0, 4))
+    B = int(rng.choice([8, 12, 16]))
+    kind = seed % 3
+    x, w = _draw(rng, (B, H, W, Ci), kind), _draw(rng, (Co, 3, 3, Ci), 0)
+    e = _draw(rng, (B, H, W, Co), kind)
+    xm = np.maximum(x, 0)
+    tag = "conv B=%d H=%d W=%d Ci=%d Co=%d kind=%d" % (B, H, W, Ci, Co, kind)
+    wy, s, b = oref.conv_fwd(xm, -7, w, -9, 1, True)
+    wp = oref.maxpool2_fwd(wy)
+    y, y_pool, s_y, b_y = niti.conv_fwd_pool(_T(niti, xm), niti.scalar(-7), _T(niti, w), niti.scalar(-9))
+    _eq(y, wy, tag + " fwd")
+    _eq(y_pool, wp, tag + " pooled")
+    assert (int(s_y), int(b_y)) == (s, b), tag
+    wd, bd = oref.conv_dgrad(e, w, (H, W), 1, xm)
+    ep, b_e = niti.conv_dgrad(_T(niti, e), _T(niti, w), (H, W), relu_mask_src=_T(niti, xm))
+    _eq(ep, wd, tag + " dgrad")
+    assert int(b_e) == bd, tag
+    wg, bg = oref.conv_wgrad(xm, e, (3, 3), 1, 5)
+    wt = _T(niti, w.copy())
+    _, b_g = niti.conv_wgrad_update(_T(niti, xm), _T(niti, e), wt)
+    _eq(wt, oref.sgd_update(w, wg), tag + " update")
+    assert int(b_g) == bg, tag
+    niti.check()
