@@ -150,3 +150,58 @@ def test_random_multi_wave_convolutions(niti, oref, seed):
     _eq(wt, oref.sgd_update(w, wg), tag + " update")
     assert int(b_g) == bg, tag
     niti.check()
+
+
+DEGENERATE_CONVS = [
+    # B, H, W, Ci, Co, R, pad, stride
+    (1, 1, 1, 64, 64, 3, 1, 1),        # one pixel: only the centre tap sees data
+    (3, 1, 40, 32, 64, 3, 1, 1),       # one image row
+    (2, 37, 1, 64, 32, 3, 1, 1),       # one image column
+    (1, 2, 2, 128, 128, 3, 1, 1),
+    (5, 3, 3, 256, 256, 3, 0, 1),      # unpadded 3 x 3 on 3 x 3: a single output pixel per image
+    (1, 7, 7, 512, 512, 7, 0, 1),      # the filter covers the whole image
+    (4, 9, 9, 32, 32, 1, 0, 2),        # pointwise, stride 2
+    (2, 10, 6, 16, 16, 5, 4, 3),       # padding larger than the data it frames
+]
+
+
+@pytest.mark.parametrize("B,H,W,Ci,Co,R,pad,stride", DEGENERATE_CONVS)
+def test_degenerate_convolution_extents(niti, oref, B, H, W, Ci, Co, R, pad, stride):
+    rng = np.random.default_rng(B + 3 * H + 5 * W + Ci + Co + R)
+    Ho, Wo = oref.conv_out_hw(H, W, R, R, pad, stride)
+    x, w, e = _draw(rng, (B, H, W, Ci), 0), _draw(rng, (Co, R, R, Ci), 0), _draw(rng, (B, Ho, Wo, Co), 0)
+    xm = np.maximum(x, 0)
+    tag = "conv B=%d H=%d W=%d Ci=%d Co=%d R=%d pad=%d stride=%d" % (B, H, W, Ci, Co, R, pad, stride)
+    for engine in (0, 1):
+        niti.set_engine(engine)
+        try:
+            wy, s, b = oref.conv_fwd(xm, -7, w, -9, pad, False, stride=stride)
+            y, s_y, b_y = niti.conv_fwd(_T(niti, xm), niti.scalar(-7), _T(niti, w), niti.scalar(-9), pad=pad,
+                                        stride=stride)
+            _eq(y, wy, tag + " fwd")
+            assert (int(s_y), int(b_y)) == (s, b), tag
+            wd, bd = oref.conv_dgrad(e, w, (H, W), pad, None, stride=stride)
+            ep, b_e = niti.conv_dgrad(_T(niti, e), _T(niti, w), (H, W), pad=pad, stride=stride)
+            _eq(ep, wd, tag + " dgrad")
+            assert int(b_e) == bd, tag
+            wg, bg = oref.conv_wgrad(xm, e, (R, R), pad, 5, stride=stride)
+            g, b_g = niti.conv_wgrad(_T(niti, xm), _T(niti, e), (R, R), pad=pad, stride=stride)
+            _eq(g, wg, tag + " wgrad")
+            assert int(b_g) == bg, tag
+        finally:
+            niti.set_engine(0)
+    niti.check()
+
+
+def test_largest_class_count_of_the_loss(niti, oref):
+    """niti_int_xent takes up to 65536 classes; both cases of Section 3.5 on such rows."""
+    rng = np.random.default_rng(65536)
+    B, N = 3, 65536
+    a = _draw(rng, (B, N), 0)
+    labels = np.array([0, N - 1, 12345], dtype=np.int32)
+    for s_a in (-9, -3):
+        want_e, want_b, want_nc = oref.int_xent(a, s_a, labels, 0)
+        e, b_e, n_correct = niti.int_xent(_T(niti, a), niti.scalar(s_a), _T(niti, labels))
+        _eq(e, want_e, "xent s_a=%d" % s_a)
+        assert (int(b_e), int(n_correct)) == (want_b, want_nc)
+    niti.check()
