@@ -377,9 +377,11 @@ def run_per_launch(args):
     wl = [(i, l) for i, l in enumerate(net.layers) if l["op"] != "pool"]
     names = ["fwd   L%d %s" % (i, l["op"]) for i, l in wl]
     for i, l in reversed(wl):
-        names.append("wgrad L%d %s" % (i, l["op"]))
+        # (the fused-update calls compute the error of the layer below first: it needs the old weights)
+        pair = ["wgrad L%d %s" % (i, l["op"])]
         if i != wl[0][0]:
-            names.append("dgrad L%d %s" % (i, l["op"]))
+            pair.append("dgrad L%d %s" % (i, l["op"]))
+        names += reversed(pair) if tr.fused_update else pair
     print("eager step %.3f ms, second passes in the step: %d" % (e0.elapsed_time(e1), niti.redo_count() - redo0))
     total = 0.0
     for k, (ms, ops) in enumerate(launches):
